@@ -1,0 +1,134 @@
+/* preserve_b200 — load anticipator and load-aware request router on one B200 (sm_100a).
+ *
+ * C ABI of the library.  The operations are those of PreServe's prediction-based
+ * management, Sec. 4.3.1 "Instance Load Anticipator" and Sec. 4.3.3 "Load-aware
+ * Request Router" of the paper (arXiv 2504.03702).
+ *
+ * Conventions for every entry point
+ *   - Pointers named d_* are DEVICE pointers owned by the caller.  The library never
+ *     frees, reallocates or keeps them after the call's work has run on the stream.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls enqueue work on that stream and return without synchronising, unless
+ *     stated otherwise.  One context serves one stream at a time; calls on one
+ *     context are not thread-safe.
+ *   - Return value: PRE_OK (0) or a negative pre_error.  Argument errors are found on
+ *     the host before anything is launched.  Errors that only the device can see
+ *     (malformed request fields, a full request table, a wait that ran out) are
+ *     recorded in a device status word that pre_status() reads; the kernels skip the
+ *     offending item and never write out of bounds or trap.
+ *
+ * Data layout
+ *   - Request table, structure of arrays, int32 each, capacity max_requests:
+ *       prompt[r]    P  prompt tokens            (0 <= P,  P + g < 2^28)
+ *       generated[r] g  tokens generated so far  (g >= 0)
+ *       predicted[r] D  predicted response tokens (D >= 1, D - g < 2^28)
+ *       instance[r]     instance the request runs on, in [0, n_instances)
+ *     A request with g >= D has finished; it stays in the table as a tombstone and
+ *     contributes nothing.  Any other violation is a malformed request: it is skipped
+ *     and PRE_EBADREQ is recorded.
+ *   - curves: int64[n_instances * horizon], row-major, 16-byte aligned.  curves[i*H + j]
+ *     is the anticipated number of KV tokens held by instance i at j decode iterations
+ *     from now: the paper's load-look-ahead map entry U_j times the capacity M,
+ *     restricted to the next H = l iterations.
+ *   - queued_p, current_d: int64[n_instances]; the router's "queued tokens to be
+ *     prefilled" and "tokens still to be generated" per instance (Sec. 4.3.3).
+ */
+#ifndef PRESERVE_B200_H
+#define PRESERVE_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pre_error {
+    PRE_OK = 0,
+    PRE_EINVAL = -1,    /* null or misaligned pointer, size out of range, bad config        */
+    PRE_ECAPACITY = -2, /* request table full: the arrivals that did not fit were not routed */
+    PRE_EBADREQ = -3,   /* a malformed request or arrival was skipped                        */
+    PRE_ETIMEOUT = -4,  /* a bounded device-side wait ran out; the batch was abandoned       */
+    PRE_ECUDA = -5,     /* a CUDA runtime call failed (see pre_last_cuda_error)              */
+    PRE_ENOMEM = -6     /* scratch allocation failed in pre_create                           */
+} pre_error;
+
+typedef struct pre_ctx pre_ctx; /* opaque; owns only internal device scratch */
+
+typedef struct pre_config {
+    int32_t n_instances;     /* I >= 1 */
+    int32_t horizon;         /* H >= 1: look-ahead window in decode iterations (the paper's l);
+                                at most 16384 */
+    int64_t capacity_tokens; /* M >= 1: KV token capacity of one instance (Sec. 4.3.1) */
+    double t_mem;            /* T_mem, ideal memory usage; 0.8 in the paper (Sec. 4.3.3) */
+    double beta;             /* penalty coefficient; 1.0 in the paper (Sec. 4.3.3) */
+    int64_t max_requests;    /* capacity of the request table arrays, >= 1, < 2^31 */
+} pre_config;
+
+/* Creates a context on the current CUDA device and allocates its scratch
+ * (8 bytes per table slot plus O(I) words).  *out is set only on success. */
+int pre_create(const pre_config* cfg, pre_ctx** out);
+
+/* Frees the scratch.  The caller must have synchronised the stream first. */
+int pre_destroy(pre_ctx* ctx);
+
+/* Load-look-ahead maps from the request table (Sec. 4.3.1: for a request with P prompt
+ * and D predicted response tokens, U'_i = (U_i*M + (P + i))/M for i in [0, D)).
+ * A request that has generated g tokens is that ramp seen g iterations later, so
+ *     curves[i][j] = sum over live requests r of instance i with j < D_r - g_r
+ *                    of (P_r + g_r + j),          0 <= j < H,
+ *     current_d[i] = sum over live requests r of instance i of (D_r - g_r).
+ * Overwrites d_curves (I*H) and d_current_d (I).  n_requests is a host value,
+ * 0 <= n_requests <= max_requests.  The request arrays are only read. */
+int pre_anticipate(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated,
+                   const int32_t* d_predicted, const int32_t* d_instance, int64_t n_requests,
+                   int64_t* d_curves, int64_t* d_current_d, void* stream);
+
+/* Routes n_arrivals requests in array order (Sec. 4.3.3).  For arrival (P, D) and every
+ * instance i the anticipator "virtually" adds the request to the map and takes the peak
+ * over the window,
+ *     peak_i = max over j in [0,H) of curves[i][j] + (j < min(D,H) ? P + j : 0),
+ *     L_i = (queued_p[i] + P) + (current_d[i] + D) + beta * max(0, peak_i - t_mem*M),
+ * evaluated in binary64 with each operation rounded separately (no fused multiply-add);
+ * the arrival goes to argmin_i L_i, the lowest index among equal scores.  The chosen
+ * instance then really receives it, before the next arrival is scored:
+ *     curves[i*][j] += P + j for j < min(D,H); queued_p[i*] += P; current_d[i*] += D;
+ *     (P, 0, D, i*) is appended to the request table at index *d_n_requests, which advances.
+ * d_choice[k] (int32) receives i*, or -1 if arrival k was malformed (P < 0, D < 1, either
+ * >= 2^28) or did not fit in the table; d_score[k] (binary64, may be NULL) the winning L.
+ * *d_n_requests is a DEVICE int64, read at the start and written at the end of the batch. */
+int pre_route_batch(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted,
+                    int64_t n_arrivals, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
+                    int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                    int64_t* d_n_requests, int32_t* d_choice, double* d_score, void* stream);
+
+/* One decode iteration (iteration-level batching, Sec. 2; the map covers "the next
+ * iterations", Sec. 4.3.1).  Every live request generates one token (g += 1; it becomes a
+ * tombstone when g reaches D); every map moves one iteration closer,
+ *     curves'[i][j] = curves[i][j+1] for j < H-1,
+ *     curves'[i][H-1] = sum over requests of i with D - g' >= H of (P + g' + H - 1), g' = g + 1;
+ * current_d[i] drops by the number of requests of i that were live; queued_p[i] becomes 0
+ * (every queued prefill is taken to finish within the iteration).  *d_n_requests (DEVICE
+ * int64) is only read.  Afterwards pre_anticipate on the table reproduces d_curves. */
+int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted,
+             int32_t* d_instance, const int64_t* d_n_requests, int64_t* d_curves,
+             int64_t* d_queued_p, int64_t* d_current_d, void* stream);
+
+/* Synchronises `stream`, then returns and clears the device status: the most severe of
+ * PRE_ETIMEOUT, PRE_ECAPACITY, PRE_EBADREQ recorded since the last call, PRE_ECUDA if the
+ * stream reports a CUDA error, else PRE_OK. */
+int pre_status(pre_ctx* ctx, void* stream);
+
+/* The cudaError_t value of the last failed runtime call on this context (0 if none). */
+int pre_last_cuda_error(const pre_ctx* ctx);
+
+/* Static, human-readable text for a pre_error value. */
+const char* pre_strerror(int code);
+
+/* Launch geometry chosen for this context, for reports: number of thread blocks of the
+ * persistent routing kernel and instance rows per build tile.  Either pointer may be NULL. */
+int pre_query(const pre_ctx* ctx, int32_t* route_blocks, int32_t* tile_rows);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRESERVE_B200_H */

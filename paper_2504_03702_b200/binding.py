@@ -1,0 +1,124 @@
+"""ctypes binding of libpreserve_b200.so: argument marshalling only.
+
+Every function has the name and the argument order of its C declaration in
+include/preserve_b200.h.  Tensors are passed as device pointers; the stream is torch's
+current stream.  There is no fallback: if the library is missing, importing fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpreserve_b200.so")
+
+PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENOMEM = 0, -1, -2, -3, -4, -5, -6
+
+EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
+           "pre_last_cuda_error", "pre_strerror", "pre_query")
+
+
+class pre_config(C.Structure):
+    _fields_ = [("n_instances", C.c_int32), ("horizon", C.c_int32), ("capacity_tokens", C.c_int64),
+                ("t_mem", C.c_double), ("beta", C.c_double), ("max_requests", C.c_int64)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2504_03702_b200.build` "
+            "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i64 = C.c_void_p, C.c_int64
+    lib.pre_create.argtypes = [C.POINTER(pre_config), C.POINTER(vp)]
+    lib.pre_destroy.argtypes = [vp]
+    lib.pre_anticipate.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.pre_route_batch.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.pre_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.pre_status.argtypes = [vp, vp]
+    lib.pre_last_cuda_error.argtypes = [vp]
+    lib.pre_strerror.argtypes = [C.c_int]
+    lib.pre_strerror.restype = C.c_char_p
+    lib.pre_query.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    for name in EXPORTS:
+        if name != "pre_strerror":
+            getattr(lib, name).restype = C.c_int
+    return lib
+
+
+lib = _load()
+
+
+class PreError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {pre_strerror(code)} ({code})")
+
+
+def _ptr(t):
+    """Device (or host) address of a tensor, None -> NULL, int passes through."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def pre_strerror(code: int) -> str:
+    return lib.pre_strerror(int(code)).decode()
+
+
+def pre_create(n_instances, horizon, capacity_tokens, t_mem, beta, max_requests):
+    """Returns (code, ctx handle or None)."""
+    cfg = pre_config(int(n_instances), int(horizon), int(capacity_tokens), float(t_mem), float(beta),
+                     int(max_requests))
+    out = C.c_void_p()
+    code = lib.pre_create(C.byref(cfg), C.byref(out))
+    return code, (out.value if code == PRE_OK else None)
+
+
+def pre_destroy(ctx):
+    return lib.pre_destroy(ctx)
+
+
+def pre_anticipate(ctx, prompt, generated, predicted, instance, n_requests, curves, current_d, stream=None):
+    return lib.pre_anticipate(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance),
+                              int(n_requests), _ptr(curves), _ptr(current_d),
+                              _stream() if stream is None else stream)
+
+
+def pre_route_batch(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
+                    predicted, instance, n_requests, choice, score, stream=None):
+    return lib.pre_route_batch(ctx, _ptr(arr_prompt), _ptr(arr_predicted), int(n_arrivals), _ptr(curves),
+                               _ptr(queued_p), _ptr(current_d), _ptr(prompt), _ptr(generated), _ptr(predicted),
+                               _ptr(instance), _ptr(n_requests), _ptr(choice), _ptr(score),
+                               _stream() if stream is None else stream)
+
+
+def pre_step(ctx, prompt, generated, predicted, instance, n_requests, curves, queued_p, current_d, stream=None):
+    return lib.pre_step(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(n_requests),
+                        _ptr(curves), _ptr(queued_p), _ptr(current_d), _stream() if stream is None else stream)
+
+
+def pre_status(ctx, stream=None):
+    return lib.pre_status(ctx, _stream() if stream is None else stream)
+
+
+def pre_last_cuda_error(ctx):
+    return lib.pre_last_cuda_error(ctx)
+
+
+def pre_query(ctx):
+    g, t = C.c_int32(), C.c_int32()
+    code = lib.pre_query(ctx, C.byref(g), C.byref(t))
+    return code, g.value, t.value
+
+
+def check(code: int, where: str = "preserve_b200"):
+    if code != PRE_OK:
+        raise PreError(code, where)

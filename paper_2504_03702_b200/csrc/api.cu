@@ -1,0 +1,190 @@
+// C-ABI layer: argument checks, context life cycle, status word.  No arithmetic of the
+// method lives here; every step of the path runs in the kernels of the other files.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "pre_common.cuh"
+
+cudaError_t pre_anticipate_configure(pre_ctx* ctx);
+
+namespace {
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int fail_cuda(pre_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return PRE_ECUDA;
+}
+
+void release(pre_ctx* c) {
+    if (!c) return;
+    cudaFree(c->d_status);
+    cudaFree(c->d_bin_count);
+    cudaFree(c->d_bin_base);
+    cudaFree(c->d_bin_cursor);
+    cudaFree(c->d_records);
+    cudaFree(c->d_slots);
+    cudaFree(c->d_enter);
+    cudaFree(c->d_active);
+    delete c;
+}
+
+template <typename T>
+cudaError_t alloc_zero(T** p, size_t count) {
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+    if (e != cudaSuccess) { *p = nullptr; return e; }
+    return cudaMemset(*p, 0, count * sizeof(T));
+}
+
+}  // namespace
+
+extern "C" {
+
+int pre_create(const pre_config* cfg, pre_ctx** out) {
+    if (!cfg || !out) return PRE_EINVAL;
+    if (cfg->n_instances < 1 || cfg->horizon < 1 || cfg->horizon > PRE_MAX_HORIZON) return PRE_EINVAL;
+    if (cfg->capacity_tokens < 1 || cfg->max_requests < 1 || cfg->max_requests >= (1LL << 31)) return PRE_EINVAL;
+    if (!std::isfinite(cfg->t_mem) || !std::isfinite(cfg->beta) || cfg->t_mem < 0.0 || cfg->beta < 0.0)
+        return PRE_EINVAL;
+    if ((long long)cfg->n_instances * cfg->horizon >= (1LL << 40)) return PRE_EINVAL;
+
+    pre_ctx* c = new (std::nothrow) pre_ctx();
+    if (!c) return PRE_ENOMEM;
+    std::memset(c, 0, sizeof(*c));
+    c->cfg = *cfg;
+    c->theta = cfg->t_mem * (double)cfg->capacity_tokens;
+    c->epoch = 1;
+
+    cudaError_t e = cudaGetDevice(&c->device);
+    cudaDeviceProp prop;
+    if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, c->device);
+    if (e != cudaSuccess) { delete c; return PRE_ECUDA; }
+    c->n_sm = prop.multiProcessorCount;
+
+    // Build tile: T rows per block, about 48 KB of shared memory (12 bytes per cell), but
+    // never so many rows that the grid falls under ~8 blocks per SM.
+    const int I = cfg->n_instances, H = cfg->horizon;
+    int t_smem = (48 * 1024) / (12 * H);
+    if (t_smem < 1) t_smem = 1;
+    if (t_smem > PRE_MAX_TILE_ROWS) t_smem = PRE_MAX_TILE_ROWS;
+    int t = I / (8 * c->n_sm);
+    if (t < 1) t = 1;
+    if (t > t_smem) t = t_smem;
+    c->tile_rows = t;
+    c->n_tiles = (I + t - 1) / t;
+    if (pre_tile_smem_bytes(t, H) > (size_t)prop.sharedMemPerBlockOptin) { delete c; return PRE_EINVAL; }
+
+    e = alloc_zero(&c->d_status, 2);
+    c->d_abort = c->d_status ? c->d_status + 1 : nullptr;
+    if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_bin_base, (size_t)c->n_tiles + 1);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_bin_cursor, (size_t)c->n_tiles);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_records, (size_t)cfg->max_requests);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_enter, (size_t)I);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
+    if (e == cudaSuccess) e = pre_anticipate_configure(c);
+    if (e == cudaSuccess) e = pre_route_configure(c);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)4 * c->route_blocks);
+    if (e != cudaSuccess) {
+        const bool oom = (e == cudaErrorMemoryAllocation);
+        cudaGetLastError();
+        release(c);
+        return oom ? PRE_ENOMEM : (e == cudaErrorInvalidConfiguration || e == cudaErrorInvalidValue ? PRE_EINVAL
+                                                                                                     : PRE_ECUDA);
+    }
+    *out = c;
+    return PRE_OK;
+}
+
+int pre_destroy(pre_ctx* ctx) {
+    if (!ctx) return PRE_EINVAL;
+    release(ctx);
+    return PRE_OK;
+}
+
+int pre_anticipate(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated,
+                   const int32_t* d_predicted, const int32_t* d_instance, int64_t n_requests,
+                   int64_t* d_curves, int64_t* d_current_d, void* stream) {
+    if (!ctx || !d_curves || !d_current_d) return PRE_EINVAL;
+    if (n_requests < 0 || n_requests > ctx->cfg.max_requests) return PRE_EINVAL;
+    if (n_requests > 0 && (!d_prompt || !d_generated || !d_predicted || !d_instance)) return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_current_d, 8)) return PRE_EINVAL;
+    if (!aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) || !aligned(d_instance, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_anticipate(ctx, d_prompt, d_generated, d_predicted, d_instance, n_requests,
+                                          d_curves, d_current_d, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_route_batch(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted,
+                    int64_t n_arrivals, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
+                    int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                    int64_t* d_n_requests, int32_t* d_choice, double* d_score, void* stream) {
+    if (!ctx || n_arrivals < 0 || n_arrivals >= (1LL << 31)) return PRE_EINVAL;
+    if (!d_curves || !d_queued_p || !d_current_d || !d_prompt || !d_generated || !d_predicted || !d_instance ||
+        !d_n_requests)
+        return PRE_EINVAL;
+    if (n_arrivals > 0 && (!d_arr_prompt || !d_arr_predicted || !d_choice)) return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_queued_p, 8) || !aligned(d_current_d, 8) || !aligned(d_n_requests, 8) ||
+        !aligned(d_score, 8) || !aligned(d_choice, 4) || !aligned(d_arr_prompt, 4) || !aligned(d_arr_predicted, 4) ||
+        !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) || !aligned(d_instance, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_route(ctx, d_arr_prompt, d_arr_predicted, n_arrivals, d_curves, d_queued_p,
+                                     d_current_d, d_prompt, d_generated, d_predicted, d_instance, d_n_requests,
+                                     d_choice, d_score, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+             const int64_t* d_n_requests, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
+             void* stream) {
+    if (!ctx || !d_prompt || !d_generated || !d_predicted || !d_instance || !d_n_requests || !d_curves ||
+        !d_queued_p || !d_current_d)
+        return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_queued_p, 8) || !aligned(d_current_d, 8) || !aligned(d_n_requests, 8) ||
+        !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) || !aligned(d_instance, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_step(ctx, d_prompt, d_generated, d_predicted, d_instance, d_n_requests, d_curves,
+                                    d_queued_p, d_current_d, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_status(pre_ctx* ctx, void* stream) {
+    if (!ctx) return PRE_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(ctx, e);
+    if (word & PRE_ST_TIMEOUT) return PRE_ETIMEOUT;
+    if (word & PRE_ST_CAPACITY) return PRE_ECAPACITY;
+    if (word & PRE_ST_BADREQ) return PRE_EBADREQ;
+    return PRE_OK;
+}
+
+int pre_last_cuda_error(const pre_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+const char* pre_strerror(int code) {
+    switch (code) {
+        case PRE_OK: return "ok";
+        case PRE_EINVAL: return "invalid argument (null or misaligned pointer, size out of range)";
+        case PRE_ECAPACITY: return "request table full: some arrivals were not routed";
+        case PRE_EBADREQ: return "malformed request or arrival skipped";
+        case PRE_ETIMEOUT: return "a bounded device-side wait ran out; the batch was abandoned";
+        case PRE_ECUDA: return "CUDA runtime error";
+        case PRE_ENOMEM: return "out of memory";
+        default: return "unknown error code";
+    }
+}
+
+int pre_query(const pre_ctx* ctx, int32_t* route_blocks, int32_t* tile_rows) {
+    if (!ctx) return PRE_EINVAL;
+    if (route_blocks) *route_blocks = ctx->route_blocks;
+    if (tile_rows) *tile_rows = ctx->tile_rows;
+    return PRE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,61 @@
+// Internal declarations shared by the kernels and the C-ABI layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "preserve_b200.h"
+
+// Bits of the device status word (OR-ed by kernels, read by pre_status).
+enum : int { PRE_ST_BADREQ = 1, PRE_ST_CAPACITY = 2, PRE_ST_TIMEOUT = 4 };
+
+// Field limits that let one binned request fit in 64 bits:
+//   [ row within tile : 8 | B = P + g : 28 | remaining = D - g : 28 ]
+constexpr int PRE_FIELD_BITS = 28;
+constexpr int32_t PRE_FIELD_MAX = (1 << PRE_FIELD_BITS) - 1;
+constexpr int PRE_MAX_TILE_ROWS = 256;
+constexpr int PRE_MAX_HORIZON = 16384;
+// Per-block shared-memory histograms over bins (count and scatter kernels, step kernel).
+constexpr int PRE_SMEM_BINS = 8192;
+
+struct pre_ctx {
+    pre_config cfg;
+    int device;
+    int n_sm;
+    int tile_rows;       // T: instance rows per build tile
+    int n_tiles;         // ceil(I / T)
+    int route_blocks;    // G: blocks of the persistent routing kernel
+    int route_threads;
+    size_t route_smem;
+    double theta;        // t_mem * M in binary64
+    uint32_t epoch;      // running arrival counter, tags the routing exchange slots
+    int last_cuda_error;
+    // device scratch
+    int* d_status;            // status word
+    int* d_abort;             // routing kernel gives up when set
+    unsigned int* d_bin_count;   // [n_tiles]   zero between calls
+    unsigned int* d_bin_base;    // [n_tiles+1]
+    unsigned int* d_bin_cursor;  // [n_tiles]
+    unsigned long long* d_records;  // [max_requests]
+    unsigned long long* d_slots;    // [2][G][2] routing exchange
+    unsigned long long* d_enter;    // [I] tokens entering the window at step H-1 (zero between calls)
+    unsigned int* d_active;         // [I] live requests per instance (zero between calls)
+};
+
+// Launchers (defined next to their kernels).  Each returns a cudaError_t.
+cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
+                                  const int32_t* predicted, const int32_t* instance, int64_t n,
+                                  int64_t* curves, int64_t* current_d, cudaStream_t s);
+cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                             int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                             int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                             int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s);
+cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                            int32_t* instance, const int64_t* n_requests, int64_t* curves,
+                            int64_t* queued_p, int64_t* current_d, cudaStream_t s);
+cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
+size_t pre_tile_smem_bytes(int tile_rows, int horizon);
+
+__device__ __forceinline__ bool pre_request_ok(int32_t P, int32_t g, int32_t D, int32_t inst, int32_t I) {
+    return P >= 0 && g >= 0 && D >= 1 && inst >= 0 && inst < I;
+}

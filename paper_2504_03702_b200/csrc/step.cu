@@ -1,0 +1,103 @@
+// One decode iteration: every live request generates a token, finished requests retire,
+// every load-look-ahead map moves one iteration closer (iteration-level batching, paper
+// Sec. 2; "the next iterations" of the map, Sec. 4.3.1).
+//
+//   pre_step_requests  one pass over the request table: g += 1 for live requests, count
+//                      them per instance, and collect what enters the window at step H-1;
+//   pre_step_shift     one pass over the maps: shift every row left by one cell, write the
+//                      entering column, update current_d and queued_p, clear the scratch.
+#include "pre_common.cuh"
+
+namespace {
+
+constexpr int STEP_THREADS = 512;
+constexpr int SHIFT_THREADS = 256;
+
+__global__ void __launch_bounds__(STEP_THREADS)
+pre_step_requests(const int32_t* __restrict__ prompt, int32_t* __restrict__ generated,
+                  const int32_t* __restrict__ predicted, const int32_t* __restrict__ instance,
+                  const int64_t* __restrict__ n_requests, long long max_requests, int I, int H,
+                  unsigned int* __restrict__ active, unsigned long long* __restrict__ enter,
+                  int* __restrict__ status) {
+    extern __shared__ unsigned int sh_active[];
+    const bool use_sh = I <= PRE_SMEM_BINS;
+    long long n = *n_requests;
+    if (n > max_requests) n = max_requests;
+    if (use_sh) {
+        for (int i = threadIdx.x; i < I; i += blockDim.x) sh_active[i] = 0;
+        __syncthreads();
+    }
+    bool any_bad = false;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += stride) {
+        const int32_t g = generated[r], D = predicted[r], inst = instance[r];
+        if (g < 0 || D < 1 || (uint32_t)inst >= (uint32_t)I) { any_bad = true; continue; }
+        if (g >= D) continue;  // tombstone
+        const int32_t P = prompt[r];
+        if (P < 0) { any_bad = true; continue; }
+        const int32_t g1 = g + 1;
+        generated[r] = g1;
+        if (use_sh) atomicAdd(&sh_active[inst], 1u); else atomicAdd(&active[inst], 1u);
+        if ((long long)D - g1 >= (long long)H)
+            atomicAdd(&enter[inst], (unsigned long long)((long long)P + g1 + (H - 1)));
+    }
+    if (use_sh) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < I; i += blockDim.x) {
+            const unsigned int c = sh_active[i];
+            if (c) atomicAdd(&active[i], c);
+        }
+    }
+    if (any_bad) atomicOr(status, PRE_ST_BADREQ);
+}
+
+// One block per row.  The row is moved in passes of blockDim cells; a pass reads all its
+// cells before it writes any, and pass p reads cell (p+1)*blockDim before pass p+1 writes it.
+__global__ void __launch_bounds__(SHIFT_THREADS)
+pre_step_shift(int64_t* __restrict__ curves, int64_t* __restrict__ queued_p, int64_t* __restrict__ current_d,
+               unsigned int* __restrict__ active, unsigned long long* __restrict__ enter, int I, int H) {
+    for (int row = blockIdx.x; row < I; row += gridDim.x) {
+        int64_t* rp = curves + (size_t)row * H;
+        const long long last = (long long)enter[row];
+        for (int base = 0; base < H; base += SHIFT_THREADS * 4) {
+            long long v[4];
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = base + u * SHIFT_THREADS + threadIdx.x;
+                v[u] = (j + 1 < H) ? rp[j + 1] : last;
+            }
+            __syncthreads();
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int j = base + u * SHIFT_THREADS + threadIdx.x;
+                if (j < H) rp[j] = v[u];
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {
+            current_d[row] -= (long long)active[row];
+            queued_p[row] = 0;
+            active[row] = 0;
+            enter[row] = 0;
+        }
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                            int32_t* instance, const int64_t* n_requests, int64_t* curves,
+                            int64_t* queued_p, int64_t* current_d, cudaStream_t s) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    const size_t smem = I <= PRE_SMEM_BINS ? (size_t)I * sizeof(unsigned int) : 0;
+    long long want = (ctx->cfg.max_requests + STEP_THREADS * 4 - 1) / (STEP_THREADS * 4);
+    int grid = (int)(want < 4LL * ctx->n_sm ? want : 4LL * ctx->n_sm);
+    if (grid < 1) grid = 1;
+    pre_step_requests<<<grid, STEP_THREADS, smem, s>>>(prompt, generated, predicted, instance, n_requests,
+                                                     ctx->cfg.max_requests, I, H, ctx->d_active, ctx->d_enter,
+                                                     ctx->d_status);
+    int sgrid = I < 16 * ctx->n_sm ? I : 16 * ctx->n_sm;
+    pre_step_shift<<<sgrid, SHIFT_THREADS, 0, s>>>(curves, queued_p, current_d, ctx->d_active, ctx->d_enter, I, H);
+    return cudaGetLastError();
+}

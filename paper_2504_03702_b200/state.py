@@ -1,0 +1,86 @@
+"""Device-resident state of the path: thin holder of the tensors the C-ABI calls act on.
+
+This is plumbing (torch allocates device memory and provides the stream); each method is
+one C-ABI call.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class DeviceState:
+    def __init__(self, n_instances, horizon, capacity_tokens, max_requests, t_mem=0.8, beta=1.0,
+                 device="cuda:0"):
+        self.I, self.H = int(n_instances), int(horizon)
+        self.max_requests = int(max_requests)
+        self.device = torch.device(device)
+        with torch.cuda.device(self.device):
+            code, self.ctx = B.pre_create(n_instances, horizon, capacity_tokens, t_mem, beta, max_requests)
+        B.check(code, "pre_create")
+        i32 = dict(dtype=torch.int32, device=self.device)
+        i64 = dict(dtype=torch.int64, device=self.device)
+        self.prompt = torch.zeros(self.max_requests, **i32)
+        self.generated = torch.zeros(self.max_requests, **i32)
+        self.predicted = torch.zeros(self.max_requests, **i32)
+        self.instance = torch.zeros(self.max_requests, **i32)
+        self.n_requests = torch.zeros(1, **i64)
+        self.curves = torch.zeros(self.I, self.H, **i64)
+        self.queued_p = torch.zeros(self.I, **i64)
+        self.current_d = torch.zeros(self.I, **i64)
+
+    @classmethod
+    def from_workload(cls, wl, device="cuda:0"):
+        st = cls(wl.n_instances, wl.horizon, wl.capacity_tokens, max(wl.max_requests, 1), wl.t_mem, wl.beta,
+                 device)
+        st.load_requests(wl.prompt, wl.generated, wl.predicted, wl.instance)
+        return st
+
+    def load_requests(self, prompt, generated, predicted, instance):
+        n = len(prompt)
+        for dst, src in ((self.prompt, prompt), (self.generated, generated), (self.predicted, predicted),
+                         (self.instance, instance)):
+            dst[:n].copy_(torch.as_tensor(np.ascontiguousarray(src, dtype=np.int32)))
+        self.n_requests.fill_(n)
+        self.n_host = n
+
+    def anticipate(self, n_requests=None):
+        n = self.n_host if n_requests is None else int(n_requests)
+        B.check(B.pre_anticipate(self.ctx, self.prompt, self.generated, self.predicted, self.instance, n,
+                                 self.curves, self.current_d), "pre_anticipate")
+
+    def route_batch(self, arr_prompt, arr_predicted, want_score=True):
+        """arr_* are int32 device tensors. Returns (choice int32[A], score float64[A] or None) on device."""
+        a = int(arr_prompt.shape[0])
+        choice = torch.empty(a, dtype=torch.int32, device=self.device)
+        score = torch.empty(a, dtype=torch.float64, device=self.device) if want_score else None
+        B.check(B.pre_route_batch(self.ctx, arr_prompt, arr_predicted, a, self.curves, self.queued_p,
+                                  self.current_d, self.prompt, self.generated, self.predicted, self.instance,
+                                  self.n_requests, choice, score), "pre_route_batch")
+        return choice, score
+
+    def step(self):
+        B.check(B.pre_step(self.ctx, self.prompt, self.generated, self.predicted, self.instance,
+                           self.n_requests, self.curves, self.queued_p, self.current_d), "pre_step")
+
+    def status(self):
+        return B.pre_status(self.ctx)
+
+    def sync_count(self):
+        """Reads the device-side request count back (synchronises)."""
+        self.n_host = int(self.n_requests.item())
+        return self.n_host
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            torch.cuda.synchronize(self.device)
+            B.pre_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,301 @@
+"""CUDA path against the CPU oracle, element by element, through the C-ABI.
+
+Bar: int64 curves, counters, table columns and routing decisions bit-exact; the binary64
+score within 1e-12 relative (in practice identical: both sides round every operation
+separately).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_03702_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import assert_scores_close, assert_state_equal, dev  # noqa: E402
+from paper_2504_03702_b200 import binding as B  # noqa: E402
+from paper_2504_03702_b200.state import DeviceState  # noqa: E402
+
+
+def both(wl):
+    st = DeviceState.from_workload(wl)
+    ref = oracle.State.from_workload(wl)
+    st.anticipate()
+    ref.anticipate()
+    return st, ref
+
+
+# ------------------------------------------------------------------ anticipator
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_anticipate_configs(idx):
+    wl = W.make_config(idx)
+    st, ref = both(wl)
+    assert_state_equal(st, ref, f"config {idx}")
+    assert st.status() == B.PRE_OK
+    # integer atomics commute: a second build gives the same bits
+    first = st.curves.clone()
+    st.anticipate()
+    assert torch.equal(first, st.curves)
+    st.close()
+
+
+SHAPES = [(1, 1, 1, 7), (2, 3, 5, 0), (3, 1, 33, 50), (4, 7, 1, 90), (5, 5, 63, 400), (6, 9, 130, 700),
+          (7, 300, 6, 5000), (8, 2, 4097, 300), (9, 1, 16384, 100), (10, 1200, 10, 20000), (11, 37, 250, 3000)]
+
+
+@pytest.mark.parametrize("seed,n_inst,h,n", SHAPES)
+def test_anticipate_shapes(seed, n_inst, h, n):
+    wl = W.make_random(seed, n_inst, h, n, 0, max_prompt=500, max_output=3 * h + 5)
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+def test_anticipate_all_on_one_instance_and_long_requests():
+    wl = W.make_random(12, 6, 64, 3000, 0, max_prompt=4000, max_output=900)
+    wl.instance[:] = 4
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    st.close()
+
+
+def test_anticipate_tombstones_and_malformed():
+    wl = W.make_random(13, 5, 40, 600, 0)
+    wl.generated[::7] = wl.predicted[::7]          # finished: silently ignored
+    wl.generated[5] = wl.predicted[5] + 3
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    assert st.status() == B.PRE_OK
+    st.close()
+    wl.instance[11] = 5                             # out of range
+    wl.instance[12] = -1
+    wl.predicted[13] = 0
+    wl.generated[14] = -2
+    wl.prompt[15] = -1
+    wl.prompt[16] = 2 ** 28                         # above the documented field limit
+    st, ref = both(wl)
+    ref2 = oracle.State.from_workload(wl)
+    ref2.predicted[16] = 0                          # the oracle has no field limit: drop that one
+    ref2.anticipate()
+    assert (st.curves.cpu().numpy() == ref2.curves).all()
+    assert (st.current_d.cpu().numpy() == ref2.current_d).all()
+    assert st.status() == B.PRE_EBADREQ
+    assert st.status() == B.PRE_OK                  # reading clears
+    st.close()
+
+
+def test_anticipate_prefix_of_table():
+    wl = W.make_random(14, 8, 32, 1000, 0)
+    st = DeviceState.from_workload(wl)
+    st.anticipate(n_requests=400)
+    ref = oracle.State(8, 32, wl.capacity_tokens, wl.prompt[:400], wl.generated[:400], wl.predicted[:400],
+                       wl.instance[:400], 400)
+    ref.anticipate()
+    assert (st.curves.cpu().numpy() == ref.curves).all()
+    st.anticipate(n_requests=0)
+    assert int(st.curves.abs().sum()) == 0 and int(st.current_d.abs().sum()) == 0
+    st.close()
+
+
+def test_argument_errors_launch_nothing():
+    wl = W.make_random(15, 4, 16, 10, 0)
+    st = DeviceState.from_workload(wl)
+    assert B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, -1, st.curves,
+                            st.current_d) == B.PRE_EINVAL
+    assert B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, 10 ** 6, st.curves,
+                            st.current_d) == B.PRE_EINVAL
+    assert B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, 10, None,
+                            st.current_d) == B.PRE_EINVAL
+    assert B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, 10,
+                            st.curves.data_ptr() + 8, st.current_d) == B.PRE_EINVAL   # misaligned
+    assert B.pre_anticipate(st.ctx, None, st.generated, st.predicted, st.instance, 10, st.curves,
+                            st.current_d) == B.PRE_EINVAL
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+# ------------------------------------------------------------------ router
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_route_configs_against_literal_oracle(idx):
+    wl = W.make_config(idx)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    want_c, want_s = ref.route_batch(ap, ad)
+    choice = choice.cpu().numpy()
+    assert (choice == want_c).all(), f"first difference at arrival {int(np.argmax(choice != want_c))}"
+    assert_scores_close(score.cpu().numpy(), want_s, want_c)
+    assert_state_equal(st, ref, f"after routing config {idx}")
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+ROUTE_SHAPES = [(21, 1, 5, 10, 6), (22, 3, 9, 30, 25), (23, 7, 16, 60, 40), (24, 4, 1, 20, 10),
+                (25, 6, 40, 0, 30), (26, 200, 7, 500, 300), (27, 150, 64, 2000, 200), (28, 5, 1001, 300, 100),
+                (29, 333, 130, 3000, 257)]
+
+
+@pytest.mark.parametrize("seed,n_inst,h,n,a", ROUTE_SHAPES)
+def test_route_shapes(seed, n_inst, h, n, a):
+    wl = W.make_random(seed, n_inst, h, n, a, max_prompt=300, max_output=2 * h + 3)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    want_c, want_s = ref.route_batch(ap, ad)
+    assert (choice.cpu().numpy() == want_c).all()
+    assert_scores_close(score.cpu().numpy(), want_s, want_c)
+    assert_state_equal(st, ref)
+    st.close()
+
+
+def test_route_fractional_threshold_and_beta_without_score_output():
+    wl = W.make_random(31, 50, 24, 800, 300, capacity=33337, beta=0.75)
+    wl.t_mem = 0.8
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    choice, score = st.route_batch(dev(ap), dev(ad), want_score=False)
+    want_c, _ = ref.route_batch(ap, ad)
+    assert score is None and (choice.cpu().numpy() == want_c).all()
+    assert_state_equal(st, ref)
+    st.close()
+
+
+def test_route_consecutive_batches_and_empty_batch():
+    wl = W.make_random(32, 40, 32, 500, 400)
+    wl.max_requests = 500 + 400
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    got, want = [], []
+    for lo, hi in [(0, 1), (1, 1), (1, 130), (130, 131), (131, 400)]:
+        c, _ = st.route_batch(dev(ap[lo:hi]), dev(ad[lo:hi]))
+        got.append(c.cpu().numpy())
+        want.append(ref.route_batch(ap[lo:hi], ad[lo:hi])[0])
+    assert (np.concatenate(got) == np.concatenate(want)).all()
+    assert_state_equal(st, ref)
+    st.close()
+
+
+def test_route_table_full_and_malformed_arrivals():
+    wl = W.make_random(33, 6, 16, 100, 20)
+    wl.max_requests = 100 + 12
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0][0].copy(), wl.ticks[0][1].copy()
+    ad[3] = 0
+    ap[5] = -4
+    choice, _ = st.route_batch(dev(ap), dev(ad))
+    want_c, _ = ref.route_batch(ap, ad)
+    assert (choice.cpu().numpy() == want_c).all()
+    assert_state_equal(st, ref)
+    assert st.status() == B.PRE_ECAPACITY        # the most severe of the two recorded conditions
+    st.close()
+    wl.max_requests = 100 + 20
+    st, ref = both(wl)
+    choice, _ = st.route_batch(dev(ap), dev(ad))
+    assert (choice.cpu().numpy() == ref.route_batch(ap, ad)[0]).all()
+    assert st.status() == B.PRE_EBADREQ
+    st.close()
+
+
+def test_route_large_prefix_against_literal_oracle():
+    """Largest configuration, launch shape of the benchmark; the literal oracle on the first arrivals."""
+    wl = W.make_config(3)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0][0][:192], wl.ticks[0][1][:192]
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    want_c, want_s = ref.route_batch(ap, ad)
+    assert (choice.cpu().numpy() == want_c).all()
+    assert_scores_close(score.cpu().numpy(), want_s, want_c)
+    assert_state_equal(st, ref)
+    st.close()
+
+
+@pytest.mark.slow
+def test_route_large_full_batch():
+    """All 65,536 decisions of the largest configuration.
+
+    Expected values come from the oracle's identity mode, which the CPU tests admit only
+    because it reproduces the literal mode bit for bit; on top of that, sampled decisions
+    are re-scored one by one with the literal scan from a state rebuilt by the oracle.
+    """
+    wl = W.make_config(3)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    choice, score = choice.cpu().numpy(), score.cpu().numpy()
+    want_c, want_s = ref.route_batch(ap, ad, fast=True)
+    assert (choice == want_c).all(), f"first difference at arrival {int(np.argmax(choice != want_c))}"
+    assert_scores_close(score, want_s, want_c)
+    assert_state_equal(st, ref)
+    n0 = wl.n_requests
+    for k in [1, 4097, 30000, 65535]:
+        probe = oracle.State(wl.n_instances, wl.horizon, wl.capacity_tokens,
+                             np.concatenate([wl.prompt, ap[:k]]), np.concatenate([wl.generated, np.zeros(k, np.int32)]),
+                             np.concatenate([wl.predicted, ad[:k]]), np.concatenate([wl.instance, choice[:k]]),
+                             n0 + k)
+        probe.anticipate()
+        probe.queued_p[:] = np.bincount(choice[:k], weights=ap[:k], minlength=wl.n_instances).astype(np.int64)
+        s_all, _ = probe.score_all(int(ap[k]), int(ad[k]))
+        assert int(np.argmin(s_all)) == int(choice[k]) and s_all.min() == score[k]
+    st.close()
+
+
+# ------------------------------------------------------------------ decode step
+
+@pytest.mark.parametrize("seed,n_inst,h,n", [(41, 3, 6, 60), (42, 5, 16, 300), (43, 2, 1, 40), (44, 4, 80, 500),
+                                             (45, 70, 1030, 2000), (46, 9000, 8, 30000)])
+def test_step_shapes(seed, n_inst, h, n):
+    wl = W.make_random(seed, n_inst, h, n, 0, max_output=2 * h + 9)
+    st, ref = both(wl)
+    for k in range(12):
+        st.step()
+        ref.step()
+        assert_state_equal(st, ref, f"after step {k + 1}")
+    # the table alone reproduces the maps
+    keep = st.curves.clone()
+    st.anticipate()
+    assert torch.equal(keep, st.curves)
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_route_then_step_configs(idx):
+    wl = W.make_config(idx)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    st.route_batch(dev(ap), dev(ad))
+    ref.route_batch(ap, ad, fast=True)
+    for _ in range(3):
+        st.step()
+        ref.step()
+    assert_state_equal(st, ref)
+    st.close()
+
+
+def run_streaming(n_ticks):
+    wl = W.make_config(4, n_ticks=n_ticks)
+    st, ref = both(wl)
+    for t, (ap, ad) in enumerate(wl.ticks):
+        st.step()
+        ref.step()
+        c, s = st.route_batch(dev(ap), dev(ad))
+        wc, ws = ref.route_batch(ap, ad, fast=True)
+        c = c.cpu().numpy()
+        assert (c == wc).all(), f"tick {t}: first difference at arrival {int(np.argmax(c != wc))}"
+        assert_scores_close(s.cpu().numpy(), ws, wc)
+    assert_state_equal(st, ref, "at the end of the stream")
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+def test_streaming_config_first_ticks():
+    run_streaming(12)
+
+
+@pytest.mark.slow
+def test_streaming_config_with_a_burst():
+    run_streaming(101)
