@@ -108,7 +108,7 @@ def run_reference(args, wl, rank):
     if rank != 0:
         return
     n_route = min(wl.n_arrivals, args.ref_arrivals)
-    for _ in range(args.warmup if args.warmup < 1 else 1):
+    for _ in range(min(args.warmup, 1)):
         oracle_sample(wl, min(n_route, 8))
     per_step = []
     for _ in range(args.steps):
