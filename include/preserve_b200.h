@@ -57,7 +57,7 @@ typedef struct pre_ctx pre_ctx; /* opaque; owns only internal device scratch */
 typedef struct pre_config {
     int32_t n_instances;     /* I >= 1 */
     int32_t horizon;         /* H >= 1: look-ahead window in decode iterations (the paper's l);
-                                at most 16384 */
+                                at most 8192 */
     int64_t capacity_tokens; /* M >= 1: KV token capacity of one instance (Sec. 4.3.1) */
     double t_mem;            /* T_mem, ideal memory usage; 0.8 in the paper (Sec. 4.3.3) */
     double beta;             /* penalty coefficient; 1.0 in the paper (Sec. 4.3.3) */
@@ -65,7 +65,7 @@ typedef struct pre_config {
 } pre_config;
 
 /* Creates a context on the current CUDA device and allocates its scratch
- * (8 bytes per table slot plus O(I) words).  *out is set only on success. */
+ * (8 bytes per table slot plus a few MB of index words).  *out is set only on success. */
 int pre_create(const pre_config* cfg, pre_ctx** out);
 
 /* Frees the scratch.  The caller must have synchronised the stream first. */

@@ -8,63 +8,35 @@
 //     N[j] = #{r : R_r > j},   A[j] = sum{B_r : R_r > j},   c[j] = A[j] + j*N[j],
 // so each request costs one shared-memory update and column 0 is not a hot spot.
 //
-// Pipeline (all on the caller's stream, no host synchronisation):
-//   1. pre_bin_count    per-tile request counts (a tile = T consecutive instance rows)
-//   2. pre_bin_scatter  scans the counts (where each tile's records start), packs every
-//                       live request into 8 bytes and writes it to its tile's span
-//      (pre_bin_scan    separate scan launch, only when there are too many tiles for the
-//                       scatter blocks to scan in shared memory)
-//   3. pre_tile_build   one block per tile: shared-memory accumulation of (count, sum B)
-//                       per (row, R-1), suffix scan over the horizon, writes the rows
+// Pipeline (all on the caller's stream, no host synchronisation).  A tile is T
+// consecutive instance rows, built by one block in shared memory.
+//   1. pre_chunk_sort   each block takes a contiguous chunk of the table, packs every live
+//                       request into 8 bytes, orders them by tile inside the chunk (counting
+//                       sort in shared memory) and records where each tile starts in it
+//   2. pre_tile_build   one block per tile: gathers the tile's requests from every chunk,
+//                       accumulates (count, sum B) per (row, R-1) with shared-memory atomics,
+//                       suffix-scans over the horizon and writes the rows
+// No global atomics, no counting pass.  When there are more tiles than a block can count in
+// shared memory, a slower path is taken: pre_bin_count, pre_bin_scan, pre_bin_scatter
+// (global per-tile cursors) feed the same pre_tile_build.
 #include "pre_common.cuh"
 
 namespace {
 
 constexpr int BIN_THREADS = 512;
-constexpr int TILE_THREADS = 512;
-constexpr int TILE_WARPS = TILE_THREADS / 32;
 
-// Per-tile request counts.  Finished and malformed requests may be counted too: the counts
-// only reserve room, the scatter pass decides what is written.
+// Slow path only.  Per-tile request counts.  Finished and malformed requests may be counted
+// too: the counts only reserve room, the scatter pass decides what is written.
 __global__ void __launch_bounds__(BIN_THREADS)
-pre_bin_count(const int32_t* __restrict__ instance, int64_t n, int I, int T, int n_tiles,
-              unsigned int* __restrict__ bin_count) {
-    extern __shared__ unsigned int sh_bins[];
-    const bool use_sh = n_tiles <= PRE_SMEM_BINS;
-    if (use_sh) {
-        for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) sh_bins[i] = 0;
-        __syncthreads();
-    }
-    auto add = [&](int32_t v) {
-        if ((uint32_t)v < (uint32_t)I) {
-            const int b = v / T;
-            if (use_sh) atomicAdd(&sh_bins[b], 1u); else atomicAdd(&bin_count[b], 1u);
-        }
-    };
+pre_bin_count(const int32_t* __restrict__ instance, int64_t n, int I, int T, unsigned int* __restrict__ bin_count) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if ((reinterpret_cast<uintptr_t>(instance) & 15) == 0) {
-        const int64_t n4 = n >> 2;
-        const int4* in4 = reinterpret_cast<const int4*>(instance);
-        for (int64_t q = gtid; q < n4; q += stride) {
-            const int4 v = __ldg(in4 + q);
-            add(v.x); add(v.y); add(v.z); add(v.w);
-        }
-        for (int64_t r = (n4 << 2) + gtid; r < n; r += stride) add(instance[r]);
-    } else {
-        for (int64_t r = gtid; r < n; r += stride) add(instance[r]);
-    }
-    if (use_sh) {
-        __syncthreads();
-        for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
-            const unsigned int c = sh_bins[i];
-            if (c) atomicAdd(&bin_count[i], c);
-        }
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += stride) {
+        const int32_t v = instance[r];
+        if ((uint32_t)v < (uint32_t)I) atomicAdd(&bin_count[v / T], 1u);
     }
 }
 
-// One block.  base[b] = sum of count[0..b).  Only used when the tile count is too large
-// for the scatter blocks to scan it themselves in shared memory.
+// Slow path only.  One block: base[b] = sum of count[0..b).
 __global__ void __launch_bounds__(1024)
 pre_bin_scan(const unsigned int* __restrict__ bin_count, int n_tiles, unsigned int* __restrict__ bin_base) {
     __shared__ unsigned int warp_tot[32];
@@ -135,20 +107,12 @@ __device__ __forceinline__ void for_each_request(const int32_t* __restrict__ pro
     }
 }
 
-// Writes every live request, packed, into its tile's span of `records`.  Each block takes a
-// contiguous chunk of the table: it counts its requests per tile in shared memory, reserves
-// one span per touched tile with a single global atomic, then writes.  When the tile counts
-// fit in shared memory every block scans them itself (no separate scan launch); block 0
-// publishes the bases for the build kernel.
+// Slow path only: one global atomic per live request on its tile's cursor.
 __global__ void __launch_bounds__(BIN_THREADS)
 pre_bin_scatter(const int32_t* __restrict__ prompt, const int32_t* __restrict__ generated,
                 const int32_t* __restrict__ predicted, const int32_t* __restrict__ instance, int64_t n,
-                int I, int T, int n_tiles, const unsigned int* __restrict__ bin_count,
-                unsigned int* __restrict__ bin_base, unsigned int* __restrict__ bin_cursor,
+                int I, int T, const unsigned int* __restrict__ bin_base, unsigned int* __restrict__ bin_cursor,
                 unsigned long long* __restrict__ records, int* __restrict__ status) {
-    extern __shared__ unsigned int sh_u32[];
-    __shared__ unsigned int warp_tot[BIN_THREADS / 32];
-    const bool use_sh = n_tiles <= PRE_SMEM_BINS;
     int64_t chunk = (n + gridDim.x - 1) / gridDim.x;
     chunk = (chunk + 3) & ~(int64_t)3;
     const int64_t r0 = (int64_t)blockIdx.x * chunk < n ? (int64_t)blockIdx.x * chunk : n;
@@ -156,18 +120,91 @@ pre_bin_scatter(const int32_t* __restrict__ prompt, const int32_t* __restrict__ 
     const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
                        reinterpret_cast<uintptr_t>(predicted) | reinterpret_cast<uintptr_t>(instance)) & 15) == 0;
     bool any_bad = false;
-    if (use_sh) {
-        unsigned int* sh_bins = sh_u32;            // [n_tiles] histogram, then write cursor
-        unsigned int* sh_base = sh_u32 + n_tiles;  // [n_tiles] exclusive scan of the global counts
-        // ---- exclusive scan of the tile counts (each thread a contiguous run)
-        const int per = (n_tiles + BIN_THREADS - 1) / BIN_THREADS;
-        const int b0 = threadIdx.x * per;
-        unsigned int local = 0;
-        for (int k = 0; k < per; ++k) {
-            const int i = b0 + k;
-            if (i < n_tiles) { sh_bins[i] = 0; local += bin_count[i]; }
+    for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
+                     [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
+                         const Packed p = pack_request(P, g, D, inst, I, T);
+                         any_bad |= p.bad;
+                         if (p.live) records[bin_base[p.tile] + atomicAdd(&bin_cursor[p.tile], 1u)] = p.rec;
+                     });
+    if (any_bad) atomicOr(status, PRE_ST_BADREQ);
+}
+
+// ---------------------------------------------------------------------------------------
+// Fast path, step 1.  Block `ch` owns table rows [ch*chunk, (ch+1)*chunk) and the same span
+// of `records`.  It writes its live requests there ordered by tile and stores, for every
+// tile t, the offset of t's first record inside the span: chunk_off[t*NC + ch]
+// (chunk_off[n_tiles*NC + ch] = number of live requests of the chunk).
+constexpr int SORT_THREADS = 512;
+constexpr int SORT_CHUNK = 4096;   // requests a block can stage in shared memory
+constexpr int SORT_MAX_CHUNKS = 1024;
+
+__global__ void __launch_bounds__(SORT_THREADS)
+pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ generated,
+               const int32_t* __restrict__ predicted, const int32_t* __restrict__ instance, int64_t n,
+               int I, int T, int n_tiles, int64_t chunk, int staged, unsigned long long* __restrict__ records,
+               unsigned int* __restrict__ chunk_off, int* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned char sort_smem[];
+    __shared__ unsigned int warp_tot[SORT_THREADS / 32];
+    // layout: [stage: u64 x SORT_CHUNK][tile_of: u16 x SORT_CHUNK] (only when staged) [hist: u32 x (n_tiles+1)]
+    unsigned long long* stage = reinterpret_cast<unsigned long long*>(sort_smem);
+    unsigned short* tile_of = reinterpret_cast<unsigned short*>(stage + (staged ? SORT_CHUNK : 0));
+    unsigned int* hist = reinterpret_cast<unsigned int*>(tile_of + (staged ? SORT_CHUNK : 0));
+
+    const int ch = blockIdx.x, NC = gridDim.x;
+    const int64_t r0 = (int64_t)ch * chunk < n ? (int64_t)ch * chunk : n;
+    const int64_t r1 = r0 + chunk < n ? r0 + chunk : n;
+    const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
+                       reinterpret_cast<uintptr_t>(predicted) | reinterpret_cast<uintptr_t>(instance)) & 15) == 0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    bool any_bad = false;
+
+    for (int i = tid; i <= n_tiles; i += SORT_THREADS) hist[i] = 0;
+    __syncthreads();
+
+    // ---- pass A: pack, count per tile (and keep the packed request when it fits)
+    if (staged) {
+        // one request per (thread, slot): slot li = r - r0 < SORT_CHUNK
+        auto take = [&](int64_t r, int32_t P, int32_t g, int32_t D, int32_t inst) {
+            const Packed p = pack_request(P, g, D, inst, I, T);
+            any_bad |= p.bad;
+            const int li = (int)(r - r0);
+            stage[li] = p.rec;
+            tile_of[li] = p.live ? (unsigned short)p.tile : (unsigned short)0xFFFF;
+            if (p.live) atomicAdd(&hist[p.tile], 1u);
+        };
+        if (vec) {
+            const int64_t q1 = r1 >> 2;
+            for (int64_t q = (r0 >> 2) + tid; q < q1; q += SORT_THREADS) {
+                const int4 p = __ldg(reinterpret_cast<const int4*>(prompt) + q);
+                const int4 g = __ldg(reinterpret_cast<const int4*>(generated) + q);
+                const int4 d = __ldg(reinterpret_cast<const int4*>(predicted) + q);
+                const int4 i = __ldg(reinterpret_cast<const int4*>(instance) + q);
+                const int64_t r = q << 2;
+                take(r, p.x, g.x, d.x, i.x); take(r + 1, p.y, g.y, d.y, i.y);
+                take(r + 2, p.z, g.z, d.z, i.z); take(r + 3, p.w, g.w, d.w, i.w);
+            }
+            for (int64_t r = (q1 << 2) + tid; r < r1; r += SORT_THREADS)
+                if (r >= r0) take(r, prompt[r], generated[r], predicted[r], instance[r]);
+        } else {
+            for (int64_t r = r0 + tid; r < r1; r += SORT_THREADS)
+                take(r, prompt[r], generated[r], predicted[r], instance[r]);
         }
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    } else {
+        for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
+                         [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
+                             const Packed p = pack_request(P, g, D, inst, I, T);
+                             any_bad |= p.bad;
+                             if (p.live) atomicAdd(&hist[p.tile], 1u);
+                         });
+    }
+    __syncthreads();
+
+    // ---- exclusive scan of the per-tile counts, in place (each thread a contiguous run)
+    {
+        const int per = (n_tiles + SORT_THREADS) / SORT_THREADS;  // covers n_tiles + 1 entries
+        const int b0 = tid * per;
+        unsigned int local = 0;
+        for (int k = 0; k < per; ++k) if (b0 + k <= n_tiles) local += hist[b0 + k];
         unsigned int x = local;
         #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -180,247 +217,298 @@ pre_bin_scatter(const int32_t* __restrict__ prompt, const int32_t* __restrict__ 
         for (int w = 0; w < warp; ++w) run += warp_tot[w];
         for (int k = 0; k < per; ++k) {
             const int i = b0 + k;
-            if (i < n_tiles) {
-                sh_base[i] = run;
-                if (blockIdx.x == 0) bin_base[i] = run;
-                run += bin_count[i];
+            if (i <= n_tiles) {
+                const unsigned int c = hist[i];
+                hist[i] = run;                              // becomes the tile's write cursor
+                chunk_off[(size_t)i * NC + ch] = run;       // entry n_tiles receives the total
+                run += c;
             }
         }
-        __syncthreads();
-        // ---- pass A: this block's requests per tile
-        for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
-                         [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
-                             const Packed p = pack_request(P, g, D, inst, I, T);
-                             any_bad |= p.bad;
-                             if (p.live) atomicAdd(&sh_bins[p.tile], 1u);
-                         });
-        __syncthreads();
-        for (int i = threadIdx.x; i < n_tiles; i += BIN_THREADS) {
-            const unsigned int c = sh_bins[i];
-            if (c) sh_bins[i] = sh_base[i] + atomicAdd(&bin_cursor[i], c);
+    }
+    __syncthreads();
+
+    // ---- pass B: place
+    unsigned long long* out = records + r0;
+    if (staged) {
+        for (int li = tid; li < (int)(r1 - r0); li += SORT_THREADS) {
+            const unsigned int t = tile_of[li];
+            if (t != 0xFFFFu) out[atomicAdd(&hist[t], 1u)] = stage[li];
         }
-        __syncthreads();
-        // ---- pass B: write (the chunk is re-read, from L2)
-        for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
-                         [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
-                             const Packed p = pack_request(P, g, D, inst, I, T);
-                             if (p.live) records[atomicAdd(&sh_bins[p.tile], 1u)] = p.rec;
-                         });
     } else {
         for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
                          [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
                              const Packed p = pack_request(P, g, D, inst, I, T);
-                             any_bad |= p.bad;
-                             if (p.live) records[bin_base[p.tile] + atomicAdd(&bin_cursor[p.tile], 1u)] = p.rec;
+                             if (p.live) out[atomicAdd(&hist[p.tile], 1u)] = p.rec;
                          });
     }
     if (any_bad) atomicOr(status, PRE_ST_BADREQ);
 }
 
-// One block per tile of T instance rows.  Shared memory: count[cells], lo[cells], hi[cells]
-// (uint32 each; the sum of B per cell is kept as lo + 2^32*hi so that only 32-bit shared
-// atomics are needed), then per-row 64-bit words.
-constexpr int CPT = 8;  // cells per thread and scan pass
+// ---------------------------------------------------------------------------------------
+// Step 2.  One block per tile.  Shared memory holds, per cell (row, j) of the tile, one
+// 64-bit word {low: sum of B mod 2^32, high: count} plus a rarely used 32-bit carry word
+// (so that only 32-bit shared atomics are needed).  Rows are padded to a multiple of RUN
+// cells; a run of RUN consecutive cells is scanned by one thread, and every run is
+// followed by 16 bytes of padding so that the threads' 16-byte loads fall in different banks.
+constexpr int TILE_THREADS = 256;
+constexpr int TILE_WARPS = TILE_THREADS / 32;
+constexpr int RUN = 16;
 
-__global__ void __launch_bounds__(TILE_THREADS, 2)
-pre_tile_build(const unsigned long long* __restrict__ records, const unsigned int* __restrict__ bin_base,
-               unsigned int* __restrict__ bin_cursor, unsigned int* __restrict__ bin_count, int I, int H, int T,
-               int cells_pad, int64_t* __restrict__ curves, int64_t* __restrict__ current_d) {
+__device__ __forceinline__ int cell_slot(int c) { return c + ((c >> 4) << 1); }  // index in 8-byte words
+
+struct TileShape { int hp, rpr, cpw; };  // padded row length, runs per row, 32-run chunks per row
+
+__host__ __device__ inline TileShape tile_shape(int H) {
+    TileShape t;
+    t.rpr = (H + RUN - 1) / RUN;
+    t.hp = t.rpr * RUN;
+    t.cpw = (t.rpr + 31) / 32;
+    return t;
+}
+
+__global__ void __launch_bounds__(TILE_THREADS, 3)
+pre_tile_build(const unsigned long long* __restrict__ records,
+               const unsigned int* __restrict__ chunk_off, int NC, int64_t chunk,          // fast path
+               const unsigned int* __restrict__ bin_base, unsigned int* __restrict__ bin_cursor,
+               unsigned int* __restrict__ bin_count,                                        // slow path
+               int I, int H, int T, int64_t* __restrict__ curves, int64_t* __restrict__ current_d) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw);
-    uint32_t* lo = cnt + cells_pad;
-    uint32_t* hi = lo + cells_pad;
-    unsigned long long* excess = reinterpret_cast<unsigned long long*>(hi + cells_pad);  // [T]
-    unsigned long long* sum_n = excess + T;                                              // [T]
-    unsigned long long* wt_s = sum_n + T;                                                // [2][TILE_WARPS]
-    uint32_t* wt_n = reinterpret_cast<uint32_t*>(wt_s + 2 * TILE_WARPS);                 // [2][TILE_WARPS]
+    const TileShape sh = tile_shape(H);
+    const int cells = T * sh.hp;            // padded cells of a full tile
+    const int n_runs_max = T * sh.rpr;
+    unsigned long long* cl = reinterpret_cast<unsigned long long*>(smem_raw);        // [cells * 9/8]
+    unsigned long long* run_s = cl + (cells + (cells >> 3));                          // [n_runs_max]
+    unsigned long long* run_w = run_s + n_runs_max;                                   // [n_runs_max]
+    unsigned long long* chk_s = run_w + n_runs_max;                                   // [T * cpw]
+    unsigned long long* excess = chk_s + T * sh.cpw;                                  // [T]
+    unsigned long long* sum_n = excess + T;                                           // [T]
+    uint32_t* run_n = reinterpret_cast<uint32_t*>(sum_n + T);                         // [n_runs_max]
+    uint32_t* chk_n = run_n + n_runs_max;                                             // [T * cpw]
+    uint32_t* hi = chk_n + T * sh.cpw;                                                // [cells]
+    __shared__ int any_hi;
 
     const int tile = blockIdx.x;
     const int row0 = tile * T;
     const int rows = (I - row0) < T ? (I - row0) : T;
+    const int n_runs = rows * sh.rpr;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    {
-        uint4* z = reinterpret_cast<uint4*>(cnt);
-        const int nz = (3 * cells_pad) >> 2;
+    {   // clear the cell words, the carry words and the per-row sums
+        uint4* z = reinterpret_cast<uint4*>(cl);
+        const int nz = (cells + (cells >> 3)) >> 1;
         for (int i = tid; i < nz; i += TILE_THREADS) z[i] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < cells; i += TILE_THREADS) hi[i] = 0;
         for (int i = tid; i < 2 * T; i += TILE_THREADS) excess[i] = 0;
+        if (tid == 0) any_hi = 0;
     }
-    const unsigned int rec0 = bin_base[tile];
-    const unsigned int rec1 = rec0 + bin_cursor[tile];
     __syncthreads();
-    if (tid == 0) { bin_cursor[tile] = 0; bin_count[tile] = 0; }  // ready for the next call
 
     // ---- accumulate: one update per request at (row, R-1)
-    for (unsigned int r = rec0 + tid; r < rec1; r += TILE_THREADS) {
-        const unsigned long long rec = records[r];
+    auto add_record = [&](unsigned long long rec) {
         const uint32_t rem = (uint32_t)(rec & PRE_FIELD_MAX);
         const uint32_t B = (uint32_t)((rec >> PRE_FIELD_BITS) & PRE_FIELD_MAX);
         const int local = (int)(rec >> (2 * PRE_FIELD_BITS));
         const uint32_t R = rem < (uint32_t)H ? rem : (uint32_t)H;
-        const int cell = local * H + (int)R - 1;
-        atomicAdd(&cnt[cell], 1u);
-        const uint32_t old = atomicAdd(&lo[cell], B);
-        if (old + B < old) atomicAdd(&hi[cell], 1u);  // exactly one thread sees each wrap
+        const int c = local * sh.hp + (int)R - 1;
+        uint32_t* w = reinterpret_cast<uint32_t*>(cl + cell_slot(c));
+        atomicAdd(w + 1, 1u);
+        const uint32_t old = atomicAdd(w, B);
+        if (old + B < old) { atomicAdd(&hi[c], 1u); any_hi = 1; }  // exactly one thread sees each wrap
         if (rem > (uint32_t)H) atomicAdd(&excess[local], (unsigned long long)(rem - (uint32_t)H));
+    };
+    if (chunk_off != nullptr) {
+        const unsigned int* o0 = chunk_off + (size_t)tile * NC;
+        const unsigned int* o1 = o0 + NC;
+        for (int ch = tid; ch < NC; ch += TILE_THREADS) {
+            const unsigned int a = o0[ch], b = o1[ch];
+            const unsigned long long* src = records + (size_t)ch * chunk;
+            for (unsigned int r = a; r < b; ++r) add_record(src[r]);
+        }
+    } else {
+        const unsigned int rec0 = bin_base[tile];
+        const unsigned int rec1 = rec0 + bin_cursor[tile];
+        for (unsigned int r = rec0 + tid; r < rec1; r += TILE_THREADS) add_record(records[r]);
+    }
+    __syncthreads();
+    if (chunk_off == nullptr && tid == 0) { bin_cursor[tile] = 0; bin_count[tile] = 0; }  // for the next call
+    const bool with_hi = any_hi != 0;
+
+    // ---- phase 1: totals of every run
+    for (int run = tid; run < n_runs; run += TILE_THREADS) {
+        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(cl + run * (RUN + 2));
+        const int j0 = (run % sh.rpr) * RUN;
+        uint32_t tn = 0;
+        unsigned long long ts = 0, tw = 0;
+        #pragma unroll
+        for (int i = 0; i < RUN / 2; ++i) {
+            const ulonglong2 v = src[i];
+            const uint32_t n0 = (uint32_t)(v.x >> 32), n1 = (uint32_t)(v.y >> 32);
+            tn += n0 + n1;
+            ts += (v.x & 0xffffffffull) + (v.y & 0xffffffffull);
+            tw += (unsigned long long)n0 * (uint32_t)(j0 + 2 * i + 1) + (unsigned long long)n1 * (uint32_t)(j0 + 2 * i + 2);
+        }
+        if (with_hi) {
+            for (int k = 0; k < RUN; ++k) ts += (unsigned long long)hi[run * RUN + k] << 32;
+        }
+        run_n[run] = tn; run_s[run] = ts; run_w[run] = tw;
     }
     __syncthreads();
 
-    // ---- suffix scan over the horizon, `team_warps` warps per row, CPT cells per thread
-    int team_warps = 1;
-    while (team_warps < TILE_WARPS && team_warps * 32 * CPT < H) team_warps <<= 1;
-    const int teams = TILE_WARPS / team_warps;
-    const int team = warp / team_warps, wteam = warp % team_warps;
-    const int span = team_warps * 32 * CPT;
-    const int passes = (H + span - 1) / span;
-    const bool vec_sm = (H & 3) == 0;
-    const bool vec_gl = (H & 1) == 0;
-    int buf = 0;
+    // ---- phase 2: suffix over the runs of each row, 32 runs per warp task
+    for (int task = warp; task < rows * sh.cpw; task += TILE_WARPS) {
+        const int row = task / sh.cpw, k = task - row * sh.cpw;
+        const int q = k * 32 + lane;
+        const bool valid = q < sh.rpr;
+        const int run = row * sh.rpr + q;
+        const uint32_t n = valid ? run_n[run] : 0u;
+        const unsigned long long s = valid ? run_s[run] : 0ull;
+        unsigned long long w = valid ? run_w[run] : 0ull;
+        uint32_t xn = n;
+        unsigned long long xs = s;
+        #pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t yn = __shfl_down_sync(0xffffffffu, xn, off);
+            const unsigned long long ys = __shfl_down_sync(0xffffffffu, xs, off);
+            if (lane + off < 32) { xn += yn; xs += ys; }
+            w += __shfl_xor_sync(0xffffffffu, w, off);
+        }
+        if (valid) { run_n[run] = xn - n; run_s[run] = xs - s; }  // what lies above, inside the chunk
+        if (lane == 0) {
+            chk_n[task] = xn; chk_s[task] = xs;
+            // sum over j of N[j] = sum over requests of R: each request is counted on R steps
+            if (w) atomicAdd(&sum_n[row], w);
+        }
+    }
+    __syncthreads();
 
-    for (int rb = 0; rb < rows; rb += teams) {
-        const int row = rb + team;
-        const bool active = row < rows;
-        uint32_t carry_n = 0;
-        unsigned long long carry_s = 0, my_sum_n = 0;
-        for (int p = passes - 1; p >= 0; --p) {
-            const int j0 = p * span + (wteam * 32 + lane) * CPT;
-            uint32_t n[CPT];
-            unsigned long long s[CPT];
-            #pragma unroll
-            for (int k = 0; k < CPT; ++k) { n[k] = 0; s[k] = 0; }
-            if (active && j0 < H) {
-                const int c0 = row * H + j0;
-                if (vec_sm) {
-                    #pragma unroll
-                    for (int v = 0; v < CPT / 4; ++v) {
-                        if (j0 + 4 * v < H) {
-                            const uint4 a = *reinterpret_cast<const uint4*>(cnt + c0 + 4 * v);
-                            const uint4 b = *reinterpret_cast<const uint4*>(lo + c0 + 4 * v);
-                            const uint4 c = *reinterpret_cast<const uint4*>(hi + c0 + 4 * v);
-                            n[4 * v] = a.x; n[4 * v + 1] = a.y; n[4 * v + 2] = a.z; n[4 * v + 3] = a.w;
-                            s[4 * v] = ((unsigned long long)c.x << 32) | b.x;
-                            s[4 * v + 1] = ((unsigned long long)c.y << 32) | b.y;
-                            s[4 * v + 2] = ((unsigned long long)c.z << 32) | b.z;
-                            s[4 * v + 3] = ((unsigned long long)c.w << 32) | b.w;
-                        }
-                    }
-                } else {
-                    #pragma unroll
-                    for (int k = 0; k < CPT; ++k) {
-                        if (j0 + k < H) {
-                            n[k] = cnt[c0 + k];
-                            s[k] = ((unsigned long long)hi[c0 + k] << 32) | lo[c0 + k];
-                        }
-                    }
-                }
+    // ---- phase 3: every run from its last cell down; results overwrite the cell words
+    for (int run = tid; run < n_runs; run += TILE_THREADS) {
+        const int row = run / sh.rpr, q = run - row * sh.rpr;
+        const int k = q >> 5;
+        uint32_t N = run_n[run];
+        unsigned long long A = run_s[run];
+        for (int kk = k + 1; kk < sh.cpw; ++kk) { N += chk_n[row * sh.cpw + kk]; A += chk_s[row * sh.cpw + kk]; }
+        ulonglong2* io = reinterpret_cast<ulonglong2*>(cl + run * (RUN + 2));
+        const int j0 = q * RUN;
+        #pragma unroll
+        for (int i = RUN / 2 - 1; i >= 0; --i) {
+            const ulonglong2 v = io[i];
+            unsigned long long s1 = v.y & 0xffffffffull, s0 = v.x & 0xffffffffull;
+            if (with_hi) {
+                s1 |= (unsigned long long)hi[run * RUN + 2 * i + 1] << 32;
+                s0 |= (unsigned long long)hi[run * RUN + 2 * i] << 32;
             }
-            uint32_t tn = 0;
-            unsigned long long ts = 0;
-            #pragma unroll
-            for (int k = 0; k < CPT; ++k) { tn += n[k]; ts += s[k]; }
-            // inclusive suffix over the lanes of this warp (higher lane = later steps)
-            uint32_t xn = tn;
-            unsigned long long xs = ts;
-            #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t yn = __shfl_down_sync(0xffffffffu, xn, off);
-                const unsigned long long ys = __shfl_down_sync(0xffffffffu, xs, off);
-                if (lane + off < 32) { xn += yn; xs += ys; }
-            }
-            uint32_t above_n = carry_n;
-            unsigned long long above_s = carry_s;
-            if (team_warps > 1) {
-                if (lane == 0) { wt_n[buf * TILE_WARPS + warp] = xn; wt_s[buf * TILE_WARPS + warp] = xs; }
-                __syncthreads();
-                // suffix over the warps of the team, done redundantly by every warp
-                uint32_t wn = 0;
-                unsigned long long ws = 0;
-                if (lane < team_warps) {
-                    wn = wt_n[buf * TILE_WARPS + team * team_warps + lane];
-                    ws = wt_s[buf * TILE_WARPS + team * team_warps + lane];
-                }
-                #pragma unroll
-                for (int off = 1; off < TILE_WARPS; off <<= 1) {
-                    const uint32_t yn = __shfl_down_sync(0xffffffffu, wn, off);
-                    const unsigned long long ys = __shfl_down_sync(0xffffffffu, ws, off);
-                    if (lane + off < 32) { wn += yn; ws += ys; }
-                }
-                above_n += __shfl_sync(0xffffffffu, wn, wteam + 1);  // lanes >= team_warps hold 0
-                above_s += __shfl_sync(0xffffffffu, ws, wteam + 1);
-                carry_n += __shfl_sync(0xffffffffu, wn, 0);
-                carry_s += __shfl_sync(0xffffffffu, ws, 0);
-                buf ^= 1;
-            } else {
-                carry_n += __shfl_sync(0xffffffffu, xn, 0);
-                carry_s += __shfl_sync(0xffffffffu, xs, 0);
-            }
-            if (active && j0 < H) {
-                uint32_t N = above_n + (xn - tn);
-                unsigned long long A = above_s + (xs - ts);
-                unsigned long long c[CPT];
-                #pragma unroll
-                for (int k = CPT - 1; k >= 0; --k) {
-                    N += n[k]; A += s[k];
-                    c[k] = A + (unsigned long long)(uint32_t)(j0 + k) * N;
-                    if (j0 + k < H) my_sum_n += N;
-                }
-                int64_t* out = curves + ((size_t)(row0 + row) * H + j0);
+            ulonglong2 o;
+            N += (uint32_t)(v.y >> 32); A += s1;
+            o.y = A + (unsigned long long)(uint32_t)(j0 + 2 * i + 1) * N;
+            N += (uint32_t)(v.x >> 32); A += s0;
+            o.x = A + (unsigned long long)(uint32_t)(j0 + 2 * i) * N;
+            io[i] = o;
+        }
+    }
+    __syncthreads();
+
+    // ---- phase 4: copy the rows out with consecutive lanes on consecutive 16 bytes
+    {
+        const int half = sh.hp >> 1;  // cell pairs per padded row
+        const int total = rows * half;
+        const bool vec_gl = (H & 1) == 0;
+        for (int p = tid; p < total; p += TILE_THREADS) {
+            const int row = p / half;
+            const int j = (p - row * half) << 1;
+            if (j < H) {
+                const int c = row * sh.hp + j;
+                const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(cl + cell_slot(c));
+                int64_t* dst = curves + ((size_t)(row0 + row) * H + j);
                 if (vec_gl) {
-                    #pragma unroll
-                    for (int k = 0; k < CPT; k += 2)
-                        if (j0 + k < H) *reinterpret_cast<ulonglong2*>(out + k) = make_ulonglong2(c[k], c[k + 1]);
+                    *reinterpret_cast<ulonglong2*>(dst) = v;
                 } else {
-                    #pragma unroll
-                    for (int k = 0; k < CPT; ++k) if (j0 + k < H) out[k] = (int64_t)c[k];
+                    dst[0] = (int64_t)v.x;
+                    if (j + 1 < H) dst[1] = (int64_t)v.y;
                 }
             }
         }
-        // sum over j of N[j] = sum over requests of R (each request is counted on R steps)
-        #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) my_sum_n += __shfl_xor_sync(0xffffffffu, my_sum_n, off);
-        if (active && lane == 0 && my_sum_n) atomicAdd(&sum_n[row], my_sum_n);
     }
-    __syncthreads();
     for (int i = tid; i < rows; i += TILE_THREADS) current_d[row0 + i] = (int64_t)(sum_n[i] + excess[i]);
-}
-
-size_t tile_cells_pad(int tile_rows, int horizon) {
-    return (((size_t)tile_rows * horizon + 3) / 4) * 4 + 4;
 }
 
 }  // namespace
 
 size_t pre_tile_smem_bytes(int tile_rows, int horizon) {
-    return 3 * tile_cells_pad(tile_rows, horizon) * sizeof(uint32_t) + 2 * (size_t)tile_rows * 8 +
-           2 * TILE_WARPS * 8 + 2 * TILE_WARPS * 4;
+    const TileShape sh = tile_shape(horizon);
+    const size_t cells = (size_t)tile_rows * sh.hp;
+    const size_t runs = (size_t)tile_rows * sh.rpr;
+    const size_t chunks = (size_t)tile_rows * sh.cpw;
+    return (cells + cells / 8) * 8 + runs * (8 + 8 + 4) + chunks * (8 + 4) + (size_t)tile_rows * 16 + cells * 4;
+}
+
+int pre_tile_rows_for(int n_instances, int horizon, int n_sm) {
+    const TileShape sh = tile_shape(horizon);
+    int t = 4096 / sh.hp;                       // about 4096 cells (16 per thread) per tile
+    if (t < 1) t = 1;
+    if (t > PRE_MAX_TILE_ROWS) t = PRE_MAX_TILE_ROWS;
+    int by_grid = n_instances / (8 * n_sm);     // but keep the grid at several blocks per SM
+    if (by_grid < 1) by_grid = 1;
+    return t < by_grid ? t : by_grid;
+}
+
+static void sort_geometry(int64_t n, int* n_chunks, int64_t* chunk, int* staged) {
+    int64_t nc = (n + SORT_CHUNK - 1) / SORT_CHUNK;
+    if (nc > SORT_MAX_CHUNKS) nc = SORT_MAX_CHUNKS;
+    if (nc < 1) nc = 1;
+    int64_t c = (n + nc - 1) / nc;
+    c = (c + 3) & ~(int64_t)3;
+    if (c < 4) c = 4;
+    *n_chunks = (int)nc;
+    *chunk = c;
+    *staged = c <= SORT_CHUNK;
+}
+
+static size_t sort_smem_bytes(int n_tiles, int staged) {
+    return (staged ? (size_t)SORT_CHUNK * (8 + 2) : 0) + ((size_t)n_tiles + 1) * 4;
+}
+
+size_t pre_chunk_off_words(int n_tiles) {
+    return n_tiles <= PRE_SMEM_BINS ? ((size_t)n_tiles + 1) * SORT_MAX_CHUNKS : 0;
 }
 
 cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
                                   const int32_t* predicted, const int32_t* instance, int64_t n,
                                   int64_t* curves, int64_t* current_d, cudaStream_t s) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon, T = ctx->tile_rows, nt = ctx->n_tiles;
-    const bool use_sh = nt <= PRE_SMEM_BINS;
-    int grid = (int)((n + BIN_THREADS * 8 - 1) / (BIN_THREADS * 8));
-    if (grid > 2 * ctx->n_sm) grid = 2 * ctx->n_sm;
-    if (grid < 1) grid = 1;
-    if (n > 0) {
-        pre_bin_count<<<grid, BIN_THREADS, use_sh ? (size_t)nt * 4 : 0, s>>>(instance, n, I, T, nt, ctx->d_bin_count);
-        if (!use_sh) pre_bin_scan<<<1, 1024, 0, s>>>(ctx->d_bin_count, nt, ctx->d_bin_base);
-        pre_bin_scatter<<<grid, BIN_THREADS, use_sh ? (size_t)nt * 8 : 0, s>>>(
-            prompt, generated, predicted, instance, n, I, T, nt, ctx->d_bin_count, ctx->d_bin_base,
-            ctx->d_bin_cursor, ctx->d_records, ctx->d_status);
+    const size_t tile_smem = pre_tile_smem_bytes(T, H);
+    if (nt <= PRE_SMEM_BINS) {
+        int nc = 1, staged = 1;
+        int64_t chunk = 4;
+        sort_geometry(n, &nc, &chunk, &staged);
+        // With n == 0 the single chunk is empty: its offsets are all zero and every tile writes zero rows.
+        pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(nt, staged), s>>>(
+            prompt, generated, predicted, instance, n, I, T, nt, chunk, staged, ctx->d_records, ctx->d_chunk_off,
+            ctx->d_status);
+        pre_tile_build<<<nt, TILE_THREADS, tile_smem, s>>>(ctx->d_records, ctx->d_chunk_off, nc, chunk, nullptr,
+                                                         nullptr, nullptr, I, H, T, curves, current_d);
+    } else {
+        int grid = (int)((n + BIN_THREADS * 8 - 1) / (BIN_THREADS * 8));
+        if (grid > 2 * ctx->n_sm) grid = 2 * ctx->n_sm;
+        if (grid < 1) grid = 1;
+        if (n > 0) {
+            pre_bin_count<<<grid, BIN_THREADS, 0, s>>>(instance, n, I, T, ctx->d_bin_count);
+            pre_bin_scan<<<1, 1024, 0, s>>>(ctx->d_bin_count, nt, ctx->d_bin_base);
+            pre_bin_scatter<<<grid, BIN_THREADS, 0, s>>>(prompt, generated, predicted, instance, n, I, T,
+                                                       ctx->d_bin_base, ctx->d_bin_cursor, ctx->d_records,
+                                                       ctx->d_status);
+        }
+        // With n == 0 the cursors are zero (every build clears them): every tile sees an empty span.
+        pre_tile_build<<<nt, TILE_THREADS, tile_smem, s>>>(ctx->d_records, nullptr, 0, 0, ctx->d_bin_base,
+                                                         ctx->d_bin_cursor, ctx->d_bin_count, I, H, T, curves,
+                                                         current_d);
     }
-    // With n == 0 the counts and cursors are all zero (every build clears them), so every
-    // tile sees an empty span and writes zero rows.
-    pre_tile_build<<<nt, TILE_THREADS, pre_tile_smem_bytes(T, H), s>>>(
-        ctx->d_records, ctx->d_bin_base, ctx->d_bin_cursor, ctx->d_bin_count, I, H, T,
-        (int)tile_cells_pad(T, H), curves, current_d);
     return cudaGetLastError();
 }
 
 cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
-    cudaError_t e = cudaFuncSetAttribute(pre_bin_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         PRE_SMEM_BINS * 8);
+    cudaError_t e = cudaFuncSetAttribute(pre_chunk_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sort_smem_bytes(PRE_SMEM_BINS, 1));
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)pre_tile_smem_bytes(ctx->tile_rows, ctx->cfg.horizon));

@@ -7,8 +7,6 @@
 
 #include "pre_common.cuh"
 
-cudaError_t pre_anticipate_configure(pre_ctx* ctx);
-
 namespace {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
@@ -21,6 +19,7 @@ int fail_cuda(pre_ctx* ctx, cudaError_t e) {
 void release(pre_ctx* c) {
     if (!c) return;
     cudaFree(c->d_status);
+    cudaFree(c->d_chunk_off);
     cudaFree(c->d_bin_count);
     cudaFree(c->d_bin_base);
     cudaFree(c->d_bin_cursor);
@@ -63,21 +62,16 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e != cudaSuccess) { delete c; return PRE_ECUDA; }
     c->n_sm = prop.multiProcessorCount;
 
-    // Build tile: T rows per block, about 48 KB of shared memory (12 bytes per cell), but
-    // never so many rows that the grid falls under ~8 blocks per SM.
     const int I = cfg->n_instances, H = cfg->horizon;
-    int t_smem = (48 * 1024) / (12 * H);
-    if (t_smem < 1) t_smem = 1;
-    if (t_smem > PRE_MAX_TILE_ROWS) t_smem = PRE_MAX_TILE_ROWS;
-    int t = I / (8 * c->n_sm);
-    if (t < 1) t = 1;
-    if (t > t_smem) t = t_smem;
+    const int t = pre_tile_rows_for(I, H, c->n_sm);
     c->tile_rows = t;
     c->n_tiles = (I + t - 1) / t;
     if (pre_tile_smem_bytes(t, H) > (size_t)prop.sharedMemPerBlockOptin) { delete c; return PRE_EINVAL; }
 
     e = alloc_zero(&c->d_status, 2);
     c->d_abort = c->d_status ? c->d_status + 1 : nullptr;
+    if (e == cudaSuccess && pre_chunk_off_words(c->n_tiles))
+        e = alloc_zero(&c->d_chunk_off, pre_chunk_off_words(c->n_tiles));
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_base, (size_t)c->n_tiles + 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_cursor, (size_t)c->n_tiles);

@@ -14,8 +14,8 @@ enum : int { PRE_ST_BADREQ = 1, PRE_ST_CAPACITY = 2, PRE_ST_TIMEOUT = 4 };
 constexpr int PRE_FIELD_BITS = 28;
 constexpr int32_t PRE_FIELD_MAX = (1 << PRE_FIELD_BITS) - 1;
 constexpr int PRE_MAX_TILE_ROWS = 256;
-constexpr int PRE_MAX_HORIZON = 16384;
-// Per-block shared-memory histograms over bins (count and scatter kernels, step kernel).
+constexpr int PRE_MAX_HORIZON = 8192;
+// Largest number of build tiles (and, in the step kernel, instances) a block counts in shared memory.
 constexpr int PRE_SMEM_BINS = 8192;
 
 struct pre_ctx {
@@ -33,9 +33,10 @@ struct pre_ctx {
     // device scratch
     int* d_status;            // status word
     int* d_abort;             // routing kernel gives up when set
-    unsigned int* d_bin_count;   // [n_tiles]   zero between calls
-    unsigned int* d_bin_base;    // [n_tiles+1]
-    unsigned int* d_bin_cursor;  // [n_tiles]
+    unsigned int* d_chunk_off;   // [(n_tiles+1) x chunks] where each tile starts inside each sorted chunk
+    unsigned int* d_bin_count;   // slow path [n_tiles]   zero between calls
+    unsigned int* d_bin_base;    // slow path [n_tiles+1]
+    unsigned int* d_bin_cursor;  // slow path [n_tiles]   zero between calls
     unsigned long long* d_records;  // [max_requests]
     unsigned long long* d_slots;    // [2][G][2] routing exchange
     unsigned long long* d_enter;    // [I] tokens entering the window at step H-1 (zero between calls)
@@ -55,6 +56,9 @@ cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, i
                             int64_t* queued_p, int64_t* current_d, cudaStream_t s);
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
 size_t pre_tile_smem_bytes(int tile_rows, int horizon);
+int pre_tile_rows_for(int n_instances, int horizon, int n_sm);
+size_t pre_chunk_off_words(int n_tiles);
+cudaError_t pre_anticipate_configure(pre_ctx* ctx);
 
 __device__ __forceinline__ bool pre_request_ok(int32_t P, int32_t g, int32_t D, int32_t inst, int32_t I) {
     return P >= 0 && g >= 0 && D >= 1 && inst >= 0 && inst < I;

@@ -51,7 +51,7 @@ def test_error_strings_and_null_handling(binding):
 @pytest.mark.parametrize("args", [
     (0, 64, 100, 0.8, 1.0, 10),        # no instances
     (8, 0, 100, 0.8, 1.0, 10),         # no horizon
-    (8, 16385, 100, 0.8, 1.0, 10),     # horizon above the documented maximum
+    (8, 8193, 100, 0.8, 1.0, 10),      # horizon above the documented maximum
     (8, 64, 0, 0.8, 1.0, 10),          # no capacity
     (8, 64, 100, float("nan"), 1.0, 10),
     (8, 64, 100, 0.8, -1.0, 10),

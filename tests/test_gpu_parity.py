@@ -42,7 +42,7 @@ def test_anticipate_configs(idx):
 
 
 SHAPES = [(1, 1, 1, 7), (2, 3, 5, 0), (3, 1, 33, 50), (4, 7, 1, 90), (5, 5, 63, 400), (6, 9, 130, 700),
-          (7, 300, 6, 5000), (8, 2, 4097, 300), (9, 1, 16384, 100), (10, 1200, 10, 20000), (11, 37, 250, 3000)]
+          (7, 300, 6, 5000), (8, 2, 4097, 300), (9, 1, 8192, 100), (10, 1200, 10, 20000), (11, 37, 250, 3000)]
 
 
 @pytest.mark.parametrize("seed,n_inst,h,n", SHAPES)
@@ -50,6 +50,17 @@ def test_anticipate_shapes(seed, n_inst, h, n):
     wl = W.make_random(seed, n_inst, h, n, 0, max_prompt=500, max_output=3 * h + 5)
     st, ref = both(wl)
     assert_state_equal(st, ref)
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+def test_anticipate_more_tiles_than_a_block_can_count():
+    """8,300 one-row tiles: the build takes its slow path (global per-tile cursors)."""
+    wl = W.make_random(16, 8300, 4096, 20000, 0, max_prompt=3000, max_output=6000)
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    st.anticipate()
+    assert (st.curves.cpu().numpy() == ref.curves).all()
     assert st.status() == B.PRE_OK
     st.close()
 
