@@ -2,23 +2,32 @@
 //
 // The grid is launched cooperatively (all blocks resident).  Block b owns a fixed,
 // contiguous set of instance rows for the whole batch, so every read and every fold of a
-// row happens inside one block and needs only block-level ordering.  Per arrival:
-//   1. every warp streams its share of the block's rows with 16-byte loads and keeps, per
-//      row, m1 = max_{j<Dc}(c[j] + j) and m2 = max_{j>=Dc} c[j]   (Dc = min(D, H));
-//      the peak with the arrival virtually added is max(P + m1, m2);
-//   2. warp 0 turns the peaks into scores, takes the block's (score, index) minimum and
-//      publishes it in a global slot tagged with the arrival's running number;
-//   3. warp 0 of every block reads all G slots (bounded spin), so every block knows the
-//      winner without a second barrier; slots are double buffered by the tag's parity;
-//   4. the owner of the winning row adds the arrival's ramp to it, updates queued_p and
-//      current_d; block 0 appends the request and writes choice/score.
+// row happens inside one block and needs only block-level ordering.
+//
+// Scoring one arrival (P, D) against a row c[0..H): with Dc = min(D, H),
+//     m1 = max_{j<Dc}(c[j] + j),  m2 = max_{j>=Dc} c[j],  peak = max(P + m1, m2),
+// i.e. the literal scan of the row with the arrival virtually added.
+//
+// The arrivals form a chain (arrival k+1 must see arrival k folded into its winner), but a
+// fold changes ONE row.  So the blocks do not wait for the winner of arrival k before they
+// scan for arrival k+1; the exchange is one step behind the scan:
+//   iteration k:  1. every warp scans its share of the block's rows for arrival k against
+//                    the maps as they are (arrival k-1 not folded yet);
+//                 2. warp 0 collects the G published minima of arrival k-1 (bounded spin;
+//                    they were published before those blocks began this scan) -> winner w;
+//                 3. the owner of row w folds arrival k-1 into it and, in the same pass,
+//                    re-scores that one row for arrival k; block 0 appends the request;
+//                 4. warp 0 turns the block's peaks into scores, takes the (score, index)
+//                    minimum and publishes it in a slot tagged with the exchange number.
+// Slots are double buffered by the tag's parity: a block publishes exchange s only after it
+// has read every slot of s-1, and nobody reads s-2 after publishing s-1.
 #include "pre_common.cuh"
 
 #include <math_constants.h>
 
 namespace {
 
-constexpr int ROUTE_THREADS = 512;
+constexpr int ROUTE_THREADS = 1024;
 constexpr int ROUTE_WARPS = ROUTE_THREADS / 32;
 constexpr long long I64_MIN = (-9223372036854775807LL - 1);
 constexpr unsigned int SPIN_LIMIT = 1u << 22;  // polls before a wait is declared lost
@@ -90,16 +99,97 @@ struct RouteArgs {
     int max_rows;  // ceil(I / G)
 };
 
+// Running maxima of one row segment.
+struct Peak2 { long long a1, a2; };
+
+// Scans 64-cell chunks [q0, q1) of one row (chunk q covers steps 64q .. 64q+63, two per lane).
+// FULL: H is a multiple of 64 and 16-byte loads are legal, so no bounds checks are needed.
+template <bool FULL>
+__device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int Dc, int H,
+                                                 int lane) {
+    long long a1x = I64_MIN, a1y = I64_MIN, a2x = I64_MIN, a2y = I64_MIN;
+    if (FULL) {
+        const int qr = Dc >> 6;          // chunks [0, qr) lie entirely on the ramp
+        const int qt = (Dc + 63) >> 6;   // chunks [qt, ..) lie entirely after it
+        const int64_t* p = row + lane * 2;
+        int q = q0;
+        const int e1 = q1 < qr ? q1 : qr;
+        for (; q + 4 <= e1; q += 4) {
+            longlong2 v[4];
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = ld_cg_v2(p + (q + u) * 64);
+            const long long j = (long long)q * 64 + lane * 2;
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                a1x = max64(a1x, v[u].x + (j + u * 64));
+                a1y = max64(a1y, v[u].y + (j + u * 64));
+            }
+        }
+        for (; q < e1; ++q) {
+            const longlong2 v = ld_cg_v2(p + q * 64);
+            const long long j = (long long)q * 64 + lane * 2;
+            a1x = max64(a1x, v.x + j);
+            a1y = max64(a1y, v.y + j);
+        }
+        if (q < q1 && q < qt) {  // the one chunk that holds the end of the ramp
+            const longlong2 v = ld_cg_v2(p + q * 64);
+            const int j = q * 64 + lane * 2;
+            if (j < Dc) a1x = max64(a1x, v.x + j); else a2x = max64(a2x, v.x);
+            if (j + 1 < Dc) a1y = max64(a1y, v.y + j); else a2y = max64(a2y, v.y);
+            ++q;
+        }
+        for (; q + 4 <= q1; q += 4) {
+            longlong2 v[4];
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = ld_cg_v2(p + (q + u) * 64);
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) { a2x = max64(a2x, v[u].x); a2y = max64(a2y, v[u].y); }
+        }
+        for (; q < q1; ++q) {
+            const longlong2 v = ld_cg_v2(p + q * 64);
+            a2x = max64(a2x, v.x);
+            a2y = max64(a2y, v.y);
+        }
+    } else {
+        for (int q = q0; q < q1; ++q) {
+            const int j = q * 64 + lane * 2;
+            if (j < H) {
+                const long long x = ld_cg(row + j);
+                if (j < Dc) a1x = max64(a1x, x + j); else a2x = max64(a2x, x);
+            }
+            if (j + 1 < H) {
+                const long long y = ld_cg(row + j + 1);
+                if (j + 1 < Dc) a1y = max64(a1y, y + j); else a2y = max64(a2y, y);
+            }
+        }
+    }
+    Peak2 r;
+    // the odd cell of each pair sits one step later: its "+ j" above lacks 1
+    r.a1 = max64(a1x, a1y == I64_MIN ? I64_MIN : a1y + 1);
+    r.a2 = max64(a2x, a2y);
+    return r;
+}
+
+__device__ __forceinline__ Peak2 warp_max(Peak2 v) {
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        v.a1 = max64(v.a1, __shfl_xor_sync(0xffffffffu, v.a1, off));
+        v.a2 = max64(v.a2, __shfl_xor_sync(0xffffffffu, v.a2, off));
+    }
+    return v;
+}
+
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    long long* m1 = reinterpret_cast<long long*>(smem_raw);  // [max_rows]
-    long long* m2 = m1 + a.max_rows;                         // [max_rows]
-    long long* sq = m2 + a.max_rows;                         // queued_p of the owned rows
+    long long* m1 = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows]  (by arrival parity)
+    long long* m2 = m1 + 2 * a.max_rows;                     // [2][max_rows]
+    long long* sq = m2 + 2 * a.max_rows;                     // queued_p of the owned rows
     long long* scd = sq + a.max_rows;                        // current_d of the owned rows
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
+    __shared__ long long sh_fix[2];  // re-scored (m1, m2) of the row that was just folded
 
     const int G = gridDim.x, b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -110,19 +200,104 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     const int cpr = (H + 63) >> 6;  // 64-cell chunks per row (one 16-byte load per lane)
     const long long nch = (long long)nrows * cpr;
     const long long ch0 = nch * warp / ROUTE_WARPS, ch1 = nch * (warp + 1) / ROUTE_WARPS;
-    const bool vec = (H & 1) == 0;
+    const bool full = (H & 63) == 0;
 
     for (int r = tid; r < nrows; r += ROUTE_THREADS) {
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
+        m1[r] = I64_MIN; m2[r] = I64_MIN;   // buffer 0, used by the first scan
     }
     if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; }
     __syncthreads();
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
     if (room < 0) room = 0;
-    long long appended = 0;  // meaningful in every thread: all blocks take the same decisions
+    // Identical in every thread of every block: all take the same decisions.
+    long long seq = 0;            // exchanges started so far (= requests appended or pending)
     bool saw_bad = false, saw_full = false;
+    bool pending = false;         // an arrival has been published but not yet folded
+    int pP = 0, pD = 0;           // ... its prompt and predicted lengths
+    long long pk = 0;             // ... its index in the batch
+
+    // Collects the published minima of exchange `s` (warp 0 only); result in sh_winner/sh_score.
+    auto gather = [&](long long s) {
+        const unsigned int tag = a.epoch + (unsigned int)s;
+        const unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 2;
+        bool lost = false;
+        double bs = CUDART_INF;
+        int bi = 0x7fffffff;
+        for (int cta = lane; cta < G && !lost; cta += 32) {
+            unsigned long long w1;
+            unsigned int polls = 0;
+            for (;;) {
+                w1 = ld_acquire_u64(&slot[cta * 2 + 1]);
+                if ((unsigned int)(w1 >> 32) == tag) break;
+                if (++polls > SPIN_LIMIT || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag))) {
+                    lost = true;
+                    break;
+                }
+                if (polls > 256) __nanosleep(64);
+            }
+            if (!lost) {
+                const double sc = __longlong_as_double((long long)ld_relaxed_u64(&slot[cta * 2]));
+                const int i = (int)(unsigned int)(w1 & 0xffffffffu);
+                if (better(sc, i, bs, bi)) { bs = sc; bi = i; }
+            }
+        }
+        lost = __any_sync(0xffffffffu, lost);
+        #pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const double os = __shfl_xor_sync(0xffffffffu, bs, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (better(os, oi, bs, bi)) { bs = os; bi = oi; }
+        }
+        if (lane == 0) {
+            if (lost) {
+                atomicOr(a.status, PRE_ST_TIMEOUT);
+                atomicExch(a.abort_flag, 1);
+                sh_dead = 1;
+            }
+            sh_winner = bi;
+            sh_score = bs;
+        }
+    };
+
+    // The winner w of the pending arrival is known: the owner really adds it to row w
+    // (Sec. 4.3.1 update), block 0 records it.  When `rescore` is set, the same pass takes the
+    // folded row's maxima for the arrival being scored now (ramp length Dc) into sh_fix.
+    auto settle = [&](int w, bool rescore, int Dc) {
+        if (w >= row0 && w < row1) {
+            int64_t* rp = a.curves + (size_t)w * H;
+            const int pDc = pD < H ? pD : H;
+            long long a1 = I64_MIN, a2 = I64_MIN;
+            for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
+                long long c = ld_cg(rp + j);
+                if (j < pDc) { c += (long long)pP + j; rp[j] = c; }
+                if (j < Dc) a1 = max64(a1, c + j); else a2 = max64(a2, c);
+            }
+            if (rescore) {
+                Peak2 v; v.a1 = a1; v.a2 = a2;
+                v = warp_max(v);
+                if (lane == 0) { atomicMax(&sh_fix[0], v.a1); atomicMax(&sh_fix[1], v.a2); }
+            }
+            if (tid == 0) {
+                const int r = w - row0;
+                sq[r] += pP;
+                scd[r] += pD;
+                a.queued_p[w] = sq[r];
+                a.current_d[w] = scd[r];
+            }
+        }
+        if (b == 0 && tid == 0) {
+            const long long slot = n0 + seq - 1;  // the pending arrival is exchange seq-1
+            a.prompt[slot] = pP;
+            a.generated[slot] = 0;
+            a.predicted[slot] = pD;
+            a.instance[slot] = w;
+            a.choice[pk] = w;
+            if (a.score) a.score[pk] = sh_score;
+        }
+    };
 
     for (long long k = 0; k < a.n_arrivals; ++k) {
         const int P = a.arr_prompt[k], D = a.arr_predicted[k];
@@ -131,79 +306,63 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             if (b == 0 && tid == 0) { a.choice[k] = -1; if (a.score) a.score[k] = 0.0; }
             continue;
         }
-        if (appended >= room) {
+        if (seq >= room) {
             saw_full = true;
             if (b == 0 && tid == 0) { a.choice[k] = -1; if (a.score) a.score[k] = 0.0; }
             continue;
         }
         const int Dc = D < H ? D : H;
-        for (int r = tid; r < nrows; r += ROUTE_THREADS) { m1[r] = I64_MIN; m2[r] = I64_MIN; }
-        __syncthreads();
+        const int buf = (int)(seq & 1);
+        long long* bm1 = m1 + buf * a.max_rows;
+        long long* bm2 = m2 + buf * a.max_rows;
 
-        // ---- 1. stream the owned rows
+        // ---- 1. scan the owned rows for arrival k (the pending arrival is not folded yet)
         long long c = ch0;
         while (c < ch1) {
             const int row = (int)(c / cpr);
-            const long long row_end = ((long long)(row + 1) * cpr < ch1) ? (long long)(row + 1) * cpr : ch1;
+            const int q0 = (int)(c - (long long)row * cpr);
+            const long long left = ch1 - c;
+            const int q1 = (cpr - q0) < left ? cpr : q0 + (int)left;
             const int64_t* rp = a.curves + (size_t)(row0 + row) * H;
-            long long a1 = I64_MIN, a2 = I64_MIN;
-            int j = (int)(c - (long long)row * cpr) * 64 + lane * 2;
-            if (vec) {
-                long long q = c;
-                for (; q + 4 <= row_end; q += 4, j += 256) {
-                    longlong2 v[4];
-                    #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        v[u] = (j + u * 64 < H) ? ld_cg_v2(rp + j + u * 64) : make_longlong2(I64_MIN, I64_MIN);
-                    }
-                    #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int jj = j + u * 64;
-                        if (jj < H) {
-                            if (jj < Dc) a1 = max64(a1, v[u].x + jj); else a2 = max64(a2, v[u].x);
-                            if (jj + 1 < Dc) a1 = max64(a1, v[u].y + jj + 1); else a2 = max64(a2, v[u].y);
-                        }
-                    }
-                }
-                for (; q < row_end; ++q, j += 64) {
-                    if (j < H) {
-                        const longlong2 v = ld_cg_v2(rp + j);
-                        if (j < Dc) a1 = max64(a1, v.x + j); else a2 = max64(a2, v.x);
-                        if (j + 1 < Dc) a1 = max64(a1, v.y + j + 1); else a2 = max64(a2, v.y);
-                    }
-                }
-            } else {
-                for (long long q = c; q < row_end; ++q, j += 64) {
-                    if (j < H) {
-                        const long long x = ld_cg(rp + j);
-                        if (j < Dc) a1 = max64(a1, x + j); else a2 = max64(a2, x);
-                    }
-                    if (j + 1 < H) {
-                        const long long y = ld_cg(rp + j + 1);
-                        if (j + 1 < Dc) a1 = max64(a1, y + j + 1); else a2 = max64(a2, y);
-                    }
-                }
-            }
-            #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                a1 = max64(a1, __shfl_xor_sync(0xffffffffu, a1, off));
-                a2 = max64(a2, __shfl_xor_sync(0xffffffffu, a2, off));
-            }
+            Peak2 v = full ? scan_row_chunks<true>(rp, q0, q1, Dc, H, lane)
+                           : scan_row_chunks<false>(rp, q0, q1, Dc, H, lane);
+            v = warp_max(v);
             if (lane == 0) {
-                atomicMax(&m1[row], a1);
-                atomicMax(&m2[row], a2);
+                atomicMax(&bm1[row], v.a1);
+                atomicMax(&bm2[row], v.a2);
             }
-            c = row_end;
+            c += q1 - q0;
         }
-        __syncthreads();
+        __syncthreads();  // S1: all partial maxima of arrival k are in
 
-        // ---- 2./3. block minimum, publish, gather
+        // ---- 2. winner of the pending arrival; prepare the other buffer for the next scan
+        for (int r = tid; r < nrows; r += ROUTE_THREADS) {
+            m1[(buf ^ 1) * a.max_rows + r] = I64_MIN;
+            m2[(buf ^ 1) * a.max_rows + r] = I64_MIN;
+        }
+        if (tid == 32) { sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN; }
+        if (pending && warp == 0) gather(seq - 1);
+        __syncthreads();  // S2
+        if (sh_dead) break;
+
+        // ---- 3. fold the pending arrival, re-score its row for arrival k
+        if (pending) {
+            const int w = sh_winner;
+            settle(w, true, Dc);
+            if (w >= row0 && w < row1) {   // block-uniform
+                __syncthreads();           // S3: sh_fix complete, fold visible to the block
+                if (tid == 0) { bm1[w - row0] = sh_fix[0]; bm2[w - row0] = sh_fix[1]; }
+                __syncthreads();
+            }
+        }
+
+        // ---- 4. block minimum for arrival k, publish
         if (warp == 0) {
             double bs = CUDART_INF;
             int bi = 0x7fffffff;
             for (int r = lane; r < nrows; r += 32) {
-                long long peak = m1[r] + P;  // Dc >= 1: the ramp part is never empty
-                if (m2[r] > peak) peak = m2[r];
+                long long peak = bm1[r] + P;  // Dc >= 1: the ramp part is never empty
+                if (bm2[r] > peak) peak = bm2[r];
                 const double s = score_of(sq[r], scd[r], peak, P, D, a.theta, a.beta);
                 if (better(s, row0 + r, bs, bi)) { bs = s; bi = row0 + r; }
             }
@@ -213,81 +372,30 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
                 if (better(os, oi, bs, bi)) { bs = os; bi = oi; }
             }
-            const unsigned int tag = a.epoch + (unsigned int)appended;  // dense: one tag per exchange
-            unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 2;
             if (lane == 0) {
+                const unsigned int tag = a.epoch + (unsigned int)seq;  // dense: one tag per exchange
+                unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 2;
                 slot[b * 2] = (unsigned long long)__double_as_longlong(bs);
                 st_release_u64(&slot[b * 2 + 1], ((unsigned long long)tag << 32) | (unsigned int)bi);
             }
-            bool lost = false;
-            bs = CUDART_INF;
-            bi = 0x7fffffff;
-            for (int cta = lane; cta < G && !lost; cta += 32) {
-                unsigned long long w1;
-                unsigned int polls = 0;
-                for (;;) {
-                    w1 = ld_acquire_u64(&slot[cta * 2 + 1]);
-                    if ((unsigned int)(w1 >> 32) == tag) break;
-                    if (++polls > SPIN_LIMIT || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag))) {
-                        lost = true;
-                        break;
-                    }
-                    if (polls > 256) __nanosleep(64);
-                }
-                if (!lost) {
-                    const double s = __longlong_as_double((long long)ld_relaxed_u64(&slot[cta * 2]));
-                    const int i = (int)(unsigned int)(w1 & 0xffffffffu);
-                    if (better(s, i, bs, bi)) { bs = s; bi = i; }
-                }
-            }
-            lost = __any_sync(0xffffffffu, lost);
-            #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const double os = __shfl_xor_sync(0xffffffffu, bs, off);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                if (better(os, oi, bs, bi)) { bs = os; bi = oi; }
-            }
-            if (lane == 0) {
-                if (lost) {
-                    atomicOr(a.status, PRE_ST_TIMEOUT);
-                    atomicExch(a.abort_flag, 1);
-                    sh_dead = 1;
-                }
-                sh_winner = bi;
-                sh_score = bs;
-            }
         }
-        __syncthreads();
-        if (sh_dead) break;
-        const int w = sh_winner;
+        pending = true; pP = P; pD = D; pk = k;
+        ++seq;
+        // No barrier here: the other warps go on to the next scan while warp 0 publishes.  The
+        // next scan writes the other (m1, m2) buffer; sq/scd change only between S2 and S3.
+    }
 
-        // ---- 4. fold
-        if (w >= row0 && w < row1) {
-            int64_t* rp = a.curves + (size_t)w * H;
-            for (int j = tid; j < Dc; j += ROUTE_THREADS) rp[j] += (long long)P + j;
-            if (tid == 0) {
-                const int r = w - row0;
-                sq[r] += P;
-                scd[r] += D;
-                a.queued_p[w] = sq[r];
-                a.current_d[w] = scd[r];
-            }
-        }
-        if (b == 0 && tid == 0) {
-            const long long slot = n0 + appended;
-            a.prompt[slot] = P;
-            a.generated[slot] = 0;
-            a.predicted[slot] = D;
-            a.instance[slot] = w;
-            a.choice[k] = w;
-            if (a.score) a.score[k] = sh_score;
-        }
-        ++appended;
+    // ---- the last arrival is still pending
+    if (pending && !sh_dead) {
         __syncthreads();
+        if (warp == 0) gather(seq - 1);
+        __syncthreads();
+        if (!sh_dead) settle(sh_winner, false, 0);
     }
 
     if (b == 0 && tid == 0) {
-        *a.n_requests = n0 + appended;
+        // after a lost wait the pending arrival was never settled
+        *a.n_requests = n0 + (sh_dead && pending ? seq - 1 : seq);
         if (saw_bad) atomicOr(a.status, PRE_ST_BADREQ);
         if (saw_full) atomicOr(a.status, PRE_ST_CAPACITY);
     }
@@ -299,7 +407,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     const int I = ctx->cfg.n_instances;
     const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
     const int max_rows = (I + G - 1) / G;
-    const size_t smem = (size_t)max_rows * 4 * sizeof(long long);
+    const size_t smem = (size_t)max_rows * 6 * sizeof(long long);
     cudaError_t e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(smem > 48 * 1024 ? smem : 48 * 1024));
     if (e != cudaSuccess) return e;
