@@ -1,8 +1,10 @@
 // Load-aware request router (paper Sec. 4.3.3) as one persistent kernel per batch.
 //
-// The grid is launched cooperatively (all blocks resident).  Block b owns a fixed,
-// contiguous set of instance rows for the whole batch, so every read and every fold of a
-// row happens inside one block and needs only block-level ordering.
+// The grid is launched cooperatively (all blocks resident, one per SM).  Block b owns a
+// fixed, contiguous set of instance rows for the whole batch, so every read and every fold
+// of a row happens inside one block and needs only block-level ordering.  As many of the
+// block's rows as fit are copied into shared memory when the kernel starts and are scanned
+// from there; folds update both copies, so global memory is current at every moment.
 //
 // Scoring one arrival (P, D) against a row c[0..H): with Dc = min(D, H),
 //     m1 = max_{j<Dc}(c[j] + j),  m2 = max_{j>=Dc} c[j],  peak = max(P + m1, m2),
@@ -10,15 +12,15 @@
 //
 // The arrivals form a chain (arrival k+1 must see arrival k folded into its winner), but a
 // fold changes ONE row.  So the blocks do not wait for the winner of arrival k before they
-// scan for arrival k+1; the exchange is one step behind the scan:
-//   iteration k:  1. every warp scans its share of the block's rows for arrival k against
-//                    the maps as they are (arrival k-1 not folded yet);
-//                 2. warp 0 collects the G published minima of arrival k-1 (bounded spin;
-//                    they were published before those blocks began this scan) -> winner w;
-//                 3. the owner of row w folds arrival k-1 into it and, in the same pass,
-//                    re-scores that one row for arrival k; block 0 appends the request;
-//                 4. warp 0 turns the block's peaks into scores, takes the (score, index)
-//                    minimum and publishes it in a slot tagged with the exchange number.
+// scan for arrival k+1; the exchange runs one arrival behind the scan.  Iteration k:
+//   1. warps 1.. scan their share of the block's rows for arrival k against the maps as
+//      they are (arrival k-1 not folded yet); meanwhile warp 0 collects the G published
+//      minima of arrival k-1 (bounded spin) -> winner w;
+//   2. the owner of row w folds arrival k-1 into it and, in the same pass, re-scores that
+//      one row for arrival k; block 0 appends the request to the table;
+//   3. warp 0 turns the block's peaks into scores, takes the (score, index) minimum and
+//      publishes it in a slot tagged with the exchange number, while the other warps go on
+//      to the next scan.
 // Slots are double buffered by the tag's parity: a block publishes exchange s only after it
 // has read every slot of s-1, and nobody reads s-2 after publishing s-1.
 #include "pre_common.cuh"
@@ -29,6 +31,7 @@ namespace {
 
 constexpr int ROUTE_THREADS = 1024;
 constexpr int ROUTE_WARPS = ROUTE_THREADS / 32;
+constexpr int SCAN_WARPS = ROUTE_WARPS - 1;  // warp 0 coordinates
 constexpr long long I64_MIN = (-9223372036854775807LL - 1);
 constexpr unsigned int SPIN_LIMIT = 1u << 22;  // polls before a wait is declared lost
 
@@ -50,15 +53,40 @@ __device__ __forceinline__ int ld_relaxed_s32(const int* p) {
     asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// Streaming loads served by L2 (no L1 allocation): a row is re-read only after ~I*H*8 bytes.
-__device__ __forceinline__ longlong2 ld_cg_v2(const int64_t* p) {
+
+// Row loads.  Global rows are streamed through L2 without L1 allocation (a row is re-read
+// only after the block's whole share has gone by); resident rows come from shared memory.
+template <bool SMEM>
+__device__ __forceinline__ longlong2 ld_row_v2(const int64_t* p) {
+    if (SMEM) {
+        longlong2 v;
+        const unsigned int addr = (unsigned int)__cvta_generic_to_shared(p);
+        asm volatile("ld.shared.v2.s64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(addr) : "memory");
+        return v;
+    }
     return __ldcg(reinterpret_cast<const longlong2*>(p));
 }
-__device__ __forceinline__ long long ld_cg(const int64_t* p) {
+template <bool SMEM>
+__device__ __forceinline__ long long ld_row(const int64_t* p) {
+    if (SMEM) {
+        long long v;
+        const unsigned int addr = (unsigned int)__cvta_generic_to_shared(p);
+        asm volatile("ld.shared.s64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+        return v;
+    }
     return __ldcg(reinterpret_cast<const long long*>(p));
 }
 
 __device__ __forceinline__ long long max64(long long a, long long b) { return a > b ? a : b; }
+
+// Maximum of a signed 64-bit value over the warp with two 32-bit warp reductions.
+__device__ __forceinline__ long long warp_max64(long long v) {
+    const unsigned int hi = (unsigned int)((unsigned long long)v >> 32) ^ 0x80000000u;  // order preserving
+    const unsigned int lo = (unsigned int)v;
+    const unsigned int mh = __reduce_max_sync(0xffffffffu, hi);
+    const unsigned int ml = __reduce_max_sync(0xffffffffu, hi == mh ? lo : 0u);
+    return (long long)(((unsigned long long)(mh ^ 0x80000000u) << 32) | ml);
+}
 
 // Score of one instance, binary64, every operation rounded on its own.
 __device__ __forceinline__ double score_of(long long queued_p, long long current_d, long long peak, int P,
@@ -96,7 +124,8 @@ struct RouteArgs {
     unsigned int epoch;
     int* status;
     int* abort_flag;
-    int max_rows;  // ceil(I / G)
+    int max_rows;       // ceil(I / G)
+    int resident_rows;  // rows per block that fit in shared memory
 };
 
 // Running maxima of one row segment.
@@ -104,7 +133,7 @@ struct Peak2 { long long a1, a2; };
 
 // Scans 64-cell chunks [q0, q1) of one row (chunk q covers steps 64q .. 64q+63, two per lane).
 // FULL: H is a multiple of 64 and 16-byte loads are legal, so no bounds checks are needed.
-template <bool FULL>
+template <bool FULL, bool SMEM>
 __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int Dc, int H,
                                                  int lane) {
     long long a1x = I64_MIN, a1y = I64_MIN, a2x = I64_MIN, a2y = I64_MIN;
@@ -117,8 +146,8 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
         for (; q + 4 <= e1; q += 4) {
             longlong2 v[4];
             #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = ld_cg_v2(p + (q + u) * 64);
-            const long long j = (long long)q * 64 + lane * 2;
+            for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
+            const long long j = (long long)(q * 64 + lane * 2);
             #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 a1x = max64(a1x, v[u].x + (j + u * 64));
@@ -126,13 +155,13 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
             }
         }
         for (; q < e1; ++q) {
-            const longlong2 v = ld_cg_v2(p + q * 64);
-            const long long j = (long long)q * 64 + lane * 2;
+            const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+            const long long j = (long long)(q * 64 + lane * 2);
             a1x = max64(a1x, v.x + j);
             a1y = max64(a1y, v.y + j);
         }
         if (q < q1 && q < qt) {  // the one chunk that holds the end of the ramp
-            const longlong2 v = ld_cg_v2(p + q * 64);
+            const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
             const int j = q * 64 + lane * 2;
             if (j < Dc) a1x = max64(a1x, v.x + j); else a2x = max64(a2x, v.x);
             if (j + 1 < Dc) a1y = max64(a1y, v.y + j); else a2y = max64(a2y, v.y);
@@ -141,12 +170,12 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
         for (; q + 4 <= q1; q += 4) {
             longlong2 v[4];
             #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = ld_cg_v2(p + (q + u) * 64);
+            for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
             #pragma unroll
             for (int u = 0; u < 4; ++u) { a2x = max64(a2x, v[u].x); a2y = max64(a2y, v[u].y); }
         }
         for (; q < q1; ++q) {
-            const longlong2 v = ld_cg_v2(p + q * 64);
+            const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
             a2x = max64(a2x, v.x);
             a2y = max64(a2y, v.y);
         }
@@ -154,11 +183,11 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
         for (int q = q0; q < q1; ++q) {
             const int j = q * 64 + lane * 2;
             if (j < H) {
-                const long long x = ld_cg(row + j);
+                const long long x = ld_row<SMEM>(row + j);
                 if (j < Dc) a1x = max64(a1x, x + j); else a2x = max64(a2x, x);
             }
             if (j + 1 < H) {
-                const long long y = ld_cg(row + j + 1);
+                const long long y = ld_row<SMEM>(row + j + 1);
                 if (j + 1 < Dc) a1y = max64(a1y, y + j); else a2y = max64(a2y, y);
             }
         }
@@ -170,21 +199,39 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
     return r;
 }
 
-__device__ __forceinline__ Peak2 warp_max(Peak2 v) {
-    #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        v.a1 = max64(v.a1, __shfl_xor_sync(0xffffffffu, v.a1, off));
-        v.a2 = max64(v.a2, __shfl_xor_sync(0xffffffffu, v.a2, off));
+// Scans chunks [c0, c1) of a group of consecutive rows that start at `base` (row stride H),
+// adding each row segment's maxima into bm1/bm2[first_row + row].
+template <bool FULL, bool SMEM>
+__device__ __forceinline__ void scan_chunk_range(const int64_t* __restrict__ base, int c0, int c1, int cpr,
+                                                 int first_row, int Dc, int H, int lane, long long* bm1,
+                                                 long long* bm2) {
+    int c = c0;
+    if (c >= c1) return;
+    int row = c / cpr;
+    int q0 = c - row * cpr;
+    while (c < c1) {
+        const int left = c1 - c;
+        const int q1 = (cpr - q0) < left ? cpr : q0 + left;
+        Peak2 v = scan_row_chunks<FULL, SMEM>(base + (size_t)row * H, q0, q1, Dc, H, lane);
+        v.a1 = warp_max64(v.a1);
+        v.a2 = warp_max64(v.a2);
+        if (lane == 0) {
+            atomicMax(&bm1[first_row + row], v.a1);
+            atomicMax(&bm2[first_row + row], v.a2);
+        }
+        c += q1 - q0;
+        ++row;
+        q0 = 0;
     }
-    return v;
 }
 
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    long long* m1 = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows]  (by arrival parity)
+    long long* m1 = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows]  (by exchange parity)
     long long* m2 = m1 + 2 * a.max_rows;                     // [2][max_rows]
     long long* sq = m2 + 2 * a.max_rows;                     // queued_p of the owned rows
     long long* scd = sq + a.max_rows;                        // current_d of the owned rows
+    int64_t* res = reinterpret_cast<int64_t*>(scd + a.max_rows);  // [resident rows][H]; 48*max_rows bytes in: 16-byte aligned
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
@@ -197,17 +244,35 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     const int row0 = (int)(((long long)b * I) / G);
     const int row1 = (int)(((long long)(b + 1) * I) / G);
     const int nrows = row1 - row0;
+    const int S = a.resident_rows < nrows ? a.resident_rows : nrows;  // rows kept in shared memory
     const int cpr = (H + 63) >> 6;  // 64-cell chunks per row (one 16-byte load per lane)
-    const long long nch = (long long)nrows * cpr;
-    const long long ch0 = nch * warp / ROUTE_WARPS, ch1 = nch * (warp + 1) / ROUTE_WARPS;
     const bool full = (H & 63) == 0;
+    // chunk ranges of this warp (warps 1..): resident rows and streamed rows are split
+    // separately, since a resident chunk costs less than a streamed one
+    const int sw = warp - 1;
+    const int nchS = S * cpr, nchG = (nrows - S) * cpr;
+    const int s0 = warp ? (int)((long long)nchS * sw / SCAN_WARPS) : 0;
+    const int s1 = warp ? (int)((long long)nchS * (sw + 1) / SCAN_WARPS) : 0;
+    const int g0 = warp ? (int)((long long)nchG * sw / SCAN_WARPS) : 0;
+    const int g1 = warp ? (int)((long long)nchG * (sw + 1) / SCAN_WARPS) : 0;
+    const int64_t* grows = a.curves + (size_t)(row0 + S) * H;  // first streamed row
 
     for (int r = tid; r < nrows; r += ROUTE_THREADS) {
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
         m1[r] = I64_MIN; m2[r] = I64_MIN;   // buffer 0, used by the first scan
     }
-    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; }
+    {   // resident copy of the first S rows
+        const int64_t* src = a.curves + (size_t)row0 * H;
+        const int total = S * H;
+        if ((H & 1) == 0) {
+            for (int i = tid * 2; i < total; i += ROUTE_THREADS * 2)
+                *reinterpret_cast<longlong2*>(res + i) = __ldcg(reinterpret_cast<const longlong2*>(src + i));
+        } else {
+            for (int i = tid; i < total; i += ROUTE_THREADS) res[i] = __ldcg(src + i);
+        }
+    }
+    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN; }
     __syncthreads();
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
@@ -267,21 +332,27 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     // folded row's maxima for the arrival being scored now (ramp length Dc) into sh_fix.
     auto settle = [&](int w, bool rescore, int Dc) {
         if (w >= row0 && w < row1) {
-            int64_t* rp = a.curves + (size_t)w * H;
+            const int r = w - row0;
+            int64_t* gp = a.curves + (size_t)w * H;
+            int64_t* sp = res + (size_t)r * H;  // valid when r < S
+            const bool in_smem = r < S;
             const int pDc = pD < H ? pD : H;
             long long a1 = I64_MIN, a2 = I64_MIN;
             for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
-                long long c = ld_cg(rp + j);
-                if (j < pDc) { c += (long long)pP + j; rp[j] = c; }
+                long long c = in_smem ? sp[j] : __ldcg(gp + j);
+                if (j < pDc) {
+                    c += (long long)pP + j;
+                    gp[j] = c;
+                    if (in_smem) sp[j] = c;
+                }
                 if (j < Dc) a1 = max64(a1, c + j); else a2 = max64(a2, c);
             }
             if (rescore) {
-                Peak2 v; v.a1 = a1; v.a2 = a2;
-                v = warp_max(v);
-                if (lane == 0) { atomicMax(&sh_fix[0], v.a1); atomicMax(&sh_fix[1], v.a2); }
+                a1 = warp_max64(a1);
+                a2 = warp_max64(a2);
+                if (lane == 0) { atomicMax(&sh_fix[0], a1); atomicMax(&sh_fix[1], a2); }
             }
             if (tid == 0) {
-                const int r = w - row0;
                 sq[r] += pP;
                 scd[r] += pD;
                 a.queued_p[w] = sq[r];
@@ -316,48 +387,37 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         long long* bm1 = m1 + buf * a.max_rows;
         long long* bm2 = m2 + buf * a.max_rows;
 
-        // ---- 1. scan the owned rows for arrival k (the pending arrival is not folded yet)
-        long long c = ch0;
-        while (c < ch1) {
-            const int row = (int)(c / cpr);
-            const int q0 = (int)(c - (long long)row * cpr);
-            const long long left = ch1 - c;
-            const int q1 = (cpr - q0) < left ? cpr : q0 + (int)left;
-            const int64_t* rp = a.curves + (size_t)(row0 + row) * H;
-            Peak2 v = full ? scan_row_chunks<true>(rp, q0, q1, Dc, H, lane)
-                           : scan_row_chunks<false>(rp, q0, q1, Dc, H, lane);
-            v = warp_max(v);
-            if (lane == 0) {
-                atomicMax(&bm1[row], v.a1);
-                atomicMax(&bm2[row], v.a2);
-            }
-            c += q1 - q0;
+        // ---- 1. scan for arrival k (the pending arrival is not folded yet) | collect its winner
+        if (warp == 0) {
+            if (pending) gather(seq - 1);
+        } else if (full) {
+            scan_chunk_range<true, true>(res, s0, s1, cpr, 0, Dc, H, lane, bm1, bm2);
+            scan_chunk_range<true, false>(grows, g0, g1, cpr, S, Dc, H, lane, bm1, bm2);
+        } else {
+            scan_chunk_range<false, true>(res, s0, s1, cpr, 0, Dc, H, lane, bm1, bm2);
+            scan_chunk_range<false, false>(grows, g0, g1, cpr, S, Dc, H, lane, bm1, bm2);
         }
-        __syncthreads();  // S1: all partial maxima of arrival k are in
+        __syncthreads();  // S1: partial maxima of arrival k are in, winner of the pending arrival known
+        if (sh_dead) break;
 
-        // ---- 2. winner of the pending arrival; prepare the other buffer for the next scan
+        // ---- 2. fold the pending arrival, re-score its row for arrival k; reset the other buffer
         for (int r = tid; r < nrows; r += ROUTE_THREADS) {
             m1[(buf ^ 1) * a.max_rows + r] = I64_MIN;
             m2[(buf ^ 1) * a.max_rows + r] = I64_MIN;
         }
-        if (tid == 32) { sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN; }
-        if (pending && warp == 0) gather(seq - 1);
-        __syncthreads();  // S2
-        if (sh_dead) break;
+        const int w = sh_winner;
+        if (pending) settle(w, true, Dc);
+        __syncthreads();  // S2: fold visible to the block, sh_fix complete
 
-        // ---- 3. fold the pending arrival, re-score its row for arrival k
-        if (pending) {
-            const int w = sh_winner;
-            settle(w, true, Dc);
-            if (w >= row0 && w < row1) {   // block-uniform
-                __syncthreads();           // S3: sh_fix complete, fold visible to the block
-                if (tid == 0) { bm1[w - row0] = sh_fix[0]; bm2[w - row0] = sh_fix[1]; }
-                __syncthreads();
-            }
-        }
-
-        // ---- 4. block minimum for arrival k, publish
+        // ---- 3. block minimum for arrival k, publish
         if (warp == 0) {
+            if (pending && w >= row0 && w < row1) {
+                if (lane == 0) {
+                    bm1[w - row0] = sh_fix[0]; bm2[w - row0] = sh_fix[1];
+                    sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN;
+                }
+                __syncwarp();
+            }
             double bs = CUDART_INF;
             int bi = 0x7fffffff;
             for (int r = lane; r < nrows; r += 32) {
@@ -381,8 +441,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         }
         pending = true; pP = P; pD = D; pk = k;
         ++seq;
-        // No barrier here: the other warps go on to the next scan while warp 0 publishes.  The
-        // next scan writes the other (m1, m2) buffer; sq/scd change only between S2 and S3.
+        // No barrier here: the other warps go on to the next scan (which fills the other
+        // (m1, m2) buffer) while warp 0 scores and publishes; sq/scd and sh_fix change only
+        // between S1 and S2 or inside warp 0.
     }
 
     // ---- the last arrival is still pending
@@ -404,12 +465,23 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
 }  // namespace
 
 cudaError_t pre_route_configure(pre_ctx* ctx) {
-    const int I = ctx->cfg.n_instances;
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
     const int max_rows = (I + G - 1) / G;
-    const size_t smem = (size_t)max_rows * 6 * sizeof(long long);
-    cudaError_t e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)(smem > 48 * 1024 ? smem : 48 * 1024));
+    const size_t fixed = (size_t)max_rows * 6 * sizeof(long long);
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes attr;
+    e = cudaFuncGetAttributes(&attr, pre_route_persistent);
+    if (e != cudaSuccess) return e;
+    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+    if (fixed + attr.sharedSizeBytes + 1024 > limit) return cudaErrorInvalidConfiguration;
+    // rows kept in shared memory: whatever fits beside the fixed part
+    size_t resident = (limit - attr.sharedSizeBytes - 1024 - fixed) / ((size_t)H * sizeof(int64_t));
+    if (resident > (size_t)max_rows) resident = (size_t)max_rows;
+    const size_t smem = fixed + resident * (size_t)H * sizeof(int64_t);
+    e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pre_route_persistent, ROUTE_THREADS, smem);
@@ -418,6 +490,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     ctx->route_blocks = G;
     ctx->route_threads = ROUTE_THREADS;
     ctx->route_smem = smem;
+    ctx->route_resident_rows = (int)resident;
     return cudaSuccess;
 }
 
@@ -439,6 +512,7 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
     a.slots = ctx->d_slots; a.epoch = ctx->epoch;
     a.status = ctx->d_status; a.abort_flag = ctx->d_abort;
     a.max_rows = (a.I + ctx->route_blocks - 1) / ctx->route_blocks;
+    a.resident_rows = ctx->route_resident_rows;
     ctx->epoch += (unsigned int)n_arrivals;
     void* params[] = {(void*)&a};
     return cudaLaunchCooperativeKernel((const void*)pre_route_persistent, dim3(ctx->route_blocks),
