@@ -7,7 +7,7 @@
 // from there; folds update both copies, so global memory is current at every moment.
 //
 // Scoring one arrival (P, D) against a row c[0..H): with Dc = min(D, H),
-//     m1 = max_{j<Dc}(c[j] + j),  m2 = max_{j>=Dc} c[j],  peak = max(P + m1, m2),
+//     peak = max( max_{j<Dc}(c[j] + P + j),  max_{j>=Dc} c[j] ),
 // i.e. the literal scan of the row with the arrival virtually added.
 //
 // The arrivals form a chain (arrival k+1 must see arrival k folded into its winner), but a
@@ -128,15 +128,14 @@ struct RouteArgs {
     int resident_rows;  // rows per block that fit in shared memory
 };
 
-// Running maxima of one row segment.
-struct Peak2 { long long a1, a2; };
-
-// Scans 64-cell chunks [q0, q1) of one row (chunk q covers steps 64q .. 64q+63, two per lane).
+// Peak over 64-cell chunks [q0, q1) of one row with the arrival (P, Dc) virtually added
+// (chunk q covers steps 64q .. 64q+63, two per lane); the result is per lane.
 // FULL: H is a multiple of 64 and 16-byte loads are legal, so no bounds checks are needed.
 template <bool FULL, bool SMEM>
-__device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int Dc, int H,
-                                                 int lane) {
-    long long a1x = I64_MIN, a1y = I64_MIN, a2x = I64_MIN, a2y = I64_MIN;
+__device__ __forceinline__ long long scan_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int P,
+                                                     int Dc, int H, int lane) {
+    // rx / ry: ramp part, even / odd cell of the pair (ry lacks the odd cell's extra +1); t: after the ramp
+    long long rx = I64_MIN, ry = I64_MIN, t = I64_MIN;
     if (FULL) {
         const int qr = Dc >> 6;          // chunks [0, qr) lie entirely on the ramp
         const int qt = (Dc + 63) >> 6;   // chunks [qt, ..) lie entirely after it
@@ -147,96 +146,70 @@ __device__ __forceinline__ Peak2 scan_row_chunks(const int64_t* __restrict__ row
             longlong2 v[4];
             #pragma unroll
             for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
-            const long long j = (long long)(q * 64 + lane * 2);
+            const long long jp = (long long)(q * 64 + lane * 2) + P;
             #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                a1x = max64(a1x, v[u].x + (j + u * 64));
-                a1y = max64(a1y, v[u].y + (j + u * 64));
+                rx = max64(rx, v[u].x + (jp + u * 64));
+                ry = max64(ry, v[u].y + (jp + u * 64));
             }
         }
         for (; q < e1; ++q) {
             const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
-            const long long j = (long long)(q * 64 + lane * 2);
-            a1x = max64(a1x, v.x + j);
-            a1y = max64(a1y, v.y + j);
+            const long long jp = (long long)(q * 64 + lane * 2) + P;
+            rx = max64(rx, v.x + jp);
+            ry = max64(ry, v.y + jp);
         }
         if (q < q1 && q < qt) {  // the one chunk that holds the end of the ramp
             const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
             const int j = q * 64 + lane * 2;
-            if (j < Dc) a1x = max64(a1x, v.x + j); else a2x = max64(a2x, v.x);
-            if (j + 1 < Dc) a1y = max64(a1y, v.y + j); else a2y = max64(a2y, v.y);
+            const long long jp = (long long)j + P;
+            if (j < Dc) rx = max64(rx, v.x + jp); else t = max64(t, v.x);
+            if (j + 1 < Dc) ry = max64(ry, v.y + jp); else t = max64(t, v.y);
             ++q;
         }
+        long long t2 = I64_MIN;
         for (; q + 4 <= q1; q += 4) {
             longlong2 v[4];
             #pragma unroll
             for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
             #pragma unroll
-            for (int u = 0; u < 4; ++u) { a2x = max64(a2x, v[u].x); a2y = max64(a2y, v[u].y); }
+            for (int u = 0; u < 4; ++u) { t = max64(t, v[u].x); t2 = max64(t2, v[u].y); }
         }
         for (; q < q1; ++q) {
             const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
-            a2x = max64(a2x, v.x);
-            a2y = max64(a2y, v.y);
+            t = max64(t, v.x);
+            t2 = max64(t2, v.y);
         }
+        t = max64(t, t2);
     } else {
         for (int q = q0; q < q1; ++q) {
             const int j = q * 64 + lane * 2;
+            const long long jp = (long long)j + P;
             if (j < H) {
                 const long long x = ld_row<SMEM>(row + j);
-                if (j < Dc) a1x = max64(a1x, x + j); else a2x = max64(a2x, x);
+                if (j < Dc) rx = max64(rx, x + jp); else t = max64(t, x);
             }
             if (j + 1 < H) {
                 const long long y = ld_row<SMEM>(row + j + 1);
-                if (j + 1 < Dc) a1y = max64(a1y, y + j); else a2y = max64(a2y, y);
+                if (j + 1 < Dc) ry = max64(ry, y + jp); else t = max64(t, y);
             }
         }
     }
-    Peak2 r;
-    // the odd cell of each pair sits one step later: its "+ j" above lacks 1
-    r.a1 = max64(a1x, a1y == I64_MIN ? I64_MIN : a1y + 1);
-    r.a2 = max64(a2x, a2y);
-    return r;
-}
-
-// Scans chunks [c0, c1) of a group of consecutive rows that start at `base` (row stride H),
-// adding each row segment's maxima into bm1/bm2[first_row + row].
-template <bool FULL, bool SMEM>
-__device__ __forceinline__ void scan_chunk_range(const int64_t* __restrict__ base, int c0, int c1, int cpr,
-                                                 int first_row, int Dc, int H, int lane, long long* bm1,
-                                                 long long* bm2) {
-    int c = c0;
-    if (c >= c1) return;
-    int row = c / cpr;
-    int q0 = c - row * cpr;
-    while (c < c1) {
-        const int left = c1 - c;
-        const int q1 = (cpr - q0) < left ? cpr : q0 + left;
-        Peak2 v = scan_row_chunks<FULL, SMEM>(base + (size_t)row * H, q0, q1, Dc, H, lane);
-        v.a1 = warp_max64(v.a1);
-        v.a2 = warp_max64(v.a2);
-        if (lane == 0) {
-            atomicMax(&bm1[first_row + row], v.a1);
-            atomicMax(&bm2[first_row + row], v.a2);
-        }
-        c += q1 - q0;
-        ++row;
-        q0 = 0;
-    }
+    if (ry != I64_MIN) rx = max64(rx, ry + 1);
+    return max64(rx, t);
 }
 
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    long long* m1 = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows]  (by exchange parity)
-    long long* m2 = m1 + 2 * a.max_rows;                     // [2][max_rows]
-    long long* sq = m2 + 2 * a.max_rows;                     // queued_p of the owned rows
+    long long* pk = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows] peaks, by exchange parity
+    long long* sq = pk + 2 * a.max_rows;                     // queued_p of the owned rows
     long long* scd = sq + a.max_rows;                        // current_d of the owned rows
-    int64_t* res = reinterpret_cast<int64_t*>(scd + a.max_rows);  // [resident rows][H]; 48*max_rows bytes in: 16-byte aligned
+    int64_t* res = reinterpret_cast<int64_t*>(scd + a.max_rows);  // [resident rows][H]; 32*max_rows bytes in: 16-byte aligned
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
-    __shared__ long long sh_fix[2];  // re-scored (m1, m2) of the row that was just folded
+    __shared__ long long sh_fix;     // re-scored peak of the row that was just folded
 
     const int G = gridDim.x, b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -247,20 +220,16 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     const int S = a.resident_rows < nrows ? a.resident_rows : nrows;  // rows kept in shared memory
     const int cpr = (H + 63) >> 6;  // 64-cell chunks per row (one 16-byte load per lane)
     const bool full = (H & 63) == 0;
-    // chunk ranges of this warp (warps 1..): resident rows and streamed rows are split
-    // separately, since a resident chunk costs less than a streamed one
-    const int sw = warp - 1;
-    const int nchS = S * cpr, nchG = (nrows - S) * cpr;
-    const int s0 = warp ? (int)((long long)nchS * sw / SCAN_WARPS) : 0;
-    const int s1 = warp ? (int)((long long)nchS * (sw + 1) / SCAN_WARPS) : 0;
-    const int g0 = warp ? (int)((long long)nchG * sw / SCAN_WARPS) : 0;
-    const int g1 = warp ? (int)((long long)nchG * (sw + 1) / SCAN_WARPS) : 0;
-    const int64_t* grows = a.curves + (size_t)(row0 + S) * H;  // first streamed row
+    // chunk range of this warp (warps 1..) over the block's rows laid end to end
+    const int nch = nrows * cpr;
+    const int c0 = warp ? (int)((long long)nch * (warp - 1) / SCAN_WARPS) : 0;
+    const int c1 = warp ? (int)((long long)nch * warp / SCAN_WARPS) : 0;
+    const int first_row = c0 / cpr, first_q = c0 - first_row * cpr;
 
     for (int r = tid; r < nrows; r += ROUTE_THREADS) {
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
-        m1[r] = I64_MIN; m2[r] = I64_MIN;   // buffer 0, used by the first scan
+        pk[r] = I64_MIN;                    // buffer 0, used by the first scan
     }
     {   // resident copy of the first S rows
         const int64_t* src = a.curves + (size_t)row0 * H;
@@ -272,7 +241,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             for (int i = tid; i < total; i += ROUTE_THREADS) res[i] = __ldcg(src + i);
         }
     }
-    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN; }
+    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix = I64_MIN; }
     __syncthreads();
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
@@ -282,7 +251,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     bool saw_bad = false, saw_full = false;
     bool pending = false;         // an arrival has been published but not yet folded
     int pP = 0, pD = 0;           // ... its prompt and predicted lengths
-    long long pk = 0;             // ... its index in the batch
+    long long pidx = 0;           // ... its index in the batch
 
     // Collects the published minima of exchange `s` (warp 0 only); result in sh_winner/sh_score.
     auto gather = [&](long long s) {
@@ -329,15 +298,15 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
 
     // The winner w of the pending arrival is known: the owner really adds it to row w
     // (Sec. 4.3.1 update), block 0 records it.  When `rescore` is set, the same pass takes the
-    // folded row's maxima for the arrival being scored now (ramp length Dc) into sh_fix.
-    auto settle = [&](int w, bool rescore, int Dc) {
+    // folded row's peak for the arrival being scored now (P, ramp length Dc) into sh_fix.
+    auto settle = [&](int w, bool rescore, int P, int Dc) {
         if (w >= row0 && w < row1) {
             const int r = w - row0;
             int64_t* gp = a.curves + (size_t)w * H;
             int64_t* sp = res + (size_t)r * H;  // valid when r < S
             const bool in_smem = r < S;
             const int pDc = pD < H ? pD : H;
-            long long a1 = I64_MIN, a2 = I64_MIN;
+            long long pkv = I64_MIN;
             for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
                 long long c = in_smem ? sp[j] : __ldcg(gp + j);
                 if (j < pDc) {
@@ -345,12 +314,11 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                     gp[j] = c;
                     if (in_smem) sp[j] = c;
                 }
-                if (j < Dc) a1 = max64(a1, c + j); else a2 = max64(a2, c);
+                pkv = max64(pkv, j < Dc ? c + ((long long)P + j) : c);
             }
             if (rescore) {
-                a1 = warp_max64(a1);
-                a2 = warp_max64(a2);
-                if (lane == 0) { atomicMax(&sh_fix[0], a1); atomicMax(&sh_fix[1], a2); }
+                pkv = warp_max64(pkv);
+                if (lane == 0) atomicMax(&sh_fix, pkv);
             }
             if (tid == 0) {
                 sq[r] += pP;
@@ -365,8 +333,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             a.generated[slot] = 0;
             a.predicted[slot] = pD;
             a.instance[slot] = w;
-            a.choice[pk] = w;
-            if (a.score) a.score[pk] = sh_score;
+            a.choice[pidx] = w;
+            if (a.score) a.score[pidx] = sh_score;
         }
     };
 
@@ -384,46 +352,55 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         }
         const int Dc = D < H ? D : H;
         const int buf = (int)(seq & 1);
-        long long* bm1 = m1 + buf * a.max_rows;
-        long long* bm2 = m2 + buf * a.max_rows;
+        long long* bpk = pk + buf * a.max_rows;
 
         // ---- 1. scan for arrival k (the pending arrival is not folded yet) | collect its winner
         if (warp == 0) {
             if (pending) gather(seq - 1);
-        } else if (full) {
-            scan_chunk_range<true, true>(res, s0, s1, cpr, 0, Dc, H, lane, bm1, bm2);
-            scan_chunk_range<true, false>(grows, g0, g1, cpr, S, Dc, H, lane, bm1, bm2);
         } else {
-            scan_chunk_range<false, true>(res, s0, s1, cpr, 0, Dc, H, lane, bm1, bm2);
-            scan_chunk_range<false, false>(grows, g0, g1, cpr, S, Dc, H, lane, bm1, bm2);
+            int c = c0, row = first_row, q0 = first_q;
+            while (c < c1) {
+                const int left = c1 - c;
+                const int q1 = (cpr - q0) < left ? cpr : q0 + left;
+                long long v;
+                if (row < S) {
+                    const int64_t* rp = res + (size_t)row * H;
+                    v = full ? scan_row_chunks<true, true>(rp, q0, q1, P, Dc, H, lane)
+                             : scan_row_chunks<false, true>(rp, q0, q1, P, Dc, H, lane);
+                } else {
+                    const int64_t* rp = a.curves + (size_t)(row0 + row) * H;
+                    v = full ? scan_row_chunks<true, false>(rp, q0, q1, P, Dc, H, lane)
+                             : scan_row_chunks<false, false>(rp, q0, q1, P, Dc, H, lane);
+                }
+                v = warp_max64(v);
+                if (lane == 0) {
+                    if (q1 - q0 == cpr) bpk[row] = v;   // the whole row is this warp's
+                    else atomicMax(&bpk[row], v);
+                }
+                c += q1 - q0;
+                ++row;
+                q0 = 0;
+            }
         }
-        __syncthreads();  // S1: partial maxima of arrival k are in, winner of the pending arrival known
+        __syncthreads();  // S1: partial peaks of arrival k are in, winner of the pending arrival known
         if (sh_dead) break;
 
         // ---- 2. fold the pending arrival, re-score its row for arrival k; reset the other buffer
-        for (int r = tid; r < nrows; r += ROUTE_THREADS) {
-            m1[(buf ^ 1) * a.max_rows + r] = I64_MIN;
-            m2[(buf ^ 1) * a.max_rows + r] = I64_MIN;
-        }
+        for (int r = tid; r < nrows; r += ROUTE_THREADS) pk[(buf ^ 1) * a.max_rows + r] = I64_MIN;
         const int w = sh_winner;
-        if (pending) settle(w, true, Dc);
+        if (pending) settle(w, true, P, Dc);
         __syncthreads();  // S2: fold visible to the block, sh_fix complete
 
         // ---- 3. block minimum for arrival k, publish
         if (warp == 0) {
             if (pending && w >= row0 && w < row1) {
-                if (lane == 0) {
-                    bm1[w - row0] = sh_fix[0]; bm2[w - row0] = sh_fix[1];
-                    sh_fix[0] = I64_MIN; sh_fix[1] = I64_MIN;
-                }
+                if (lane == 0) { bpk[w - row0] = sh_fix; sh_fix = I64_MIN; }
                 __syncwarp();
             }
             double bs = CUDART_INF;
             int bi = 0x7fffffff;
             for (int r = lane; r < nrows; r += 32) {
-                long long peak = bm1[r] + P;  // Dc >= 1: the ramp part is never empty
-                if (bm2[r] > peak) peak = bm2[r];
-                const double s = score_of(sq[r], scd[r], peak, P, D, a.theta, a.beta);
+                const double s = score_of(sq[r], scd[r], bpk[r], P, D, a.theta, a.beta);
                 if (better(s, row0 + r, bs, bi)) { bs = s; bi = row0 + r; }
             }
             #pragma unroll
@@ -439,10 +416,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 st_release_u64(&slot[b * 2 + 1], ((unsigned long long)tag << 32) | (unsigned int)bi);
             }
         }
-        pending = true; pP = P; pD = D; pk = k;
+        pending = true; pP = P; pD = D; pidx = k;
         ++seq;
         // No barrier here: the other warps go on to the next scan (which fills the other
-        // (m1, m2) buffer) while warp 0 scores and publishes; sq/scd and sh_fix change only
+        // peak buffer) while warp 0 scores and publishes; sq/scd and sh_fix change only
         // between S1 and S2 or inside warp 0.
     }
 
@@ -451,7 +428,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         __syncthreads();
         if (warp == 0) gather(seq - 1);
         __syncthreads();
-        if (!sh_dead) settle(sh_winner, false, 0);
+        if (!sh_dead) settle(sh_winner, false, 0, 0);
     }
 
     if (b == 0 && tid == 0) {
@@ -468,7 +445,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
     const int max_rows = (I + G - 1) / G;
-    const size_t fixed = (size_t)max_rows * 6 * sizeof(long long);
+    const size_t fixed = (size_t)max_rows * 4 * sizeof(long long);
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
     if (e != cudaSuccess) return e;
