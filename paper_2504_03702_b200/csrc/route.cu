@@ -22,7 +22,8 @@
 //      publishes it in a slot tagged with the exchange number, while the other warps go on
 //      to the next scan.
 // Slots are double buffered by the tag's parity: a block publishes exchange s only after it
-// has read every slot of s-1, and nobody reads s-2 after publishing s-1.
+// has read every slot of s-1, and nobody reads s-2 after publishing s-1.  Every 64-bit word
+// of a slot carries the exchange tag, so the exchange needs no fence on either side.
 #include "pre_common.cuh"
 
 #include <math_constants.h>
@@ -33,15 +34,12 @@ constexpr int ROUTE_THREADS = 1024;
 constexpr int ROUTE_WARPS = ROUTE_THREADS / 32;
 constexpr int SCAN_WARPS = ROUTE_WARPS - 1;  // warp 0 coordinates
 constexpr long long I64_MIN = (-9223372036854775807LL - 1);
+constexpr long long I64_MAX = 9223372036854775807LL;
 constexpr unsigned int SPIN_LIMIT = 1u << 22;  // polls before a wait is declared lost
+constexpr int GATHER_ILP = 5;                  // exchange slots a lane polls at once
 
-__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
-    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
     unsigned long long v;
@@ -120,7 +118,7 @@ struct RouteArgs {
     double* score;
     int I, H;
     double theta, beta;
-    unsigned long long* slots;  // [2][G][2]
+    unsigned long long* slots;  // [2][G][4]: index, score high, score low (each tagged), unused
     unsigned int epoch;
     int* status;
     int* abort_flag;
@@ -199,12 +197,84 @@ __device__ __forceinline__ long long scan_row_chunks(const int64_t* __restrict__
     return max64(rx, t);
 }
 
+// The same scan when every cell of the row segment, with the arrival added, is known to lie
+// in [0, 2^32): only the low words take part, one 32-bit max per cell.  H is a multiple of 64.
+template <bool SMEM>
+__device__ __forceinline__ unsigned int scan_row_chunks_narrow(const int64_t* __restrict__ row, int q0, int q1,
+                                                               int P, int Dc, int lane) {
+    unsigned int rx = 0, ry = 0, t = 0, t2 = 0;   // all cells are >= 0, so 0 is a neutral start
+    bool any_ry = false;
+    const int qr = Dc >> 6, qt = (Dc + 63) >> 6;
+    const int64_t* p = row + lane * 2;
+    int q = q0;
+    const int e1 = q1 < qr ? q1 : qr;
+    any_ry = q < e1;
+    for (; q + 4 <= e1; q += 4) {
+        longlong2 v[4];
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
+        const unsigned int jp = (unsigned int)(q * 64 + lane * 2 + P);
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            rx = max(rx, (unsigned int)v[u].x + (jp + u * 64));
+            ry = max(ry, (unsigned int)v[u].y + (jp + u * 64));
+        }
+    }
+    for (; q < e1; ++q) {
+        const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+        const unsigned int jp = (unsigned int)(q * 64 + lane * 2 + P);
+        rx = max(rx, (unsigned int)v.x + jp);
+        ry = max(ry, (unsigned int)v.y + jp);
+    }
+    if (q < q1 && q < qt) {  // the one chunk that holds the end of the ramp
+        const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+        const int j = q * 64 + lane * 2;
+        const unsigned int jp = (unsigned int)(j + P);
+        if (j < Dc) rx = max(rx, (unsigned int)v.x + jp); else t = max(t, (unsigned int)v.x);
+        if (j + 1 < Dc) { ry = max(ry, (unsigned int)v.y + jp); any_ry = true; } else t = max(t, (unsigned int)v.y);
+        ++q;
+    }
+    for (; q + 4 <= q1; q += 4) {
+        longlong2 v[4];
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_row_v2<SMEM>(p + (q + u) * 64);
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) { t = max(t, (unsigned int)v[u].x); t2 = max(t2, (unsigned int)v[u].y); }
+    }
+    for (; q < q1; ++q) {
+        const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+        t = max(t, (unsigned int)v.x);
+        t2 = max(t2, (unsigned int)v.y);
+    }
+    if (any_ry) rx = max(rx, ry + 1);   // the odd cell of a pair sits one step later
+    return max(max(rx, t), t2);
+}
+
+// OR of the high words of chunks [q0, q1) of one row (zero: every cell lies in [0, 2^32)).
+template <bool SMEM>
+__device__ __forceinline__ unsigned int or_high_words(const int64_t* __restrict__ row, int q0, int q1, int lane) {
+    unsigned int acc = 0;
+    const int64_t* p = row + lane * 2;
+    for (int q = q0; q < q1; ++q) {
+        const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+        acc |= (unsigned int)((unsigned long long)v.x >> 32) | (unsigned int)((unsigned long long)v.y >> 32);
+    }
+    return acc;
+}
+
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     long long* pk = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows] peaks, by exchange parity
     long long* sq = pk + 2 * a.max_rows;                     // queued_p of the owned rows
     long long* scd = sq + a.max_rows;                        // current_d of the owned rows
-    int64_t* res = reinterpret_cast<int64_t*>(scd + a.max_rows);  // [resident rows][H]; 32*max_rows bytes in: 16-byte aligned
+    // bound[r]: an upper bound of row r's largest cell, or I64_MAX while none is known or the
+    // row has a cell outside [0, 2^32); rows with a small bound take the 32-bit scan.
+    long long* bound = scd + a.max_rows;
+    unsigned long long* wide = reinterpret_cast<unsigned long long*>(bound + a.max_rows);  // OR of high words
+    // order[L]: the L-th row of the scan order; resident and streamed rows alternate, so that
+    // every warp's stretch holds both kinds (a streamed chunk waits far longer for its data)
+    int* order = reinterpret_cast<int*>(wide + a.max_rows);
+    int64_t* res = reinterpret_cast<int64_t*>(order + ((a.max_rows + 3) & ~3));  // [resident rows][H], 16-byte aligned
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
@@ -230,6 +300,15 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
         pk[r] = I64_MIN;                    // buffer 0, used by the first scan
+        bound[r] = I64_MAX;
+        wide[r] = 0;
+        {
+            const int pairs = S < nrows - S ? S : nrows - S;   // r-th position of the scan order
+            int phys;
+            if (r < 2 * pairs) phys = (r & 1) ? S + (r >> 1) : (r >> 1);
+            else phys = S <= nrows - S ? r : r - pairs;         // the kind that is left over
+            order[r] = phys;
+        }
     }
     {   // resident copy of the first S rows
         const int64_t* src = a.curves + (size_t)row0 * H;
@@ -243,6 +322,23 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     }
     if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix = I64_MIN; }
     __syncthreads();
+    // Which rows hold only values in [0, 2^32)?  One pass over the block's rows.
+    if (warp && full) {
+        int c = c0, row = first_row, q0 = first_q;
+        while (c < c1) {
+            const int left = c1 - c;
+            const int q1 = (cpr - q0) < left ? cpr : q0 + left;
+            const int ph = order[row];
+            unsigned int acc = ph < S ? or_high_words<true>(res + (size_t)ph * H, q0, q1, lane)
+                                      : or_high_words<false>(a.curves + (size_t)(row0 + ph) * H, q0, q1, lane);
+            acc = __reduce_or_sync(0xffffffffu, acc);
+            if (lane == 0 && acc) atomicOr(&wide[ph], 1ull);
+            c += q1 - q0;
+            ++row;
+            q0 = 0;
+        }
+    }
+    __syncthreads();
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
     if (room < 0) room = 0;
@@ -254,31 +350,50 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     long long pidx = 0;           // ... its index in the batch
 
     // Collects the published minima of exchange `s` (warp 0 only); result in sh_winner/sh_score.
+    // A block's slot is three 64-bit words (index, score high, score low), each tagged with
+    // the exchange number, so a word is known to be current by itself and plain relaxed
+    // loads suffice; all of a lane's slots are polled at once.
     auto gather = [&](long long s) {
         const unsigned int tag = a.epoch + (unsigned int)s;
-        const unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 2;
+        const unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 4;
         bool lost = false;
         double bs = CUDART_INF;
         int bi = 0x7fffffff;
-        for (int cta = lane; cta < G && !lost; cta += 32) {
-            unsigned long long w1;
+        for (int base = 0; base < G && !lost; base += 32 * GATHER_ILP) {
+            unsigned long long w[GATHER_ILP][3];
             unsigned int polls = 0;
             for (;;) {
-                w1 = ld_acquire_u64(&slot[cta * 2 + 1]);
-                if ((unsigned int)(w1 >> 32) == tag) break;
-                if (++polls > SPIN_LIMIT || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag))) {
-                    lost = true;
-                    break;
+                bool all = true;
+                #pragma unroll
+                for (int i = 0; i < GATHER_ILP; ++i) {
+                    const int cta = base + lane + 32 * i;
+                    #pragma unroll
+                    for (int x = 0; x < 3; ++x)
+                        w[i][x] = cta < G ? ld_relaxed_u64(&slot[cta * 4 + x]) : ((unsigned long long)tag << 32);
                 }
+                #pragma unroll
+                for (int i = 0; i < GATHER_ILP; ++i) {
+                    #pragma unroll
+                    for (int x = 0; x < 3; ++x) all &= (unsigned int)(w[i][x] >> 32) == tag;
+                }
+                if (__all_sync(0xffffffffu, all)) break;
+                ++polls;
+                const bool give_up = polls > SPIN_LIMIT || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag));
+                if (__any_sync(0xffffffffu, give_up)) { lost = true; break; }
                 if (polls > 256) __nanosleep(64);
             }
-            if (!lost) {
-                const double sc = __longlong_as_double((long long)ld_relaxed_u64(&slot[cta * 2]));
-                const int i = (int)(unsigned int)(w1 & 0xffffffffu);
-                if (better(sc, i, bs, bi)) { bs = sc; bi = i; }
+            if (lost) break;
+            #pragma unroll
+            for (int i = 0; i < GATHER_ILP; ++i) {
+                const int cta = base + lane + 32 * i;
+                if (cta < G) {
+                    const unsigned long long bits = (w[i][1] << 32) | (w[i][2] & 0xffffffffull);
+                    const double sc = __longlong_as_double((long long)bits);
+                    const int idx = (int)(unsigned int)(w[i][0] & 0xffffffffu);
+                    if (better(sc, idx, bs, bi)) { bs = sc; bi = idx; }
+                }
             }
         }
-        lost = __any_sync(0xffffffffu, lost);
         #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
             const double os = __shfl_xor_sync(0xffffffffu, bs, off);
@@ -321,6 +436,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 if (lane == 0) atomicMax(&sh_fix, pkv);
             }
             if (tid == 0) {
+                if (bound[r] != I64_MAX) bound[r] += (long long)pP + pDc;  // the ramp adds less than this
                 sq[r] += pP;
                 scd[r] += pD;
                 a.queued_p[w] = sq[r];
@@ -363,19 +479,29 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 const int left = c1 - c;
                 const int q1 = (cpr - q0) < left ? cpr : q0 + left;
                 long long v;
-                if (row < S) {
-                    const int64_t* rp = res + (size_t)row * H;
-                    v = full ? scan_row_chunks<true, true>(rp, q0, q1, P, Dc, H, lane)
-                             : scan_row_chunks<false, true>(rp, q0, q1, P, Dc, H, lane);
+                // every cell with the arrival's ramp added stays below 2^32
+                const int ph = order[row];
+                const bool narrow = full && bound[ph] < (long long)0xffffffffu - P - H;
+                if (narrow) {
+                    const unsigned int u = ph < S
+                        ? scan_row_chunks_narrow<true>(res + (size_t)ph * H, q0, q1, P, Dc, lane)
+                        : scan_row_chunks_narrow<false>(a.curves + (size_t)(row0 + ph) * H, q0, q1, P, Dc, lane);
+                    v = (long long)__reduce_max_sync(0xffffffffu, u);
                 } else {
-                    const int64_t* rp = a.curves + (size_t)(row0 + row) * H;
-                    v = full ? scan_row_chunks<true, false>(rp, q0, q1, P, Dc, H, lane)
-                             : scan_row_chunks<false, false>(rp, q0, q1, P, Dc, H, lane);
+                    if (ph < S) {
+                        const int64_t* rp = res + (size_t)ph * H;
+                        v = full ? scan_row_chunks<true, true>(rp, q0, q1, P, Dc, H, lane)
+                                 : scan_row_chunks<false, true>(rp, q0, q1, P, Dc, H, lane);
+                    } else {
+                        const int64_t* rp = a.curves + (size_t)(row0 + ph) * H;
+                        v = full ? scan_row_chunks<true, false>(rp, q0, q1, P, Dc, H, lane)
+                                 : scan_row_chunks<false, false>(rp, q0, q1, P, Dc, H, lane);
+                    }
+                    v = warp_max64(v);
                 }
-                v = warp_max64(v);
                 if (lane == 0) {
-                    if (q1 - q0 == cpr) bpk[row] = v;   // the whole row is this warp's
-                    else atomicMax(&bpk[row], v);
+                    if (q1 - q0 == cpr) bpk[ph] = v;   // the whole row is this warp's
+                    else atomicMax(&bpk[ph], v);
                 }
                 c += q1 - q0;
                 ++row;
@@ -400,6 +526,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             double bs = CUDART_INF;
             int bi = 0x7fffffff;
             for (int r = lane; r < nrows; r += 32) {
+                // the peak with the arrival added is an upper bound of the row as it stands
+                if (wide[r] == 0) bound[r] = bpk[r];
                 const double s = score_of(sq[r], scd[r], bpk[r], P, D, a.theta, a.beta);
                 if (better(s, row0 + r, bs, bi)) { bs = s; bi = row0 + r; }
             }
@@ -409,11 +537,14 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
                 if (better(os, oi, bs, bi)) { bs = os; bi = oi; }
             }
-            if (lane == 0) {
+            if (lane < 3) {
+                // three words, each carrying the exchange tag: valid on its own, no fence needed
                 const unsigned int tag = a.epoch + (unsigned int)seq;  // dense: one tag per exchange
-                unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * 2;
-                slot[b * 2] = (unsigned long long)__double_as_longlong(bs);
-                st_release_u64(&slot[b * 2 + 1], ((unsigned long long)tag << 32) | (unsigned int)bi);
+                unsigned long long* slot = a.slots + ((size_t)(tag & 1u) * G + b) * 4;
+                const unsigned long long bits = (unsigned long long)__double_as_longlong(bs);
+                const unsigned int payload = lane == 0 ? (unsigned int)bi
+                                           : lane == 1 ? (unsigned int)(bits >> 32) : (unsigned int)bits;
+                st_relaxed_u64(&slot[lane], ((unsigned long long)tag << 32) | payload);
             }
         }
         pending = true; pP = P; pD = D; pidx = k;
@@ -445,7 +576,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
     const int max_rows = (I + G - 1) / G;
-    const size_t fixed = (size_t)max_rows * 4 * sizeof(long long);
+    const size_t fixed = (size_t)max_rows * 6 * sizeof(long long) + (size_t)((max_rows + 3) & ~3) * sizeof(int);
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
     if (e != cudaSuccess) return e;

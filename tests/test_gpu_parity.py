@@ -163,6 +163,21 @@ def test_route_shapes(seed, n_inst, h, n, a):
     st.close()
 
 
+@pytest.mark.parametrize("max_prompt,n", [(2 ** 27, 6000), (2 ** 24, 18000), (2 ** 24, 20000), (2 ** 20, 40000)])
+def test_route_values_around_and_above_32_bits(max_prompt, n):
+    """Rows whose cells cross 2^32 during the batch, start above it, or stay below it."""
+    wl = W.make_random(35, 40, 128, n, 400, max_prompt=max_prompt, max_output=300, capacity=10 ** 9)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    ap = (ap.astype(np.int64) * 4000 % (2 ** 27)).astype(np.int32)   # heavy arrivals push rows over the edge
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    want_c, want_s = ref.route_batch(ap, ad)
+    assert (choice.cpu().numpy() == want_c).all()
+    assert_scores_close(score.cpu().numpy(), want_s, want_c)
+    assert_state_equal(st, ref)
+    st.close()
+
+
 def test_route_fractional_threshold_and_beta_without_score_output():
     wl = W.make_random(31, 50, 24, 800, 300, capacity=33337, beta=0.75)
     wl.t_mem = 0.8
