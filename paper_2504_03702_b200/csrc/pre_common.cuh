@@ -27,7 +27,7 @@ struct pre_ctx {
     int route_blocks;    // G: blocks of the persistent routing kernel
     int route_threads;
     size_t route_smem;
-    int route_resident_rows;  // rows per routing block held in shared memory
+    size_t route_resident_bytes;  // shared memory per routing block left for resident rows
     double theta;        // t_mem * M in binary64
     uint32_t epoch;      // running arrival counter, tags the routing exchange slots
     int last_cuda_error;

@@ -123,7 +123,7 @@ struct RouteArgs {
     int* status;
     int* abort_flag;
     int max_rows;       // ceil(I / G)
-    int resident_rows;  // rows per block that fit in shared memory
+    size_t resident_bytes;  // shared memory per block left for resident rows
 };
 
 // Peak over 64-cell chunks [q0, q1) of one row with the arrival (P, Dc) virtually added
@@ -250,16 +250,71 @@ __device__ __forceinline__ unsigned int scan_row_chunks_narrow(const int64_t* __
     return max(max(rx, t), t2);
 }
 
-// OR of the high words of chunks [q0, q1) of one row (zero: every cell lies in [0, 2^32)).
-template <bool SMEM>
-__device__ __forceinline__ unsigned int or_high_words(const int64_t* __restrict__ row, int q0, int q1, int lane) {
-    unsigned int acc = 0;
+// The same again for a resident row kept as 32-bit cells (8-byte load = two cells per lane).
+__device__ __forceinline__ unsigned int scan_row_chunks_packed(const uint32_t* __restrict__ row, int q0, int q1,
+                                                               int P, int Dc, int lane) {
+    unsigned int rx = 0, ry = 0, t = 0, t2 = 0;
+    const int qr = Dc >> 6, qt = (Dc + 63) >> 6;
+    const unsigned int base = (unsigned int)__cvta_generic_to_shared(row + lane * 2);
+    auto ld2 = [&](int q) {
+        uint2 v;
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(base + q * 256) : "memory");
+        return v;
+    };
+    int q = q0;
+    const int e1 = q1 < qr ? q1 : qr;
+    bool any_ry = q < e1;
+    for (; q + 4 <= e1; q += 4) {
+        uint2 v[4];
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld2(q + u);
+        const unsigned int jp = (unsigned int)(q * 64 + lane * 2 + P);
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) { rx = max(rx, v[u].x + (jp + u * 64)); ry = max(ry, v[u].y + (jp + u * 64)); }
+    }
+    for (; q < e1; ++q) {
+        const uint2 v = ld2(q);
+        const unsigned int jp = (unsigned int)(q * 64 + lane * 2 + P);
+        rx = max(rx, v.x + jp);
+        ry = max(ry, v.y + jp);
+    }
+    if (q < q1 && q < qt) {  // the one chunk that holds the end of the ramp
+        const uint2 v = ld2(q);
+        const int j = q * 64 + lane * 2;
+        const unsigned int jp = (unsigned int)(j + P);
+        if (j < Dc) rx = max(rx, v.x + jp); else t = max(t, v.x);
+        if (j + 1 < Dc) { ry = max(ry, v.y + jp); any_ry = true; } else t = max(t, v.y);
+        ++q;
+    }
+    for (; q + 4 <= q1; q += 4) {
+        uint2 v[4];
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld2(q + u);
+        #pragma unroll
+        for (int u = 0; u < 4; ++u) { t = max(t, v[u].x); t2 = max(t2, v[u].y); }
+    }
+    for (; q < q1; ++q) {
+        const uint2 v = ld2(q);
+        t = max(t, v.x);
+        t2 = max(t2, v.y);
+    }
+    if (any_ry) rx = max(rx, ry + 1);
+    return max(max(rx, t), t2);
+}
+
+// OR of the high words and maximum of the low words of chunks [q0, q1) of one global row.
+// A zero OR means every cell lies in [0, 2^32) and the maximum is the true maximum.
+__device__ __forceinline__ void survey_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int lane,
+                                                  unsigned int* or_hi, unsigned int* max_lo) {
+    unsigned int acc = 0, m = 0;
     const int64_t* p = row + lane * 2;
     for (int q = q0; q < q1; ++q) {
-        const longlong2 v = ld_row_v2<SMEM>(p + q * 64);
+        const longlong2 v = ld_row_v2<false>(p + q * 64);
         acc |= (unsigned int)((unsigned long long)v.x >> 32) | (unsigned int)((unsigned long long)v.y >> 32);
+        m = max(m, max((unsigned int)v.x, (unsigned int)v.y));
     }
-    return acc;
+    *or_hi = acc;
+    *max_lo = m;
 }
 
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
@@ -267,19 +322,22 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     long long* pk = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows] peaks, by exchange parity
     long long* sq = pk + 2 * a.max_rows;                     // queued_p of the owned rows
     long long* scd = sq + a.max_rows;                        // current_d of the owned rows
-    // bound[r]: an upper bound of row r's largest cell, or I64_MAX while none is known or the
-    // row has a cell outside [0, 2^32); rows with a small bound take the 32-bit scan.
+    // bound[r]: an upper bound of row r's largest cell, or I64_MAX when the row has a cell
+    // outside [0, 2^32) (or H is not a multiple of 64); a small bound allows the 32-bit scans.
     long long* bound = scd + a.max_rows;
-    unsigned long long* wide = reinterpret_cast<unsigned long long*>(bound + a.max_rows);  // OR of high words
     // order[L]: the L-th row of the scan order; resident and streamed rows alternate, so that
     // every warp's stretch holds both kinds (a streamed chunk waits far longer for its data)
-    int* order = reinterpret_cast<int*>(wide + a.max_rows);
-    int64_t* res = reinterpret_cast<int64_t*>(order + ((a.max_rows + 3) & ~3));  // [resident rows][H], 16-byte aligned
+    int* order = reinterpret_cast<int*>(bound + a.max_rows);
+    // rstate[r]: RS_RESIDENT while the row's shared-memory copy is in use, RS_WIDE once the row
+    // is known to need 64 bits
+    int* rstate = order + a.max_rows;
+    unsigned char* res = reinterpret_cast<unsigned char*>(rstate + a.max_rows);  // 48*max_rows bytes in: 16-byte aligned
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
     __shared__ long long sh_fix;     // re-scored peak of the row that was just folded
+    constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
 
     const int G = gridDim.x, b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -287,7 +345,6 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     const int row0 = (int)(((long long)b * I) / G);
     const int row1 = (int)(((long long)(b + 1) * I) / G);
     const int nrows = row1 - row0;
-    const int S = a.resident_rows < nrows ? a.resident_rows : nrows;  // rows kept in shared memory
     const int cpr = (H + 63) >> 6;  // 64-cell chunks per row (one 16-byte load per lane)
     const bool full = (H & 63) == 0;
     // chunk range of this warp (warps 1..) over the block's rows laid end to end
@@ -300,42 +357,66 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
         pk[r] = I64_MIN;                    // buffer 0, used by the first scan
-        bound[r] = I64_MAX;
-        wide[r] = 0;
-        {
-            const int pairs = S < nrows - S ? S : nrows - S;   // r-th position of the scan order
-            int phys;
-            if (r < 2 * pairs) phys = (r & 1) ? S + (r >> 1) : (r >> 1);
-            else phys = S <= nrows - S ? r : r - pairs;         // the kind that is left over
-            order[r] = phys;
-        }
-    }
-    {   // resident copy of the first S rows
-        const int64_t* src = a.curves + (size_t)row0 * H;
-        const int total = S * H;
-        if ((H & 1) == 0) {
-            for (int i = tid * 2; i < total; i += ROUTE_THREADS * 2)
-                *reinterpret_cast<longlong2*>(res + i) = __ldcg(reinterpret_cast<const longlong2*>(src + i));
-        } else {
-            for (int i = tid; i < total; i += ROUTE_THREADS) res[i] = __ldcg(src + i);
-        }
+        bound[r] = full ? 0 : I64_MAX;      // the survey raises it
+        rstate[r] = full ? 0 : RS_WIDE;
     }
     if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix = I64_MIN; }
     __syncthreads();
-    // Which rows hold only values in [0, 2^32)?  One pass over the block's rows.
+    // Survey: which rows hold only values in [0, 2^32), and their maxima.  One pass over the
+    // block's rows in global memory.
     if (warp && full) {
         int c = c0, row = first_row, q0 = first_q;
         while (c < c1) {
             const int left = c1 - c;
             const int q1 = (cpr - q0) < left ? cpr : q0 + left;
-            const int ph = order[row];
-            unsigned int acc = ph < S ? or_high_words<true>(res + (size_t)ph * H, q0, q1, lane)
-                                      : or_high_words<false>(a.curves + (size_t)(row0 + ph) * H, q0, q1, lane);
-            acc = __reduce_or_sync(0xffffffffu, acc);
-            if (lane == 0 && acc) atomicOr(&wide[ph], 1ull);
+            unsigned int or_hi, max_lo;
+            survey_row_chunks(a.curves + (size_t)(row0 + row) * H, q0, q1, lane, &or_hi, &max_lo);
+            or_hi = __reduce_or_sync(0xffffffffu, or_hi);
+            max_lo = __reduce_max_sync(0xffffffffu, max_lo);
+            if (lane == 0) {
+                if (or_hi) atomicOr(&rstate[row], RS_WIDE);
+                atomicMax(&bound[row], (long long)max_lo);
+            }
             c += q1 - q0;
             ++row;
             q0 = 0;
+        }
+    }
+    __syncthreads();
+    // Resident rows: 32-bit cells when every row of the block fits them (twice as many rows
+    // stay on chip), else 64-bit cells.
+    bool any_wide = false;
+    for (int r = tid; r < nrows; r += ROUTE_THREADS) {
+        if (rstate[r] & RS_WIDE) { any_wide = true; bound[r] = I64_MAX; }
+    }
+    const bool packed = __syncthreads_or(any_wide) == 0;
+    const size_t row_bytes = (size_t)H * (packed ? 4 : 8);
+    const int S = (int)((size_t)nrows < a.resident_bytes / row_bytes ? (size_t)nrows : a.resident_bytes / row_bytes);
+    for (int r = tid; r < nrows; r += ROUTE_THREADS) {
+        if (r < S) rstate[r] |= RS_RESIDENT;
+        const int pairs = S < nrows - S ? S : nrows - S;   // r-th position of the scan order
+        int phys;
+        if (r < 2 * pairs) phys = (r & 1) ? S + (r >> 1) : (r >> 1);
+        else phys = S <= nrows - S ? r : r - pairs;         // the kind that is left over
+        order[r] = phys;
+    }
+    {
+        const int64_t* src = a.curves + (size_t)row0 * H;
+        const int total = S * H;
+        if (packed) {   // H is a multiple of 64 here
+            uint32_t* dst = reinterpret_cast<uint32_t*>(res);
+            for (int i = tid * 2; i < total; i += ROUTE_THREADS * 2) {
+                const longlong2 v = __ldcg(reinterpret_cast<const longlong2*>(src + i));
+                *reinterpret_cast<uint2*>(dst + i) = make_uint2((unsigned int)v.x, (unsigned int)v.y);
+            }
+        } else {
+            int64_t* dst = reinterpret_cast<int64_t*>(res);
+            if ((H & 1) == 0) {
+                for (int i = tid * 2; i < total; i += ROUTE_THREADS * 2)
+                    *reinterpret_cast<longlong2*>(dst + i) = __ldcg(reinterpret_cast<const longlong2*>(src + i));
+            } else {
+                for (int i = tid; i < total; i += ROUTE_THREADS) dst[i] = __ldcg(src + i);
+            }
         }
     }
     __syncthreads();
@@ -418,16 +499,23 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         if (w >= row0 && w < row1) {
             const int r = w - row0;
             int64_t* gp = a.curves + (size_t)w * H;
-            int64_t* sp = res + (size_t)r * H;  // valid when r < S
-            const bool in_smem = r < S;
             const int pDc = pD < H ? pD : H;
+            const int st = rstate[r];
+            const bool in_smem = (st & RS_RESIDENT) != 0;
+            // a packed row leaves shared memory when the fold may take a cell to 2^32
+            const bool evict = in_smem && packed && bound[r] + pP + pDc > 0xffffffffLL;
+            uint32_t* sp32 = reinterpret_cast<uint32_t*>(res) + (size_t)r * H;
+            int64_t* sp64 = reinterpret_cast<int64_t*>(res) + (size_t)r * H;
             long long pkv = I64_MIN;
             for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
-                long long c = in_smem ? sp[j] : __ldcg(gp + j);
+                long long c = !in_smem ? __ldcg(gp + j) : packed ? (long long)sp32[j] : sp64[j];
                 if (j < pDc) {
                     c += (long long)pP + j;
                     gp[j] = c;
-                    if (in_smem) sp[j] = c;
+                    if (in_smem) {
+                        if (!packed) sp64[j] = c;
+                        else if (!evict) sp32[j] = (uint32_t)c;
+                    }
                 }
                 pkv = max64(pkv, j < Dc ? c + ((long long)P + j) : c);
             }
@@ -435,7 +523,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 pkv = warp_max64(pkv);
                 if (lane == 0) atomicMax(&sh_fix, pkv);
             }
+            __syncthreads();   // block-uniform branch; every thread has read rstate/bound above
             if (tid == 0) {
+                if (evict) rstate[r] = st & ~RS_RESIDENT;
                 if (bound[r] != I64_MAX) bound[r] += (long long)pP + pDc;  // the ramp adds less than this
                 sq[r] += pP;
                 scd[r] += pD;
@@ -478,24 +568,32 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             while (c < c1) {
                 const int left = c1 - c;
                 const int q1 = (cpr - q0) < left ? cpr : q0 + left;
-                long long v;
-                // every cell with the arrival's ramp added stays below 2^32
                 const int ph = order[row];
-                const bool narrow = full && bound[ph] < (long long)0xffffffffu - P - H;
-                if (narrow) {
-                    const unsigned int u = ph < S
-                        ? scan_row_chunks_narrow<true>(res + (size_t)ph * H, q0, q1, P, Dc, lane)
-                        : scan_row_chunks_narrow<false>(a.curves + (size_t)(row0 + ph) * H, q0, q1, P, Dc, lane);
+                // every cell with the arrival's ramp added stays below 2^32
+                const bool narrow = bound[ph] < (long long)0xffffffffu - P - H;
+                const bool in_smem = (rstate[ph] & RS_RESIDENT) != 0;
+                const int64_t* gp = a.curves + (size_t)(row0 + ph) * H;
+                long long v;
+                if (in_smem && packed) {
+                    if (narrow) {
+                        const uint32_t* rp = reinterpret_cast<const uint32_t*>(res) + (size_t)ph * H;
+                        v = (long long)__reduce_max_sync(0xffffffffu, scan_row_chunks_packed(rp, q0, q1, P, Dc, lane));
+                    } else {   // this arrival's ramp would overflow 32 bits: take the row from global memory
+                        v = warp_max64(scan_row_chunks<true, false>(gp, q0, q1, P, Dc, H, lane));
+                    }
+                } else if (narrow) {
+                    const unsigned int u = in_smem
+                        ? scan_row_chunks_narrow<true>(reinterpret_cast<const int64_t*>(res) + (size_t)ph * H, q0, q1, P, Dc, lane)
+                        : scan_row_chunks_narrow<false>(gp, q0, q1, P, Dc, lane);
                     v = (long long)__reduce_max_sync(0xffffffffu, u);
                 } else {
-                    if (ph < S) {
-                        const int64_t* rp = res + (size_t)ph * H;
+                    if (in_smem) {
+                        const int64_t* rp = reinterpret_cast<const int64_t*>(res) + (size_t)ph * H;
                         v = full ? scan_row_chunks<true, true>(rp, q0, q1, P, Dc, H, lane)
                                  : scan_row_chunks<false, true>(rp, q0, q1, P, Dc, H, lane);
                     } else {
-                        const int64_t* rp = a.curves + (size_t)(row0 + ph) * H;
-                        v = full ? scan_row_chunks<true, false>(rp, q0, q1, P, Dc, H, lane)
-                                 : scan_row_chunks<false, false>(rp, q0, q1, P, Dc, H, lane);
+                        v = full ? scan_row_chunks<true, false>(gp, q0, q1, P, Dc, H, lane)
+                                 : scan_row_chunks<false, false>(gp, q0, q1, P, Dc, H, lane);
                     }
                     v = warp_max64(v);
                 }
@@ -527,7 +625,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             int bi = 0x7fffffff;
             for (int r = lane; r < nrows; r += 32) {
                 // the peak with the arrival added is an upper bound of the row as it stands
-                if (wide[r] == 0) bound[r] = bpk[r];
+                if (!(rstate[r] & RS_WIDE)) bound[r] = bpk[r];
                 const double s = score_of(sq[r], scd[r], bpk[r], P, D, a.theta, a.beta);
                 if (better(s, row0 + r, bs, bi)) { bs = s; bi = row0 + r; }
             }
@@ -576,7 +674,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
     const int max_rows = (I + G - 1) / G;
-    const size_t fixed = (size_t)max_rows * 6 * sizeof(long long) + (size_t)((max_rows + 3) & ~3) * sizeof(int);
+    const size_t fixed = (size_t)max_rows * 48;  // five 8-byte and two 4-byte words per row
     cudaDeviceProp prop;
     cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
     if (e != cudaSuccess) return e;
@@ -585,10 +683,11 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     if (e != cudaSuccess) return e;
     const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
     if (fixed + attr.sharedSizeBytes + 1024 > limit) return cudaErrorInvalidConfiguration;
-    // rows kept in shared memory: whatever fits beside the fixed part
-    size_t resident = (limit - attr.sharedSizeBytes - 1024 - fixed) / ((size_t)H * sizeof(int64_t));
-    if (resident > (size_t)max_rows) resident = (size_t)max_rows;
-    const size_t smem = fixed + resident * (size_t)H * sizeof(int64_t);
+    // what is left beside the fixed part holds resident rows (the kernel decides how many)
+    size_t resident_bytes = limit - attr.sharedSizeBytes - 1024 - fixed;
+    if (resident_bytes > (size_t)max_rows * H * sizeof(int64_t)) resident_bytes = (size_t)max_rows * H * sizeof(int64_t);
+    resident_bytes &= ~(size_t)15;
+    const size_t smem = fixed + resident_bytes;
     e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
@@ -598,7 +697,7 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     ctx->route_blocks = G;
     ctx->route_threads = ROUTE_THREADS;
     ctx->route_smem = smem;
-    ctx->route_resident_rows = (int)resident;
+    ctx->route_resident_bytes = resident_bytes;
     return cudaSuccess;
 }
 
@@ -620,7 +719,7 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
     a.slots = ctx->d_slots; a.epoch = ctx->epoch;
     a.status = ctx->d_status; a.abort_flag = ctx->d_abort;
     a.max_rows = (a.I + ctx->route_blocks - 1) / ctx->route_blocks;
-    a.resident_rows = ctx->route_resident_rows;
+    a.resident_bytes = ctx->route_resident_bytes;
     ctx->epoch += (unsigned int)n_arrivals;
     void* params[] = {(void*)&a};
     return cudaLaunchCooperativeKernel((const void*)pre_route_persistent, dim3(ctx->route_blocks),
