@@ -132,6 +132,11 @@ def run_reference(args, wl, rank):
 
 METRIC = "routes/sec over the whole step (anticipate + route batch + decode step)"
 
+# DRAM bytes (read + write) of one pre_route_persistent launch on the full batch of a
+# configuration, from an ncu capture (profiles/): the kernel reads the maps once and writes
+# only the folded cells and the appended requests.  None: not captured for the kernel as it stands.
+ROUTE_DRAM_TRAFFIC = {}
+
 
 def config_dict(wl, args):
     return {"workload": f"config {args.config} ({wl.name}): {wl.n_instances} instances, H={wl.horizon}, "
@@ -304,15 +309,19 @@ def main():
         "parts_ms": {"anticipate": t_build, "route_batch": t_route, "step": t_dstep},
         "anticipated_request_steps_per_s": world * wl.n_requests * wl.horizon / (t_build * 1e-3),
         "routes_per_s_route_call_only": world * a / (t_route * 1e-3),
-        "roofline": dict(roof(b_route, t_route, 1), kernel="pre_route_persistent",
-                         note="the 64 MiB of maps are re-read once per arrival; when they stay resident in the "
-                              "126 MB L2 the achieved figure is L2-served and may exceed the HBM peak"),
-        "roofline_anticipate": dict(roof(b_build, t_build, 4), kernel="pre_bin_count + pre_bin_scan + "
-                                                                       "pre_bin_scatter + pre_tile_build"),
+        "roofline": dict(roof(b_route, t_route, 1, ROUTE_DRAM_TRAFFIC.get(args.config) if args.arrivals == 0 else None),
+                         kernel="pre_route_persistent", served_from="shared memory",
+                         limiter="latency of the per-arrival exchange between the blocks",
+                         note="achieved = bytes of the literal scan (every arrival reads all I*H map cells) over "
+                              "time. The maps are copied on chip once per batch (packed to 32-bit cells when they "
+                              "fit) and every scan reads them from shared memory, so the figure is a scan-equivalent "
+                              "rate, not HBM traffic, and exceeds the HBM peak; 'traffic' is the DRAM traffic of "
+                              "the whole launch from an ncu capture scaled to this batch"),
+        "roofline_anticipate": dict(roof(b_build, t_build, 2), kernel="pre_chunk_sort + pre_tile_build"),
         "roofline_step": dict(roof(b_step, t_dstep, 2), kernel="pre_step_requests + pre_step_shift"),
         "e2e": {"value": world * a / (t_e2e * 1e-3), "unit": "routes/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": 5 * args.steps,
         "clocks": clocks,
         "wall_s_timed_region": wall1 - wall0,
         "routed": routed_ok,

@@ -507,9 +507,19 @@ cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int
 }
 
 cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
-    cudaError_t e = cudaFuncSetAttribute(pre_chunk_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)sort_smem_bytes(PRE_SMEM_BINS, 1));
+    // The limit is a property of the kernel, shared by every context of the process: always
+    // raise it to the device maximum, so that contexts of different shapes do not undo each other.
+    int optin = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device);
+    if (e != cudaSuccess) return e;
+    cudaFuncAttributes attr;
+    e = cudaFuncGetAttributes(&attr, pre_chunk_sort);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(pre_chunk_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             optin - (int)attr.sharedSizeBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncGetAttributes(&attr, pre_tile_build);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)pre_tile_smem_bytes(ctx->tile_rows, ctx->cfg.horizon));
+                                optin - (int)attr.sharedSizeBytes);
 }

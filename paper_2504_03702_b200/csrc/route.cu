@@ -688,7 +688,9 @@ cudaError_t pre_route_configure(pre_ctx* ctx) {
     if (resident_bytes > (size_t)max_rows * H * sizeof(int64_t)) resident_bytes = (size_t)max_rows * H * sizeof(int64_t);
     resident_bytes &= ~(size_t)15;
     const size_t smem = fixed + resident_bytes;
-    e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // (the limit is shared by every context of the process: always the device maximum)
+    e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(limit - attr.sharedSizeBytes));
     if (e != cudaSuccess) return e;
     int per_sm = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pre_route_persistent, ROUTE_THREADS, smem);

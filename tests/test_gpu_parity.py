@@ -111,6 +111,23 @@ def test_anticipate_prefix_of_table():
     st.close()
 
 
+def test_two_contexts_of_different_shapes():
+    """Kernel attributes are process-wide: a second, smaller context must not break the first."""
+    big = W.make_random(17, 64, 2048, 3000, 50, max_output=3000)
+    small = W.make_random(18, 5, 64, 200, 20)
+    st_big, ref_big = both(big)
+    st_small, ref_small = both(small)
+    st_big.anticipate()
+    c, _ = st_big.route_batch(dev(big.ticks[0][0]), dev(big.ticks[0][1]))
+    assert (c.cpu().numpy() == ref_big.route_batch(*big.ticks[0])[0]).all()
+    c, _ = st_small.route_batch(dev(small.ticks[0][0]), dev(small.ticks[0][1]))
+    assert (c.cpu().numpy() == ref_small.route_batch(*small.ticks[0])[0]).all()
+    assert_state_equal(st_big, ref_big)
+    assert_state_equal(st_small, ref_small)
+    st_big.close()
+    st_small.close()
+
+
 def test_argument_errors_launch_nothing():
     wl = W.make_random(15, 4, 16, 10, 0)
     st = DeviceState.from_workload(wl)
