@@ -49,7 +49,8 @@ typedef enum pre_error {
     PRE_EBADREQ = -3,   /* a malformed request or arrival was skipped                        */
     PRE_ETIMEOUT = -4,  /* a bounded device-side wait ran out; the batch was abandoned       */
     PRE_ECUDA = -5,     /* a CUDA runtime call failed (see pre_last_cuda_error)              */
-    PRE_ENOMEM = -6     /* scratch allocation failed in pre_create                           */
+    PRE_ENOMEM = -6,    /* scratch allocation failed in pre_create                           */
+    PRE_ESIZE = -7      /* problem larger than the built-in scratch of pre_anticipate_static */
 } pre_error;
 
 typedef struct pre_ctx pre_ctx; /* opaque; owns only internal device scratch */
@@ -82,6 +83,38 @@ int pre_destroy(pre_ctx* ctx);
 int pre_anticipate(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated,
                    const int32_t* d_predicted, const int32_t* d_instance, int64_t n_requests,
                    int64_t* d_curves, int64_t* d_current_d, void* stream);
+
+/* pre_anticipate without a context and without any allocation.  (The paper has no counterpart:
+ * this entry point exists for the sake of its callers, it computes exactly what pre_anticipate
+ * computes.)
+ *
+ * Who needs it: code that runs where device memory may not be requested or returned - for
+ * example a plug-in inside a serving engine that has handed the whole GPU to its own pool
+ * allocator, a callback that runs while the CUDA allocator's lock is held, or a latency-critical
+ * control loop where a cudaMalloc (which can synchronise the device) is not acceptable.
+ * pre_create allocates scratch; this call uses scratch that is part of the library image
+ * instead, about 2.6 MB that every GPU which loads the library holds until the process exits.
+ *
+ * Limits (PRE_ESIZE beyond them): n_requests <= 262,144; at most 2,048 build tiles, which
+ * covers n_instances * horizon up to roughly 8 million cells (e.g. 4,096 x 2,048); device
+ * ordinal below 64.  horizon <= 8192 as everywhere.
+ *
+ * Arguments as for pre_anticipate, with the shape passed directly.  d_flags (DEVICE int32,
+ * may be NULL, zeroed by the caller) receives a non-zero value if a malformed request was
+ * skipped.  The call launches on `stream` and returns without synchronising; it calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ * The first call on each device, made with that device current, looks up the device address
+ * of the built-in scratch and raises the kernels' shared-memory limits; make that first call
+ * before any stream capture begins.  All calls on a device share the one scratch area, which
+ * keeps whatever the last call left in it: two calls whose work overlaps on the GPU (different
+ * streams, or different host threads) race and give wrong maps - order them on one stream or
+ * with events.  Nothing in the scratch needs clearing between calls.  As with the other
+ * entry points, do not call it from two host threads at the same time. */
+int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d_prompt,
+                          const int32_t* d_generated, const int32_t* d_predicted, const int32_t* d_instance,
+                          int64_t n_requests, int64_t* d_curves, int64_t* d_current_d, int32_t* d_flags,
+                          void* stream);
 
 /* Routes n_arrivals requests in array order (Sec. 4.3.3).  For arrival (P, D) and every
  * instance i the anticipator "virtually" adds the request to the map and takes the peak

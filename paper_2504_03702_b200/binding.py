@@ -12,10 +12,10 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpreserve_b200.so")
 
-PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENOMEM = 0, -1, -2, -3, -4, -5, -6
+PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENOMEM, PRE_ESIZE = 0, -1, -2, -3, -4, -5, -6, -7
 
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
-           "pre_last_cuda_error", "pre_strerror", "pre_query")
+           "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static")
 
 
 class pre_config(C.Structure):
@@ -33,6 +33,7 @@ def _load():
     lib.pre_create.argtypes = [C.POINTER(pre_config), C.POINTER(vp)]
     lib.pre_destroy.argtypes = [vp]
     lib.pre_anticipate.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
+    lib.pre_anticipate_static.argtypes = [C.c_int32, C.c_int32, vp, vp, vp, vp, i64, vp, vp, vp, vp]
     lib.pre_route_batch.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
@@ -90,6 +91,14 @@ def pre_anticipate(ctx, prompt, generated, predicted, instance, n_requests, curv
     return lib.pre_anticipate(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance),
                               int(n_requests), _ptr(curves), _ptr(current_d),
                               _stream() if stream is None else stream)
+
+
+def pre_anticipate_static(n_instances, horizon, prompt, generated, predicted, instance, n_requests, curves,
+                          current_d, flags=None, stream=None):
+    """pre_anticipate for callers that must not allocate: no context, scratch built into the library."""
+    return lib.pre_anticipate_static(int(n_instances), int(horizon), _ptr(prompt), _ptr(generated),
+                                     _ptr(predicted), _ptr(instance), int(n_requests), _ptr(curves),
+                                     _ptr(current_d), _ptr(flags), _stream() if stream is None else stream)
 
 
 def pre_route_batch(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,

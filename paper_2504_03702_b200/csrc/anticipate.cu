@@ -523,3 +523,108 @@ cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
     return cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 optin - (int)attr.sharedSizeBytes);
 }
+
+// ---------------------------------------------------------------------------------------
+// pre_anticipate_static: the same build for callers that must not allocate.
+//
+// Its scratch (the packed, tile-ordered requests and the per-chunk tile offsets) lives in
+// one array that is part of the library image: every GPU that loads the library holds these
+// bytes until the process exits.  The sizes below are therefore deliberately modest.
+constexpr int PRE_STATIC_MAX_REQUESTS = 262144;   // table rows one call may cover
+constexpr int PRE_STATIC_MAX_TILES = 2048;        // build tiles one call may need
+constexpr int PRE_STATIC_MAX_CHUNKS = PRE_STATIC_MAX_REQUESTS / SORT_CHUNK;   // 64
+constexpr size_t PRE_STATIC_STATUS_BYTES = 256;
+constexpr size_t PRE_STATIC_OFF_BYTES = (size_t)(PRE_STATIC_MAX_TILES + 1) * PRE_STATIC_MAX_CHUNKS * sizeof(unsigned int);
+constexpr size_t PRE_STATIC_REC_BYTES = (size_t)PRE_STATIC_MAX_REQUESTS * sizeof(unsigned long long);
+constexpr size_t PRE_STATIC_BYTES = PRE_STATIC_STATUS_BYTES + ((PRE_STATIC_OFF_BYTES + 255) & ~(size_t)255) + PRE_STATIC_REC_BYTES;
+
+static __device__ __align__(256) unsigned char pre_static_scratch[PRE_STATIC_BYTES];
+
+namespace {
+
+constexpr int PRE_STATIC_MAX_DEVICES = 64;
+
+struct StaticSetup {
+    bool ready;
+    unsigned char* base;   // device address of pre_static_scratch on this device
+    int n_sm;
+    int smem_optin;
+};
+StaticSetup g_static_setup[PRE_STATIC_MAX_DEVICES];
+
+// Once per device, with that device current.  In host code `pre_static_scratch` is only a
+// handle of the symbol, not an address the GPU can use: the device address has to be asked for.
+cudaError_t static_setup(int device, StaticSetup** out) {
+    StaticSetup* st = &g_static_setup[device];
+    if (!st->ready) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, pre_static_scratch);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&st->n_sm, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&st->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        if (e != cudaSuccess) return e;
+        cudaFuncAttributes attr;
+        e = cudaFuncGetAttributes(&attr, pre_chunk_sort);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(pre_chunk_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 st->smem_optin - (int)attr.sharedSizeBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncGetAttributes(&attr, pre_tile_build);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 st->smem_optin - (int)attr.sharedSizeBytes);
+        if (e != cudaSuccess) return e;
+        st->base = static_cast<unsigned char*>(p);
+        st->ready = true;
+    }
+    *out = st;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d_prompt,
+                                     const int32_t* d_generated, const int32_t* d_predicted,
+                                     const int32_t* d_instance, int64_t n_requests, int64_t* d_curves,
+                                     int64_t* d_current_d, int32_t* d_flags, void* stream) {
+    if (n_instances < 1 || horizon < 1 || horizon > PRE_MAX_HORIZON) return PRE_EINVAL;
+    if (n_requests < 0 || !d_curves || !d_current_d) return PRE_EINVAL;
+    if (n_requests > 0 && (!d_prompt || !d_generated || !d_predicted || !d_instance)) return PRE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_curves) & 15) || (reinterpret_cast<uintptr_t>(d_current_d) & 7) ||
+        (reinterpret_cast<uintptr_t>(d_flags) & 3) || (reinterpret_cast<uintptr_t>(d_prompt) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_generated) & 3) || (reinterpret_cast<uintptr_t>(d_predicted) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_instance) & 3))
+        return PRE_EINVAL;
+    if (n_requests > PRE_STATIC_MAX_REQUESTS) return PRE_ESIZE;
+
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return PRE_ECUDA;
+    if (device < 0 || device >= PRE_STATIC_MAX_DEVICES) return PRE_ESIZE;
+    StaticSetup* st = nullptr;
+    if (static_setup(device, &st) != cudaSuccess) return PRE_ECUDA;
+
+    const int T = pre_tile_rows_for(n_instances, horizon, st->n_sm);
+    const int n_tiles = (n_instances + T - 1) / T;
+    if (n_tiles > PRE_STATIC_MAX_TILES) return PRE_ESIZE;
+    const size_t tile_smem = pre_tile_smem_bytes(T, horizon);
+    if (tile_smem > (size_t)st->smem_optin) return PRE_EINVAL;
+
+    int nc = 1, staged = 1;
+    int64_t chunk = 4;
+    sort_geometry(n_requests, &nc, &chunk, &staged);   // nc <= 64 and staged, given the request limit
+
+    int* status = d_flags ? d_flags : reinterpret_cast<int*>(st->base);
+    unsigned int* chunk_off = reinterpret_cast<unsigned int*>(st->base + PRE_STATIC_STATUS_BYTES);
+    unsigned long long* records = reinterpret_cast<unsigned long long*>(
+        st->base + PRE_STATIC_STATUS_BYTES + ((PRE_STATIC_OFF_BYTES + 255) & ~(size_t)255));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Nothing in the scratch has to start at zero: pre_chunk_sort writes every offset that
+    // pre_tile_build reads, and a record is read only where an offset says one was written.
+    pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(n_tiles, staged), s>>>(
+        d_prompt, d_generated, d_predicted, d_instance, n_requests, n_instances, T, n_tiles, chunk, staged, records,
+        chunk_off, status);
+    pre_tile_build<<<n_tiles, TILE_THREADS, tile_smem, s>>>(records, chunk_off, nc, chunk, nullptr, nullptr, nullptr,
+                                                          n_instances, horizon, T, d_curves, d_current_d);
+    return cudaGetLastError() == cudaSuccess ? PRE_OK : PRE_ECUDA;
+}

@@ -170,6 +170,7 @@ const char* pre_strerror(int code) {
         case PRE_ETIMEOUT: return "a bounded device-side wait ran out; the batch was abandoned";
         case PRE_ECUDA: return "CUDA runtime error";
         case PRE_ENOMEM: return "out of memory";
+        case PRE_ESIZE: return "problem larger than the built-in scratch of pre_anticipate_static";
         default: return "unknown error code";
     }
 }
