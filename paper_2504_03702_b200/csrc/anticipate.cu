@@ -135,7 +135,7 @@ pre_bin_scatter(const int32_t* __restrict__ prompt, const int32_t* __restrict__ 
 // tile t, the offset of t's first record inside the span: chunk_off[t*NC + ch]
 // (chunk_off[n_tiles*NC + ch] = number of live requests of the chunk).
 constexpr int SORT_THREADS = 512;
-constexpr int SORT_CHUNK = 4096;   // requests a block can stage in shared memory
+constexpr int SORT_CHUNK = 6144;   // requests a block can stage in shared memory
 constexpr int SORT_MAX_CHUNKS = 1024;
 
 __global__ void __launch_bounds__(SORT_THREADS)
@@ -230,9 +230,19 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
     // ---- pass B: place
     unsigned long long* out = records + r0;
     if (staged) {
-        for (int li = tid; li < (int)(r1 - r0); li += SORT_THREADS) {
-            const unsigned int t = tile_of[li];
-            if (t != 0xFFFFu) out[atomicAdd(&hist[t], 1u)] = stage[li];
+        const int cnt = (int)(r1 - r0);
+        for (int l0 = tid; l0 < cnt; l0 += 4 * SORT_THREADS) {   // four independent cursor bumps in flight
+            unsigned int t[4], pos[4];
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int li = l0 + u * SORT_THREADS;
+                t[u] = li < cnt ? tile_of[li] : 0xFFFFu;
+            }
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) pos[u] = t[u] != 0xFFFFu ? atomicAdd(&hist[t[u]], 1u) : 0u;
+            #pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (t[u] != 0xFFFFu) out[pos[u]] = stage[l0 + u * SORT_THREADS];
         }
     } else {
         for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
@@ -319,10 +329,18 @@ pre_tile_build(const unsigned long long* __restrict__ records,
     if (chunk_off != nullptr) {
         const unsigned int* o0 = chunk_off + (size_t)tile * NC;
         const unsigned int* o1 = o0 + NC;
+        // A tile has a few records per chunk (about n / (tiles * chunks)): take up to four with
+        // independent loads, then whatever is left one by one.
         for (int ch = tid; ch < NC; ch += TILE_THREADS) {
             const unsigned int a = o0[ch], b = o1[ch];
-            const unsigned long long* src = records + (size_t)ch * chunk;
-            for (unsigned int r = a; r < b; ++r) add_record(src[r]);
+            const unsigned long long* src = records + (size_t)ch * chunk + a;
+            const unsigned int len = b - a;
+            unsigned long long rec[4];
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) rec[u] = (unsigned int)u < len ? src[u] : 0ull;
+            #pragma unroll
+            for (int u = 0; u < 4; ++u) if ((unsigned int)u < len) add_record(rec[u]);
+            for (unsigned int r = 4; r < len; ++r) add_record(src[r]);
         }
     } else {
         const unsigned int rec0 = bin_base[tile];
@@ -413,8 +431,9 @@ pre_tile_build(const unsigned long long* __restrict__ records,
         const int half = sh.hp >> 1;  // cell pairs per padded row
         const int total = rows * half;
         const bool vec_gl = (H & 1) == 0;
+        const int shift = (half & (half - 1)) == 0 ? 31 - __clz(half) : -1;  // log2 when a power of two
         for (int p = tid; p < total; p += TILE_THREADS) {
-            const int row = p / half;
+            const int row = shift >= 0 ? p >> shift : p / half;
             const int j = (p - row * half) << 1;
             if (j < H) {
                 const int c = row * sh.hp + j;
@@ -452,9 +471,15 @@ int pre_tile_rows_for(int n_instances, int horizon, int n_sm) {
     return t < by_grid ? t : by_grid;
 }
 
-static void sort_geometry(int64_t n, int* n_chunks, int64_t* chunk, int* staged) {
+// How the table is cut into chunks: enough chunks that each fits the staging buffer, and, when
+// the table allows it, as many as the GPU runs blocks at once (`slots`), so that the sort is a
+// single wave; never more than `max_chunks` (the width of the offset table).
+static void sort_geometry(int64_t n, int slots, int max_chunks, int* n_chunks, int64_t* chunk, int* staged) {
     int64_t nc = (n + SORT_CHUNK - 1) / SORT_CHUNK;
-    if (nc > SORT_MAX_CHUNKS) nc = SORT_MAX_CHUNKS;
+    int64_t wave = (n + 1023) / 1024;            // but no chunk below ~1024 requests
+    if (wave > slots) wave = slots;
+    if (nc < wave) nc = wave;
+    if (nc > max_chunks) nc = max_chunks;
     if (nc < 1) nc = 1;
     int64_t c = (n + nc - 1) / nc;
     c = (c + 3) & ~(int64_t)3;
@@ -480,7 +505,7 @@ cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int
     if (nt <= PRE_SMEM_BINS) {
         int nc = 1, staged = 1;
         int64_t chunk = 4;
-        sort_geometry(n, &nc, &chunk, &staged);
+        sort_geometry(n, 3 * ctx->n_sm, SORT_MAX_CHUNKS, &nc, &chunk, &staged);
         // With n == 0 the single chunk is empty: its offsets are all zero and every tile writes zero rows.
         pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(nt, staged), s>>>(
             prompt, generated, predicted, instance, n, I, T, nt, chunk, staged, ctx->d_records, ctx->d_chunk_off,
@@ -532,7 +557,7 @@ cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
 // bytes until the process exits.  The sizes below are therefore deliberately modest.
 constexpr int PRE_STATIC_MAX_REQUESTS = 262144;   // table rows one call may cover
 constexpr int PRE_STATIC_MAX_TILES = 2048;        // build tiles one call may need
-constexpr int PRE_STATIC_MAX_CHUNKS = PRE_STATIC_MAX_REQUESTS / SORT_CHUNK;   // 64
+constexpr int PRE_STATIC_MAX_CHUNKS = 64;          // chunks of at most 4,096 requests
 constexpr size_t PRE_STATIC_STATUS_BYTES = 256;
 constexpr size_t PRE_STATIC_OFF_BYTES = (size_t)(PRE_STATIC_MAX_TILES + 1) * PRE_STATIC_MAX_CHUNKS * sizeof(unsigned int);
 constexpr size_t PRE_STATIC_REC_BYTES = (size_t)PRE_STATIC_MAX_REQUESTS * sizeof(unsigned long long);
@@ -612,7 +637,7 @@ extern "C" int pre_anticipate_static(int32_t n_instances, int32_t horizon, const
 
     int nc = 1, staged = 1;
     int64_t chunk = 4;
-    sort_geometry(n_requests, &nc, &chunk, &staged);   // nc <= 64 and staged, given the request limit
+    sort_geometry(n_requests, 3 * st->n_sm, PRE_STATIC_MAX_CHUNKS, &nc, &chunk, &staged);  // staged: chunk <= 4096
 
     int* status = d_flags ? d_flags : reinterpret_cast<int*>(st->base);
     unsigned int* chunk_off = reinterpret_cast<unsigned int*>(st->base + PRE_STATIC_STATUS_BYTES);

@@ -28,18 +28,43 @@ pre_step_requests(const int32_t* __restrict__ prompt, int32_t* __restrict__ gene
         __syncthreads();
     }
     bool any_bad = false;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += stride) {
-        const int32_t g = generated[r], D = predicted[r], inst = instance[r];
-        if (g < 0 || D < 1 || (uint32_t)inst >= (uint32_t)I) { any_bad = true; continue; }
-        if (g >= D) continue;  // tombstone
-        const int32_t P = prompt[r];
-        if (P < 0) { any_bad = true; continue; }
+    // one request: returns the new g (the old one when nothing changes)
+    auto tick = [&](int32_t P, int32_t g, int32_t D, int32_t inst) -> int32_t {
+        if (P < 0 || g < 0 || D < 1 || (uint32_t)inst >= (uint32_t)I) { any_bad = true; return g; }
+        if (g >= D) return g;  // tombstone
         const int32_t g1 = g + 1;
-        generated[r] = g1;
         if (use_sh) atomicAdd(&sh_active[inst], 1u); else atomicAdd(&active[inst], 1u);
-        if ((long long)D - g1 >= (long long)H)
+        if ((long long)D - g1 >= (long long)H)   // still running when step H-1 enters the window
             atomicAdd(&enter[inst], (unsigned long long)((long long)P + g1 + (H - 1)));
+        return g1;
+    };
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
+                       reinterpret_cast<uintptr_t>(predicted) | reinterpret_cast<uintptr_t>(instance)) & 15) == 0;
+    if (vec) {
+        const long long n4 = n >> 2;
+        for (long long q = gtid; q < n4; q += stride) {
+            const int4 p = __ldg(reinterpret_cast<const int4*>(prompt) + q);
+            int4 g = *(reinterpret_cast<const int4*>(generated) + q);
+            const int4 d = __ldg(reinterpret_cast<const int4*>(predicted) + q);
+            const int4 i = __ldg(reinterpret_cast<const int4*>(instance) + q);
+            const int4 o = g;
+            g.x = tick(p.x, g.x, d.x, i.x); g.y = tick(p.y, g.y, d.y, i.y);
+            g.z = tick(p.z, g.z, d.z, i.z); g.w = tick(p.w, g.w, d.w, i.w);
+            if (g.x != o.x || g.y != o.y || g.z != o.z || g.w != o.w) *(reinterpret_cast<int4*>(generated) + q) = g;
+        }
+        for (long long r = (n4 << 2) + gtid; r < n; r += stride) {
+            const int32_t g = generated[r];
+            const int32_t g1 = tick(prompt[r], g, predicted[r], instance[r]);
+            if (g1 != g) generated[r] = g1;
+        }
+    } else {
+        for (long long r = gtid; r < n; r += stride) {
+            const int32_t g = generated[r];
+            const int32_t g1 = tick(prompt[r], g, predicted[r], instance[r]);
+            if (g1 != g) generated[r] = g1;
+        }
     }
     if (use_sh) {
         __syncthreads();
