@@ -80,7 +80,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
     if (e == cudaSuccess) e = pre_anticipate_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
-    if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)8 * c->route_blocks);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)32 * c->route_blocks);
     if (e != cudaSuccess) {
         const bool oom = (e == cudaErrorMemoryAllocation);
         cudaGetLastError();

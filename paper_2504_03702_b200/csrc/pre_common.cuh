@@ -39,7 +39,7 @@ struct pre_ctx {
     unsigned int* d_bin_base;    // slow path [n_tiles+1]
     unsigned int* d_bin_cursor;  // slow path [n_tiles]   zero between calls
     unsigned long long* d_records;  // [max_requests]
-    unsigned long long* d_slots;    // [2][G][4] routing exchange
+    unsigned long long* d_slots;    // [2][G][16] routing exchange, one 128-byte line per block and parity
     unsigned long long* d_enter;    // [I] tokens entering the window at step H-1 (zero between calls)
     unsigned int* d_active;         // [I] live requests per instance (zero between calls)
 };
