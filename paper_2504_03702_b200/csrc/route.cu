@@ -341,6 +341,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
     __shared__ long long sh_fix;     // re-scored peak of the row that was just folded
+    __shared__ double sh_best_s[2];  // the block's best and second-best score for the arrival being scored
+    __shared__ int sh_best_i[2];     // ... and their rows
     constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
 
     const int G = gridDim.x, b = blockIdx.x;
@@ -351,10 +353,26 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     const int nrows = row1 - row0;
     const int cpr = (H + 63) >> 6;  // 64-cell chunks per row (one 16-byte load per lane)
     const bool full = (H & 63) == 0;
-    // chunk range of this warp (warps 1..) over the block's rows laid end to end
+    // Chunk range [c0, c1) of this warp (warps 1..) over the block's rows laid end to end.
+    // With few rows each row is cut into `parts` equal stretches and a warp takes exactly one
+    // (one reduction per warp and arrival); with many rows the chunks are dealt out evenly.
     const int nch = nrows * cpr;
-    const int c0 = warp ? (int)((long long)nch * (warp - 1) / SCAN_WARPS) : 0;
-    const int c1 = warp ? (int)((long long)nch * warp / SCAN_WARPS) : 0;
+    int c0 = 0, c1 = 0;
+    if (warp) {
+        int parts = nrows <= SCAN_WARPS ? SCAN_WARPS / nrows : 0;
+        if (parts > cpr) parts = cpr;
+        if (parts) {
+            const int unit = warp - 1;
+            if (unit < nrows * parts) {
+                const int row = unit / parts, part = unit - row * parts;
+                c0 = row * cpr + (int)((long long)cpr * part / parts);
+                c1 = row * cpr + (int)((long long)cpr * (part + 1) / parts);
+            }
+        } else {
+            c0 = (int)((long long)nch * (warp - 1) / SCAN_WARPS);
+            c1 = (int)((long long)nch * warp / SCAN_WARPS);
+        }
+    }
     const int first_row = c0 / cpr, first_q = c0 - first_row * cpr;
 
     for (int r = tid; r < nrows; r += ROUTE_THREADS) {
@@ -564,10 +582,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         const int buf = (int)(seq & 1);
         long long* bpk = pk + buf * a.max_rows;
 
-        // ---- 1. scan for arrival k (the pending arrival is not folded yet) | collect its winner
-        if (warp == 0) {
-            if (pending) gather(seq - 1);
-        } else {
+        // ---- 1. scan for arrival k (the pending arrival is not folded yet)
+        if (warp != 0) {
             int c = c0, row = first_row, q0 = first_q;
             while (c < c1) {
                 const int left = c1 - c;
@@ -610,50 +626,75 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 q0 = 0;
             }
         }
-        __syncthreads();  // S1: partial peaks of arrival k are in, winner of the pending arrival known
+        // ---- 2. Warp 0 collects the winner of the pending arrival while the scan runs.  When the
+        //         scan warps are done (named barrier 1 among warps 1..), warp 1 takes the block's two
+        //         best rows for arrival k.  Only the row that receives the pending arrival can still
+        //         change, so for every other block the best row found here is final.
+        if (warp == 0) {
+            if (pending) gather(seq - 1);
+        } else {
+            asm volatile("bar.sync 1, %0;" ::"n"(ROUTE_THREADS - 32) : "memory");
+            if (warp == 1) {
+                double b1s = CUDART_INF, b2s = CUDART_INF;
+                int b1i = 0x7fffffff, b2i = 0x7fffffff;
+                for (int r = lane; r < nrows; r += 32) {
+                    // the peak with the arrival added is an upper bound of the row as it stands
+                    if (!(rstate[r] & RS_WIDE)) bound[r] = bpk[r];
+                    const double s = score_of(sq[r], scd[r], bpk[r], P, D, a.theta, a.beta);
+                    const int i = row0 + r;
+                    if (better(s, i, b1s, b1i)) { b2s = b1s; b2i = b1i; b1s = s; b1i = i; }
+                    else if (better(s, i, b2s, b2i)) { b2s = s; b2i = i; }
+                }
+                #pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    const double o1s = __shfl_xor_sync(0xffffffffu, b1s, off), o2s = __shfl_xor_sync(0xffffffffu, b2s, off);
+                    const int o1i = __shfl_xor_sync(0xffffffffu, b1i, off), o2i = __shfl_xor_sync(0xffffffffu, b2i, off);
+                    if (better(o1s, o1i, b1s, b1i)) {
+                        // the other side's best wins: second = better(my best, its second)
+                        if (better(b1s, b1i, o2s, o2i)) { b2s = b1s; b2i = b1i; } else { b2s = o2s; b2i = o2i; }
+                        b1s = o1s; b1i = o1i;
+                    } else if (better(o1s, o1i, b2s, b2i)) { b2s = o1s; b2i = o1i; }
+                }
+                if (lane == 0) { sh_best_s[0] = b1s; sh_best_s[1] = b2s; sh_best_i[0] = b1i; sh_best_i[1] = b2i; }
+            } else {
+                for (int r = tid - 64; r < nrows; r += ROUTE_THREADS - 64) pk[(buf ^ 1) * a.max_rows + r] = I64_MIN;
+            }
+        }
+        __syncthreads();  // B: winner of the pending arrival known to the block
         if (sh_dead) break;
 
-        // ---- 2. fold the pending arrival, re-score its row for arrival k; reset the other buffer
-        for (int r = tid; r < nrows; r += ROUTE_THREADS) pk[(buf ^ 1) * a.max_rows + r] = I64_MIN;
+        // ---- 3. fold the pending arrival (owner only), publish the block's best row for arrival k
         const int w = sh_winner;
-        if (pending) settle(w, true, P, Dc);
-        __syncthreads();  // S2: fold visible to the block, sh_fix complete
-
-        // ---- 3. block minimum for arrival k, publish
+        const bool owner = pending && w >= row0 && w < row1;
+        if (pending) settle(w, true, P, Dc);   // for the owner: ends with the folded row's peak in sh_fix
         if (warp == 0) {
-            if (pending && w >= row0 && w < row1) {
-                if (lane == 0) { bpk[w - row0] = sh_fix; sh_fix = I64_MIN; }
+            double b1s = sh_best_s[0];
+            int b1i = sh_best_i[0];
+            if (owner) {
+                // the folded row's score changed: best = better(best of the other rows, folded row)
+                __syncwarp();   // lane 0 updated sq/scd of that row inside settle
+                const int r = w - row0;
+                const double s = score_of(sq[r], scd[r], sh_fix, P, D, a.theta, a.beta);
+                if (b1i == w) { b1s = sh_best_s[1]; b1i = sh_best_i[1]; }
+                if (better(s, w, b1s, b1i)) { b1s = s; b1i = w; }
                 __syncwarp();
-            }
-            double bs = CUDART_INF;
-            int bi = 0x7fffffff;
-            for (int r = lane; r < nrows; r += 32) {
-                // the peak with the arrival added is an upper bound of the row as it stands
-                if (!(rstate[r] & RS_WIDE)) bound[r] = bpk[r];
-                const double s = score_of(sq[r], scd[r], bpk[r], P, D, a.theta, a.beta);
-                if (better(s, row0 + r, bs, bi)) { bs = s; bi = row0 + r; }
-            }
-            #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const double os = __shfl_xor_sync(0xffffffffu, bs, off);
-                const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-                if (better(os, oi, bs, bi)) { bs = os; bi = oi; }
+                if (lane == 0) sh_fix = I64_MIN;
             }
             if (lane < 3) {
                 // three words, each carrying the exchange tag: valid on its own, no fence needed
                 const unsigned int tag = a.epoch + (unsigned int)seq;  // dense: one tag per exchange
                 unsigned long long* slot = a.slots + ((size_t)(tag & 1u) * G + b) * SLOT_WORDS;
-                const unsigned long long bits = (unsigned long long)__double_as_longlong(bs);
-                const unsigned int payload = lane == 0 ? (unsigned int)bi
+                const unsigned long long bits = (unsigned long long)__double_as_longlong(b1s);
+                const unsigned int payload = lane == 0 ? (unsigned int)b1i
                                            : lane == 1 ? (unsigned int)(bits >> 32) : (unsigned int)bits;
                 st_relaxed_u64(&slot[lane], ((unsigned long long)tag << 32) | payload);
             }
         }
+        if (owner) __syncthreads();  // C: nobody scans the folded row before the fold is complete
         pending = true; pP = P; pD = D; pidx = k;
         ++seq;
-        // No barrier here: the other warps go on to the next scan (which fills the other
-        // peak buffer) while warp 0 scores and publishes; sq/scd and sh_fix change only
-        // between S1 and S2 or inside warp 0.
+        // No barrier here for the other blocks: their warps go on to the next scan (which fills
+        // the other peak buffer) while warp 0 publishes.
     }
 
     // ---- the last arrival is still pending
