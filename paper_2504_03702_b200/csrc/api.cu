@@ -54,7 +54,6 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     std::memset(c, 0, sizeof(*c));
     c->cfg = *cfg;
     c->theta = cfg->t_mem * (double)cfg->capacity_tokens;
-    c->epoch = 1;
 
     cudaError_t e = cudaGetDevice(&c->device);
     cudaDeviceProp prop;
@@ -68,8 +67,13 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     c->n_tiles = (I + t - 1) / t;
     if (pre_tile_smem_bytes(t, H) > (size_t)prop.sharedMemPerBlockOptin) { delete c; return PRE_EINVAL; }
 
-    e = alloc_zero(&c->d_status, 2);
+    e = alloc_zero(&c->d_status, 4);
     c->d_abort = c->d_status ? c->d_status + 1 : nullptr;
+    c->d_epoch = c->d_status ? reinterpret_cast<unsigned int*>(c->d_status + 2) : nullptr;
+    if (e == cudaSuccess) {   // the slots start as zeros: the first tags must not be zero
+        const unsigned int first = 2;
+        e = cudaMemcpy(c->d_epoch, &first, sizeof(first), cudaMemcpyHostToDevice);
+    }
     if (e == cudaSuccess && pre_chunk_off_words(c->n_tiles))
         e = alloc_zero(&c->d_chunk_off, pre_chunk_off_words(c->n_tiles));
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);

@@ -29,11 +29,11 @@ struct pre_ctx {
     size_t route_smem;
     size_t route_resident_bytes;  // shared memory per routing block left for resident rows
     double theta;        // t_mem * M in binary64
-    uint32_t epoch;      // running arrival counter, tags the routing exchange slots
     int last_cuda_error;
     // device scratch
     int* d_status;            // status word
     int* d_abort;             // routing kernel gives up when set
+    unsigned int* d_epoch;    // running exchange counter of the routing kernel (tags of the exchange slots)
     unsigned int* d_chunk_off;   // [(n_tiles+1) x chunks] where each tile starts inside each sorted chunk
     unsigned int* d_bin_count;   // slow path [n_tiles]   zero between calls
     unsigned int* d_bin_base;    // slow path [n_tiles+1]
