@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     __shared__ double sh_score;
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
-    __shared__ long long sh_fix;     // re-scored peak of the row that was just folded
+    __shared__ long long sh_part[ROUTE_WARPS];  // per-warp peaks of the row that was just folded and re-scored
     __shared__ double sh_best_s[2];  // the block's best and second-best score for the arrival being scored
     __shared__ int sh_best_i[2];     // ... and their rows
     constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
@@ -385,7 +385,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         bound[r] = full ? 0 : I64_MAX;      // the survey raises it
         rstate[r] = full ? 0 : RS_WIDE;
     }
-    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; sh_fix = I64_MIN; }
+    if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; }
     __syncthreads();
     // Survey: which rows hold only values in [0, 2^32), and their maxima.  One pass over the
     // block's rows in global memory.
@@ -519,7 +519,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
 
     // The winner w of the pending arrival is known: the owner really adds it to row w
     // (Sec. 4.3.1 update), block 0 records it.  When `rescore` is set, the same pass takes the
-    // folded row's peak for the arrival being scored now (P, ramp length Dc) into sh_fix.
+    // folded row's peak for the arrival being scored now (P, ramp length Dc), one partial per warp in sh_part.
     auto settle = [&](int w, bool rescore, int P, int Dc) {
         if (w >= row0 && w < row1) {
             const int r = w - row0;
@@ -544,9 +544,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 }
                 pkv = max64(pkv, j < Dc ? c + ((long long)P + j) : c);
             }
-            if (rescore) {
+            if (rescore) {   // one partial per warp, reduced by warp 0 after the barrier (no contended atomics)
                 pkv = warp_max64(pkv);
-                if (lane == 0) atomicMax(&sh_fix, pkv);
+                if (lane == 0) sh_part[warp] = pkv;
             }
             __syncthreads();   // block-uniform branch; every thread has read rstate/bound above
             if (tid == 0) {
@@ -669,7 +669,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         // ---- 3. fold the pending arrival (owner only), publish the block's best row for arrival k
         const int w = sh_winner;
         const bool owner = pending && w >= row0 && w < row1;
-        if (pending) settle(w, true, P, Dc);   // for the owner: ends with the folded row's peak in sh_fix
+        if (pending) settle(w, true, P, Dc);   // for the owner: ends with the folded row's peak in sh_part
         if (warp == 0) {
             double b1s = sh_best_s[0];
             int b1i = sh_best_i[0];
@@ -677,11 +677,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 // the folded row's score changed: best = better(best of the other rows, folded row)
                 __syncwarp();   // lane 0 updated sq/scd of that row inside settle
                 const int r = w - row0;
-                const double s = score_of(sq[r], scd[r], sh_fix, P, D, a.theta, a.beta);
+                const long long fixed_peak = warp_max64(sh_part[lane]);
+                const double s = score_of(sq[r], scd[r], fixed_peak, P, D, a.theta, a.beta);
                 if (b1i == w) { b1s = sh_best_s[1]; b1i = sh_best_i[1]; }
                 if (better(s, w, b1s, b1i)) { b1s = s; b1i = w; }
-                __syncwarp();
-                if (lane == 0) sh_fix = I64_MIN;
             }
             if (lane == 0) {
                 const unsigned int tag = epoch + (unsigned int)seq;  // dense: one tag per exchange
