@@ -133,9 +133,11 @@ def run_reference(args, wl, rank):
 METRIC = "routes/sec over the whole step (anticipate + route batch + decode step)"
 
 # DRAM bytes (read + write) of one pre_route_persistent launch on the full batch of a
-# configuration, from an ncu capture (profiles/): the kernel reads the maps once and writes
-# only the folded cells and the appended requests.  None: not captured for the kernel as it stands.
-ROUTE_DRAM_TRAFFIC = {}
+# configuration.  From an ncu capture of a 256-arrival batch on the same maps
+# (profiles/ncu_dram_route_config3_256_arrivals.txt): 67.31 MB read (the maps, once per launch, whatever
+# the batch length) + 655 B written per arrival (folded cells, appended requests), the written part
+# scaled to 65,536 arrivals.  A configuration without a capture reports null.
+ROUTE_DRAM_TRAFFIC = {3: 67312384 + 655 * 65536}
 
 
 def config_dict(wl, args):
