@@ -124,7 +124,9 @@ def run_reference(args, wl, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "routes/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int64+f64", "data": "synthetic",
-        "config": config_dict(wl, args),
+        "config": dict(config_dict(wl, args), l2="not applicable (host run)",
+                       timing="time.perf_counter around the oracle calls; routing time scaled from the sample "
+                              "to the full batch"),
         "cpu_baseline": {"value": value, "unit": "routes/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "routes/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))

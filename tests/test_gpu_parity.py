@@ -342,3 +342,9 @@ def test_streaming_config_first_ticks():
 @pytest.mark.slow
 def test_streaming_config_with_a_burst():
     run_streaming(101)
+
+
+@pytest.mark.slow
+def test_streaming_config_all_ticks():
+    """The whole streaming configuration: 1,000 ticks, about 4.2 million routed arrivals."""
+    run_streaming(1000)
