@@ -310,7 +310,7 @@ __device__ __forceinline__ unsigned int scan_row_chunks_packed(const uint32_t* _
 
 // OR of the high words and maximum of the low words of chunks [q0, q1) of one global row.
 // A zero OR means every cell lies in [0, 2^32) and the maximum is the true maximum.
-__device__ __forceinline__ void survey_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int lane,
+__device__ __forceinline__ void inspect_row_chunks(const int64_t* __restrict__ row, int q0, int q1, int lane,
                                                   unsigned int* or_hi, unsigned int* max_lo) {
     unsigned int acc = 0, m = 0;
     const int64_t* p = row + lane * 2;
@@ -382,12 +382,12 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         sq[r] = a.queued_p[row0 + r];
         scd[r] = a.current_d[row0 + r];
         pk[r] = I64_MIN;                    // buffer 0, used by the first scan
-        bound[r] = full ? 0 : I64_MAX;      // the survey raises it
+        bound[r] = full ? 0 : I64_MAX;      // the inspection pass raises it
         rstate[r] = full ? 0 : RS_WIDE;
     }
     if (tid == 0) { sh_dead = 0; sh_n0 = *a.n_requests; }
     __syncthreads();
-    // Survey: which rows hold only values in [0, 2^32), and their maxima.  One pass over the
+    // Inspection: which rows hold only values in [0, 2^32), and their maxima.  One pass over the
     // block's rows in global memory.
     if (warp && full) {
         int c = c0, row = first_row, q0 = first_q;
@@ -395,7 +395,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             const int left = c1 - c;
             const int q1 = (cpr - q0) < left ? cpr : q0 + left;
             unsigned int or_hi, max_lo;
-            survey_row_chunks(a.curves + (size_t)(row0 + row) * H, q0, q1, lane, &or_hi, &max_lo);
+            inspect_row_chunks(a.curves + (size_t)(row0 + row) * H, q0, q1, lane, &or_hi, &max_lo);
             or_hi = __reduce_or_sync(0xffffffffu, or_hi);
             max_lo = __reduce_max_sync(0xffffffffu, max_lo);
             if (lane == 0) {
