@@ -33,6 +33,9 @@ def lib():
         _lib.orc_score_all.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_double,
                                        C.c_double, i64p, i64p, i64p, f64p, i64p]
         _lib.orc_score_all.restype = None
+        _lib.orc_scaler_signals.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_double,
+                                            C.c_double, i32p, i64p, i64p]
+        _lib.orc_scaler_signals.restype = None
         _lib.orc_step.argtypes = [i32p, i32p, i32p, i32p, C.c_int64, C.c_int32, C.c_int32, i64p, i64p, i64p]
         _lib.orc_step.restype = None
     return _lib
@@ -99,3 +102,13 @@ class State:
                        _p(self.predicted, C.c_int32), _p(self.instance, C.c_int32), int(self.n[0]),
                        self.I, self.H, _p(self.curves, C.c_int64), _p(self.queued_p, C.c_int64),
                        _p(self.current_d, C.c_int64))
+
+    def scaler_signals(self, overload_level=0.95, overload_share=0.10, idle_level=0.30):
+        """Returns (over_count int32[I], row_max int64[I], summary int64[3])."""
+        over = np.zeros(self.I, np.int32)
+        mx = np.zeros(self.I, np.int64)
+        summary = np.zeros(3, np.int64)
+        lib().orc_scaler_signals(_p(self.curves, C.c_int64), self.I, self.H, self.M, float(overload_level),
+                                 float(overload_share), float(idle_level), _p(over, C.c_int32),
+                                 _p(mx, C.c_int64), _p(summary, C.c_int64))
+        return over, mx, summary

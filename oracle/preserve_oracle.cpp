@@ -214,4 +214,40 @@ void orc_step(int32_t* P, int32_t* g, int32_t* D, int32_t* inst, int64_t n, int3
     }
 }
 
+// Signals for the proactive instance scaler (Sec. 4.3.2), read off the maps as they stand.
+//   over_count[i] = number of steps j in [0, H) whose anticipated KV usage exceeds
+//                   overload_level (95 %) of the capacity:  c_i[j] > overload_level * M;
+//   instance i is "potentially overloaded" when that happens in more than overload_share
+//   (10 %) of the steps:  over_count[i] > overload_share * H;
+//   row_max[i]    = max_j c_i[j]  (the paper's max(U') times M);
+//   an instance keeps the scale-down action from firing unless its usage stays below
+//   idle_level (T_f = 30 %) throughout the window:  row_max[i] < idle_level * M.
+// summary = { number of potentially overloaded instances,
+//             number of instances that are NOT below idle_level throughout,
+//             sum over instances of row_max }   (the number of instances to isolate is then
+//             N_c - summary[2] / (M * T_f), left to the caller).
+// Thresholds are binary64 products; token counts (< 2^53) convert exactly.
+void orc_scaler_signals(const int64_t* curves, int32_t I, int32_t H, int64_t M, double overload_level,
+                        double overload_share, double idle_level, int32_t* over_count, int64_t* row_max,
+                        int64_t* summary) {
+    const double hot = overload_level * (double)M;
+    const double many = overload_share * (double)H;
+    const double idle = idle_level * (double)M;
+    summary[0] = summary[1] = summary[2] = 0;
+    for (int32_t i = 0; i < I; ++i) {
+        const int64_t* c = curves + (size_t)i * H;
+        int32_t cnt = 0;
+        int64_t mx = INT64_MIN;
+        for (int32_t j = 0; j < H; ++j) {
+            if ((double)c[j] > hot) ++cnt;
+            if (c[j] > mx) mx = c[j];
+        }
+        over_count[i] = cnt;
+        row_max[i] = mx;
+        if ((double)cnt > many) summary[0] += 1;
+        if (!((double)mx < idle)) summary[1] += 1;
+        summary[2] += mx;
+    }
+}
+
 }  // extern "C"
