@@ -289,6 +289,19 @@ def main():
     B.check(st.status(), "end-to-end steps")
     routed_ok = int((host_choice >= 0).sum())
 
+    # scaler signals over the maps (Sec. 4.3.2): a separate, HBM-bound call, not part of the step
+    flush.zero_()
+    sc_ev = []
+    for _ in range(4):
+        flush.zero_()
+        e0, e1 = ev(), ev()
+        e0.record()
+        st.scaler_signals()
+        e1.record()
+        sc_ev.append((e0, e1))
+    torch.cuda.synchronize()
+    t_scaler = float(np.median([x.elapsed_time(y) for x, y in sc_ev[1:]]))
+
     if rank != 0:
         D.finish(group)
         return 0
@@ -323,6 +336,8 @@ def main():
                               "the whole launch from an ncu capture scaled to this batch"),
         "roofline_anticipate": dict(roof(b_build, t_build, 2), kernel="pre_chunk_sort + pre_tile_build"),
         "roofline_step": dict(roof(b_step, t_dstep, 2), kernel="pre_step_requests + pre_step_shift"),
+        "roofline_scaler_signals": dict(roof(8 * wl.n_instances * wl.horizon + 12 * wl.n_instances, t_scaler, 1),
+                                        kernel="pre_scaler_rows", note="separate call, not part of the step"),
         "e2e": {"value": world * a / (t_e2e * 1e-3), "unit": "routes/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e},
         "gpu_launches": 5 * args.steps,

@@ -146,6 +146,22 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
              int32_t* d_instance, const int64_t* d_n_requests, int64_t* d_curves,
              int64_t* d_queued_p, int64_t* d_current_d, void* stream);
 
+/* Signals for the proactive instance scaler (Sec. 4.3.2), read off the maps as they stand.
+ * "An instance is regarded as potentially overloaded if ... its KV memory usage exceeds 95 % in
+ * more than 10 % of those [next l] iterations"; the scale-down action needs every instance
+ * below T_f = 30 % throughout the window and isolates N_c - sum(max U')/T_f instances.
+ *     d_over_count[i] (int32) = #{ j in [0,H) : curves[i][j] > overload_level * M }
+ *     d_row_max[i]    (int64) = max_j curves[i][j]                      (= max(U') * M)
+ *     d_summary[0] = #{ i : over_count[i] > overload_share * H }        (potentially overloaded)
+ *     d_summary[1] = #{ i : not (row_max[i] < idle_level * M) }         (0: scale-down may fire)
+ *     d_summary[2] = sum_i row_max[i]          (isolate N_c - d_summary[2] / (M * idle_level))
+ * The three products are binary64; comparisons are made in binary64 (token counts below 2^53
+ * convert exactly).  The paper's values are 0.95, 0.10 and 0.30.  d_summary is int64[3], all
+ * pointers DEVICE, the maps are only read. */
+int pre_scaler_signals(pre_ctx* ctx, const int64_t* d_curves, double overload_level, double overload_share,
+                       double idle_level, int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary,
+                       void* stream);
+
 /* Synchronises `stream`, then returns and clears the device status: the most severe of
  * PRE_ETIMEOUT, PRE_ECAPACITY, PRE_EBADREQ recorded since the last call, PRE_ECUDA if the
  * stream reports a CUDA error, else PRE_OK. */

@@ -27,6 +27,8 @@ void release(pre_ctx* c) {
     cudaFree(c->d_slots);
     cudaFree(c->d_enter);
     cudaFree(c->d_active);
+    cudaFree(c->d_scaler_partial);
+    cudaFree(c->d_scaler_done);
     delete c;
 }
 
@@ -82,6 +84,8 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_records, (size_t)cfg->max_requests);
     if (e == cudaSuccess) e = alloc_zero(&c->d_enter, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_done, 1);
     if (e == cudaSuccess) e = pre_anticipate_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
     if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)32 * c->route_blocks);
@@ -146,6 +150,19 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
         return PRE_EINVAL;
     cudaError_t e = pre_launch_step(ctx, d_prompt, d_generated, d_predicted, d_instance, d_n_requests, d_curves,
                                     d_queued_p, d_current_d, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_scaler_signals(pre_ctx* ctx, const int64_t* d_curves, double overload_level, double overload_share,
+                       double idle_level, int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary,
+                       void* stream) {
+    if (!ctx || !d_curves || !d_over_count || !d_row_max || !d_summary) return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_over_count, 4) || !aligned(d_row_max, 8) || !aligned(d_summary, 8))
+        return PRE_EINVAL;
+    if (!std::isfinite(overload_level) || !std::isfinite(overload_share) || !std::isfinite(idle_level))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_scaler(ctx, d_curves, overload_level, overload_share, idle_level, d_over_count,
+                                      d_row_max, d_summary, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
 }
 

@@ -42,6 +42,8 @@ struct pre_ctx {
     unsigned long long* d_slots;    // [2][G][16] routing exchange, one 128-byte line per block and parity
     unsigned long long* d_enter;    // [I] tokens entering the window at step H-1 (zero between calls)
     unsigned int* d_active;         // [I] live requests per instance (zero between calls)
+    long long* d_scaler_partial;    // [8 * n_sm][3] block totals of the scaler-signal kernel
+    unsigned int* d_scaler_done;    // blocks of that kernel that have finished (zero between calls)
 };
 
 // Launchers (defined next to their kernels).  Each returns a cudaError_t.
@@ -55,6 +57,9 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
 cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
                             int32_t* instance, const int64_t* n_requests, int64_t* curves,
                             int64_t* queued_p, int64_t* current_d, cudaStream_t s);
+cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overload_level, double overload_share,
+                              double idle_level, int32_t* over_count, int64_t* row_max, int64_t* summary,
+                              cudaStream_t s);
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
 size_t pre_tile_smem_bytes(int tile_rows, int horizon);
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm);

@@ -65,6 +65,15 @@ class DeviceState:
         B.check(B.pre_step(self.ctx, self.prompt, self.generated, self.predicted, self.instance,
                            self.n_requests, self.curves, self.queued_p, self.current_d), "pre_step")
 
+    def scaler_signals(self, overload_level=0.95, overload_share=0.10, idle_level=0.30):
+        """Returns device tensors (over_count int32[I], row_max int64[I], summary int64[3])."""
+        over = torch.empty(self.I, dtype=torch.int32, device=self.device)
+        row_max = torch.empty(self.I, dtype=torch.int64, device=self.device)
+        summary = torch.empty(3, dtype=torch.int64, device=self.device)
+        B.check(B.pre_scaler_signals(self.ctx, self.curves, overload_level, overload_share, idle_level, over,
+                                     row_max, summary), "pre_scaler_signals")
+        return over, row_max, summary
+
     def status(self):
         return B.pre_status(self.ctx)
 

@@ -348,3 +348,40 @@ def test_streaming_config_with_a_burst():
 def test_streaming_config_all_ticks():
     """The whole streaming configuration: 1,000 ticks, about 4.2 million routed arrivals."""
     run_streaming(1000)
+
+
+# ------------------------------------------------------------------ scaler signals (Sec. 4.3.2)
+
+def check_scaler(st, ref, **kw):
+    over, row_max, summary = st.scaler_signals(**kw)
+    w_over, w_max, w_sum = ref.scaler_signals(**kw)
+    assert (over.cpu().numpy() == w_over).all()
+    assert (row_max.cpu().numpy() == w_max).all()
+    assert summary.cpu().numpy().tolist() == w_sum.tolist()
+    return w_sum
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_scaler_signals_configs(idx):
+    wl = W.make_config(idx)
+    st, ref = both(wl)
+    total = check_scaler(st, ref)
+    assert total[1] > 0                      # the configurations are busy: the scale-down action may not fire
+    check_scaler(st, ref, overload_level=0.7, overload_share=0.5, idle_level=0.9)
+    st.close()
+
+
+@pytest.mark.parametrize("seed,n_inst,h,n", [(81, 1, 1, 3), (82, 5, 63, 200), (83, 33, 130, 900), (84, 700, 8, 4000),
+                                             (85, 9, 4100, 500)])
+def test_scaler_signals_shapes(seed, n_inst, h, n):
+    wl = W.make_random(seed, n_inst, h, n, 0, max_prompt=300, max_output=2 * h + 3)
+    st, ref = both(wl)
+    cap = int(np.percentile(ref.curves.max(axis=1), 50)) + 1
+    for s in (st, ):
+        s.close()
+    wl.capacity_tokens = cap
+    st, ref = both(wl)
+    check_scaler(st, ref)
+    check_scaler(st, ref, overload_level=0.5, overload_share=0.0, idle_level=0.3)
+    assert B.pre_scaler_signals(st.ctx, st.curves, 0.95, 0.10, 0.30, None, st.current_d, st.current_d) == B.PRE_EINVAL
+    st.close()
