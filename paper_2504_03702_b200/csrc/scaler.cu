@@ -15,6 +15,8 @@ namespace {
 
 constexpr int SCALER_THREADS = 256;
 constexpr int SCALER_WARPS = SCALER_THREADS / 32;
+constexpr int SCALER_BATCH = 8;            // 16-byte loads a lane has in flight
+constexpr int SCALER_BLOCKS_PER_SM = 8;
 constexpr long long I64_MIN = (-9223372036854775807LL - 1);
 
 __device__ __forceinline__ long long warp_max64(long long v) {
@@ -41,12 +43,12 @@ pre_scaler_rows(const int64_t* __restrict__ curves, int I, int H, long long hot,
         long long mx = I64_MIN;
         if (vec) {
             int j = lane * 2;
-            for (; j + 7 * 64 < H; j += 8 * 64) {
-                longlong2 v[8];
+            for (; j + (SCALER_BATCH - 1) * 64 < H; j += SCALER_BATCH * 64) {
+                longlong2 v[SCALER_BATCH];
                 #pragma unroll
-                for (int u = 0; u < 8; ++u) v[u] = __ldcs(reinterpret_cast<const longlong2*>(rp + j + u * 64));
+                for (int u = 0; u < SCALER_BATCH; ++u) v[u] = __ldcs(reinterpret_cast<const longlong2*>(rp + j + u * 64));
                 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < SCALER_BATCH; ++u) {
                     cnt += (v[u].x > hot) + (v[u].y > hot);
                     mx = v[u].x > mx ? v[u].x : mx;
                     mx = v[u].y > mx ? v[u].y : mx;
@@ -118,7 +120,7 @@ cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overlo
     const double many = overload_share * (double)H;
     const double idle = idle_level * (double)ctx->cfg.capacity_tokens;
     int grid = (I + SCALER_WARPS - 1) / SCALER_WARPS;
-    const int cap = 8 * ctx->n_sm;   // 8 blocks of 8 warps fill an SM
+    const int cap = SCALER_BLOCKS_PER_SM * ctx->n_sm;
     if (grid > cap) grid = cap;
     pre_scaler_rows<<<grid, SCALER_THREADS, 0, s>>>(curves, I, H, hot, many, idle, over_count, row_max,
                                                     reinterpret_cast<long long*>(summary), ctx->d_scaler_partial,
