@@ -36,6 +36,8 @@ def lib():
         _lib.orc_scaler_signals.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_double,
                                             C.c_double, i32p, i64p, i64p]
         _lib.orc_scaler_signals.restype = None
+        _lib.orc_refine.argtypes = [i32p, i32p, i32p, i32p, i32p, C.c_int64, C.c_int32, C.c_int32, i64p, i64p, i64p]
+        _lib.orc_refine.restype = None
         _lib.orc_step.argtypes = [i32p, i32p, i32p, i32p, C.c_int64, C.c_int32, C.c_int32, i64p, i64p, i64p]
         _lib.orc_step.restype = None
     return _lib
@@ -102,6 +104,18 @@ class State:
                        _p(self.predicted, C.c_int32), _p(self.instance, C.c_int32), int(self.n[0]),
                        self.I, self.H, _p(self.curves, C.c_int64), _p(self.queued_p, C.c_int64),
                        _p(self.current_d, C.c_int64))
+
+    def refine(self, actual):
+        """Misprediction refinement against the real lengths `actual` (one per table row in use).
+        Returns counts int64[3] = (early finishes, extensions, malformed entries)."""
+        n = int(self.n[0])
+        act = _i32(actual)
+        assert len(act) >= n
+        counts = np.zeros(3, np.int64)
+        lib().orc_refine(_p(self.prompt, C.c_int32), _p(self.generated, C.c_int32), _p(self.predicted, C.c_int32),
+                         _p(self.instance, C.c_int32), _p(act, C.c_int32), n, self.I, self.H,
+                         _p(self.curves, C.c_int64), _p(self.current_d, C.c_int64), _p(counts, C.c_int64))
+        return counts
 
     def scaler_signals(self, overload_level=0.95, overload_share=0.10, idle_level=0.30):
         """Returns (over_count int32[I], row_max int64[I], summary int64[3])."""

@@ -24,7 +24,9 @@
 // Pins (tests/test_oracle_*.py): brute-force enumeration written separately in
 // the tests, the closed forms of a single ramp, the step/rebuild identity, the
 // fold/rebuild identity, greedy least-loaded routing as the beta = 0 special
-// case, exact rational evaluation of the score.  The capacity rule M and the
+// case, exact rational evaluation of the score; for the refinement a second
+// hand-computed example, the closed form of the removed tokens, the chain of
+// extensions and the equality with the definition on the refined table.  The capacity rule M and the
 // queued_p model are this build's readings, not the paper's: parity unpinned
 // for those two (they are inputs, the arithmetic on them is pinned).
 #include <cstdint>
@@ -247,6 +249,50 @@ void orc_scaler_signals(const int64_t* curves, int32_t I, int32_t H, int64_t M, 
         if ((double)cnt > many) summary[0] += 1;
         if (!((double)mx < idle)) summary[1] += 1;
         summary[2] += mx;
+    }
+}
+
+// Refinement of the maps when a request's real response length differs from the predicted
+// one (Sec. 4.3.1, the paragraph after the map update).  actual[r] is the real length as the
+// serving engine learns it; the call is made after the decode iteration of a tick.
+//   * finished early (g < D and the engine reports the request done, actual <= g): the tokens
+//     anticipated for the rest of the prediction are taken out again,
+//         U_i*M -= P + i   for i in [g, D)     (request steps; window step j = i - g),
+//     and the request is closed at its real length (D <- g).
+//   * still running at the predicted end (g == D and actual > g): the response is virtually
+//     extended by 0.2 times its length so far and the map updated for the extension,
+//         U_i*M += P + i   for i in [D, D + E),  E = ceil(D / 5)  (at least one token),
+//     D <- D + E.  Repeated on later ticks until the request completes; an extension that
+//     overshoots is taken out by the first rule.
+// Readings: the paper writes the extension as 0.2 times the ground-truth length, which is not
+// known while the request runs; the length reached so far (g = D at that moment) is used, as
+// the exact fraction D/5 rounded up.  The decode backlog follows the prediction: -(D - g) on
+// an early finish, +E on an extension.  Steps beyond the stored window are cut as in the build.
+// counts = { early finishes, extensions, malformed entries skipped }.
+void orc_refine(const int32_t* P, const int32_t* g, int32_t* D, const int32_t* inst, const int32_t* actual,
+                int64_t n, int32_t I, int32_t H, int64_t* curves, int64_t* current_d, int64_t* counts) {
+    counts[0] = counts[1] = counts[2] = 0;
+    for (int64_t r = 0; r < n; ++r) {
+        if (!well_formed(P[r], g[r], D[r], inst[r], I) || actual[r] < 1) { counts[2] += 1; continue; }
+        int64_t* c = curves + (size_t)inst[r] * H;
+        if (g[r] < D[r] && actual[r] <= g[r]) {
+            for (int64_t i = g[r]; i < D[r]; ++i) {
+                const int64_t j = i - g[r];
+                if (j < H) c[j] -= (int64_t)P[r] + i;
+            }
+            current_d[inst[r]] -= (int64_t)D[r] - g[r];
+            D[r] = g[r];
+            counts[0] += 1;
+        } else if (g[r] == D[r] && actual[r] > g[r]) {
+            const int64_t E = ((int64_t)D[r] + 4) / 5;
+            for (int64_t i = D[r]; i < (int64_t)D[r] + E; ++i) {
+                const int64_t j = i - g[r];
+                if (j < H) c[j] += (int64_t)P[r] + i;
+            }
+            current_d[inst[r]] += E;
+            D[r] = (int32_t)((int64_t)D[r] + E);
+            counts[1] += 1;
+        }
     }
 }
 
