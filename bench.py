@@ -302,6 +302,26 @@ def main():
     torch.cuda.synchronize()
     t_scaler = float(np.median([x.elapsed_time(y) for x, y in sc_ev[1:]]))
 
+    # misprediction refinement (Sec. 4.3.1): one pass over the table per tick against real lengths;
+    # separate call, timed on four further ticks of the state the steps left behind
+    table_actual, tick_actual = W.make_actual(wl, W.BASE_SEED + args.config)
+    actual = torch.zeros(wl.max_requests, dtype=torch.int32, device=device)
+    actual[:n0] = torch.from_numpy(table_actual).to(device)
+    actual[n0:n0 + a] = torch.from_numpy(tick_actual[0][:a]).to(device)
+    rf_ev, rf_counts = [], None
+    for _ in range(4):
+        st.step()
+        flush.zero_()
+        e0, e1 = ev(), ev()
+        e0.record()
+        rf_counts = st.refine(actual)
+        e1.record()
+        rf_ev.append((e0, e1))
+    torch.cuda.synchronize()
+    t_refine = float(np.median([x.elapsed_time(y) for x, y in rf_ev[1:]]))
+    rf_counts = [int(v) for v in rf_counts.cpu().tolist()]
+    B.check(st.status(), "refinement ticks")
+
     if rank != 0:
         D.finish(group)
         return 0
@@ -338,6 +358,10 @@ def main():
         "roofline_step": dict(roof(b_step, t_dstep, 2), kernel="pre_step_requests + pre_step_shift"),
         "roofline_scaler_signals": dict(roof(8 * wl.n_instances * wl.horizon + 12 * wl.n_instances, t_scaler, 1),
                                         kernel="pre_scaler_rows", note="separate call, not part of the step"),
+        "roofline_refine": dict(roof(20 * n_after, t_refine, 1), kernel="pre_refine_requests",
+                                events_last_tick={"early_finish": rf_counts[0], "extended": rf_counts[1]},
+                                note="separate call, not part of the step; bytes = five int32 columns of the "
+                                     "table, the read-modify-write of the touched map cells is not counted"),
         "e2e": {"value": world * a / (t_e2e * 1e-3), "unit": "routes/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e},
         "gpu_launches": 5 * args.steps,

@@ -146,10 +146,32 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
              int32_t* d_instance, const int64_t* d_n_requests, int64_t* d_curves,
              int64_t* d_queued_p, int64_t* d_current_d, void* stream);
 
+/* Refinement of the maps against real response lengths (Sec. 4.3.1, the paragraph after the
+ * map update).  d_actual[r] (DEVICE int32, >= 1) is the real response length of table row r as
+ * the serving engine learns it; call once per tick, after pre_step.  For every row r below
+ * *d_n_requests (DEVICE int64, only read):
+ *   finished early:  g < D and d_actual[r] <= g.  The tokens anticipated for the rest of the
+ *       prediction are taken out, curves[inst][j] -= P + g + j for j in [0, min(D-g, H)),
+ *       current_d[inst] -= D - g, and the row is closed at its real length, d_predicted[r] = g.
+ *   still running at the predicted end:  g == D and d_actual[r] > g.  The response is extended
+ *       by E = ceil(D / 5) tokens (0.2 times the length reached, at least one),
+ *       curves[inst][j] += P + g + j for j in [0, min(E, H)), current_d[inst] += E,
+ *       d_predicted[r] = D + E.  Repeats on later ticks until the request ends; an extension
+ *       that overshoots is taken out by the first rule.
+ *   otherwise nothing changes.  Afterwards pre_anticipate on the table reproduces d_curves.
+ * d_counts (DEVICE int64[3], may be NULL) receives {early finishes, extensions, malformed rows}.
+ * A malformed row (as for pre_anticipate, or d_actual[r] < 1, or D > 2^30) is skipped and
+ * PRE_EBADREQ reported by pre_status.  Asynchronous on `stream`; map cells are updated with
+ * integer reductions, so the result does not depend on the order of the rows. */
+int pre_refine(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated, int32_t* d_predicted,
+               const int32_t* d_instance, const int32_t* d_actual, const int64_t* d_n_requests,
+               int64_t* d_curves, int64_t* d_current_d, int64_t* d_counts, void* stream);
+
 /* Signals for the proactive instance scaler (Sec. 4.3.2), read off the maps as they stand.
- * "An instance is regarded as potentially overloaded if ... its KV memory usage exceeds 95 % in
- * more than 10 % of those [next l] iterations"; the scale-down action needs every instance
- * below T_f = 30 % throughout the window and isolates N_c - sum(max U')/T_f instances.
+ * The scaler treats an instance as potentially overloaded when its anticipated KV usage is
+ * above 95 % of the capacity on more than 10 % of the window's steps, and it may scale down only
+ * when every instance stays below T_f = 30 % over the whole window, the number of instances to
+ * isolate being N_c - sum(max U')/T_f.
  *     d_over_count[i] (int32) = #{ j in [0,H) : curves[i][j] > overload_level * M }
  *     d_row_max[i]    (int64) = max_j curves[i][j]                      (= max(U') * M)
  *     d_summary[0] = #{ i : over_count[i] > overload_share * H }        (potentially overloaded)

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "libpreserve_b200.so")
 PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENOMEM, PRE_ESIZE = 0, -1, -2, -3, -4, -5, -6, -7
 
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
-           "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals")
+           "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
+           "pre_refine")
 
 
 class pre_config(C.Structure):
@@ -36,6 +37,7 @@ def _load():
     lib.pre_anticipate_static.argtypes = [C.c_int32, C.c_int32, vp, vp, vp, vp, i64, vp, vp, vp, vp]
     lib.pre_route_batch.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.pre_refine.argtypes = [vp] * 11
     lib.pre_scaler_signals.argtypes = [vp, vp, C.c_double, C.c_double, C.c_double, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
     lib.pre_last_cuda_error.argtypes = [vp]
@@ -113,6 +115,13 @@ def pre_route_batch(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p
 def pre_step(ctx, prompt, generated, predicted, instance, n_requests, curves, queued_p, current_d, stream=None):
     return lib.pre_step(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(n_requests),
                         _ptr(curves), _ptr(queued_p), _ptr(current_d), _stream() if stream is None else stream)
+
+
+def pre_refine(ctx, prompt, generated, predicted, instance, actual, n_requests, curves, current_d, counts,
+               stream=None):
+    return lib.pre_refine(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(actual),
+                          _ptr(n_requests), _ptr(curves), _ptr(current_d), _ptr(counts),
+                          _stream() if stream is None else stream)
 
 
 def pre_scaler_signals(ctx, curves, overload_level, overload_share, idle_level, over_count, row_max, summary,

@@ -65,6 +65,14 @@ class DeviceState:
         B.check(B.pre_step(self.ctx, self.prompt, self.generated, self.predicted, self.instance,
                            self.n_requests, self.curves, self.queued_p, self.current_d), "pre_step")
 
+    def refine(self, actual, want_counts=True):
+        """`actual`: device int32 tensor of real response lengths, one per table row in use.
+        Returns the device tensor int64[3] (early finishes, extensions, malformed rows) or None."""
+        counts = torch.empty(3, dtype=torch.int64, device=self.device) if want_counts else None
+        B.check(B.pre_refine(self.ctx, self.prompt, self.generated, self.predicted, self.instance, actual,
+                             self.n_requests, self.curves, self.current_d, counts), "pre_refine")
+        return counts
+
     def scaler_signals(self, overload_level=0.95, overload_share=0.10, idle_level=0.30):
         """Returns device tensors (over_count int32[I], row_max int64[I], summary int64[3])."""
         over = torch.empty(self.I, dtype=torch.int32, device=self.device)

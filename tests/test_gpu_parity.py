@@ -385,3 +385,120 @@ def test_scaler_signals_shapes(seed, n_inst, h, n):
     check_scaler(st, ref, overload_level=0.5, overload_share=0.0, idle_level=0.3)
     assert B.pre_scaler_signals(st.ctx, st.curves, 0.95, 0.10, 0.30, None, st.current_d, st.current_d) == B.PRE_EINVAL
     st.close()
+
+
+# ------------------------------------------------------------------ misprediction refinement (Sec. 4.3.1)
+
+def refine_both(st, ref, actual_dev, actual_host, what=""):
+    got = st.refine(actual_dev)
+    want = ref.refine(actual_host)
+    assert got.cpu().numpy().tolist() == want.tolist(), f"event counts differ {what}"
+    return want
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_refine_configs_over_ticks(idx):
+    """Ticks of step + refinement on the one-shot configurations after their batch was routed."""
+    wl = W.make_config(idx)
+    table_actual, tick_actual = W.make_actual(wl, W.BASE_SEED + idx)
+    st, ref = both(wl)
+    ap, ad = wl.ticks[0]
+    st.route_batch(dev(ap), dev(ad), want_score=False)
+    ref.route_batch(ap, ad, fast=True, want_score=False)
+    actual = np.concatenate([table_actual, tick_actual[0]])
+    actual_dev = dev(actual)
+    events = np.zeros(3, np.int64)
+    for t in range(24):
+        st.step()
+        ref.step()
+        events += refine_both(st, ref, actual_dev, actual, f"tick {t}")
+        if t % 6 == 5:
+            assert_state_equal(st, ref, f"after tick {t}")
+    assert_state_equal(st, ref, "at the end")
+    assert events[0] > 0 and events[1] > 0 and events[2] == 0
+    # the maps still are what the build gives on the refined table
+    after = st.curves.clone()
+    st.anticipate()
+    assert (st.curves == after).all()
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+@pytest.mark.parametrize("seed,n_inst,h,n", [(91, 1, 1, 5), (92, 3, 7, 70), (93, 9, 40, 1000), (94, 130, 33, 5000),
+                                             (95, 2, 300, 64)])
+def test_refine_shapes_to_completion(seed, n_inst, h, n):
+    wl = W.make_random(seed, n_inst, h, n, 0, max_prompt=50, max_output=40)
+    err = np.rint((W.Stream(seed, 7).uniform(n) - 0.5) * 30).astype(np.int32)
+    actual = np.maximum(1, wl.predicted + err).astype(np.int32)        # some real ends already lie behind
+    actual_dev = dev(actual)
+    st, ref = both(wl)
+    refine_both(st, ref, actual_dev, actual, "before the first tick")
+    assert_state_equal(st, ref, "before the first tick")
+    for t in range(int(actual.max()) + 2):
+        st.step()
+        ref.step()
+        refine_both(st, ref, actual_dev, actual, f"tick {t}")
+    assert_state_equal(st, ref, "at the end")
+    assert not ref.curves.any()
+    assert (st.predicted[:n].cpu().numpy() == np.maximum(actual, wl.generated)).all()
+    st.close()
+
+
+def test_refine_many_events_on_one_row_and_beyond_the_window():
+    """Every request on one instance, all ending at once, ramps longer than the window."""
+    n, h = 3000, 16
+    prompt = np.full(n, 1000, np.int32)
+    predicted = (np.arange(n) % 200 + 50).astype(np.int32)
+    generated = np.full(n, 10, np.int32)
+    wl = W.make_random(5, 2, h, n, 0)
+    wl.prompt, wl.generated, wl.predicted = prompt, generated, predicted
+    wl.instance = np.zeros(n, np.int32)
+    st, ref = both(wl)
+    actual = np.full(n, 3, np.int32)
+    counts = refine_both(st, ref, dev(actual), actual)
+    assert counts.tolist() == [n, 0, 0]
+    assert_state_equal(st, ref)
+    assert not ref.curves.any()
+    st.close()
+
+
+def test_refine_malformed_rows_and_no_counts():
+    wl = W.make_random(6, 4, 12, 200, 0)
+    actual = np.maximum(1, wl.predicted - 3).astype(np.int32)
+    actual[5] = 0                                   # malformed: real length below 1
+    bad_inst = wl.instance.copy()
+    bad_inst[9] = 77                                # malformed row in the table
+    wl.instance = bad_inst
+    st, ref = both(wl)
+    assert st.status() == B.PRE_EBADREQ             # the build already reports row 9
+    for _ in range(6):
+        st.step()
+        ref.step()
+        assert st.refine(dev(actual), want_counts=False) is None
+        ref.refine(actual)
+    assert_state_equal(st, ref)
+    assert st.status() == B.PRE_EBADREQ
+    st.close()
+
+
+def test_refine_streaming_ticks():
+    """The streaming configuration with real lengths: step, refinement, then the tick's arrivals."""
+    wl = W.make_config(4, n_ticks=16)
+    table_actual, tick_actual = W.make_actual(wl, W.BASE_SEED + 4)
+    st, ref = both(wl)
+    actual = np.zeros(wl.max_requests, np.int32)
+    actual[: len(table_actual)] = table_actual
+    filled = len(table_actual)
+    actual_dev = dev(actual)
+    for t, (ap, ad) in enumerate(wl.ticks):
+        st.step()
+        ref.step()
+        refine_both(st, ref, actual_dev, actual, f"tick {t}")
+        c, _ = st.route_batch(dev(ap), dev(ad))
+        wc, _ = ref.route_batch(ap, ad, fast=True)
+        assert (c.cpu().numpy() == wc).all(), f"tick {t}"
+        actual[filled: filled + len(ap)] = tick_actual[t]
+        actual_dev[filled: filled + len(ap)] = dev(tick_actual[t])
+        filled += len(ap)
+    assert_state_equal(st, ref, "at the end of the stream")
+    st.close()
