@@ -36,6 +36,11 @@ def lib():
         _lib.orc_scaler_signals.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_double,
                                             C.c_double, i32p, i64p, i64p]
         _lib.orc_scaler_signals.restype = None
+        _lib.orc_route_admit.argtypes = [i32p, i32p, C.c_int64, C.c_int32, C.c_int32, C.c_int64, C.c_double, C.c_double,
+                                         C.c_double, C.c_double, i32p, i32p, i64p, C.c_int64, i32p,
+                                         i64p, i64p, i64p, i32p, i32p, i32p, i32p, i64p, C.c_int64, i32p, f64p,
+                                         C.c_int32]
+        _lib.orc_route_admit.restype = None
         _lib.orc_refine.argtypes = [i32p, i32p, i32p, i32p, i32p, C.c_int64, C.c_int32, C.c_int32, i64p, i64p, i64p]
         _lib.orc_refine.restype = None
         _lib.orc_step.argtypes = [i32p, i32p, i32p, i32p, C.c_int64, C.c_int32, C.c_int32, i64p, i64p, i64p]
@@ -90,6 +95,39 @@ class State:
            _p(self.instance, C.c_int32), _p(self.n, C.c_int64), self.max_requests,
            _p(choice, C.c_int32), _p(score, C.c_double) if want_score else None)
         return choice, score
+
+    def make_queue(self, capacity):
+        """Empty admission queue (ring) of the given capacity."""
+        self.queue_capacity = int(capacity)
+        self.queue_prompt = np.zeros(max(self.queue_capacity, 1), np.int32)
+        self.queue_predicted = np.zeros(max(self.queue_capacity, 1), np.int32)
+        self.queue_state = np.zeros(2, np.int64)       # head, length
+
+    def queue_items(self):
+        """Waiting requests, oldest first, as (prompt, predicted) arrays."""
+        head, n = (int(v) for v in self.queue_state)
+        idx = (head + np.arange(n)) % max(self.queue_capacity, 1)
+        return self.queue_prompt[idx].copy(), self.queue_predicted[idx].copy()
+
+    def route_admit(self, arr_prompt, arr_predicted, overload_level=0.95, overload_share=0.10, fast=False,
+                    want_score=True):
+        """Router with the admission queue. Returns (queue_choice, choice, score)."""
+        ap, ad = _i32(arr_prompt), _i32(arr_predicted)
+        a = len(ap)
+        waiting = int(self.queue_state[1])
+        qchoice = np.full(max(waiting, 1), -9, np.int32)
+        choice = np.full(max(a, 1), -9, np.int32)
+        score = np.zeros(max(a, 1), np.float64)
+        lib().orc_route_admit(_p(ap, C.c_int32), _p(ad, C.c_int32), a, self.I, self.H, self.M, self.t_mem,
+                              self.beta, float(overload_level), float(overload_share),
+                              _p(self.queue_prompt, C.c_int32), _p(self.queue_predicted, C.c_int32),
+                              _p(self.queue_state, C.c_int64), self.queue_capacity, _p(qchoice, C.c_int32),
+                              _p(self.curves, C.c_int64), _p(self.queued_p, C.c_int64), _p(self.current_d, C.c_int64),
+                              _p(self.prompt, C.c_int32), _p(self.generated, C.c_int32),
+                              _p(self.predicted, C.c_int32), _p(self.instance, C.c_int32), _p(self.n, C.c_int64),
+                              self.max_requests, _p(choice, C.c_int32), _p(score, C.c_double) if want_score else None,
+                              1 if fast else 0)
+        return qchoice[:waiting], choice[:a], score[:a]
 
     def score_all(self, p, d):
         score = np.zeros(self.I, np.float64)

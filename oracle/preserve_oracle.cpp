@@ -26,7 +26,9 @@
 // fold/rebuild identity, greedy least-loaded routing as the beta = 0 special
 // case, exact rational evaluation of the score; for the refinement a second
 // hand-computed example, the closed form of the removed tokens, the chain of
-// extensions and the equality with the definition on the refined table.  The capacity rule M and the
+// extensions and the equality with the definition on the refined table; for
+// the admission queue a hand-computed example, the plain router as the special
+// case that never blocks, and an exact-arithmetic restatement over several calls.  The capacity rule M and the
 // queued_p model are this build's readings, not the paper's: parity unpinned
 // for those two (they are inputs, the arithmetic on them is pinned).
 #include <cstdint>
@@ -294,6 +296,120 @@ void orc_refine(const int32_t* P, const int32_t* g, int32_t* D, const int32_t* i
             counts[1] += 1;
         }
     }
+}
+
+// Router with its admission queue (Sec. 4.3.3, the sentences before the score: an incoming
+// request waits when all instances are overloaded and is turned away when the queue is full).
+// The paper does not say when an instance counts as overloaded for the router; the scaler's
+// criterion of Sec. 4.3.2 is taken, evaluated on the maps as they stand, without the request:
+//   instance i is overloaded  <=>  #{ j in [0,H) : c_i[j] > overload_level * M } > overload_share * H.
+// One call handles, in this order, the requests already waiting (oldest first) and then the
+// new arrivals.  For each: if every instance is overloaded the request waits (a waiting one
+// keeps its place, a new one joins the tail while the queue has room, otherwise it is turned
+// away); if not, it is routed exactly as by orc_route_batch.  Maps only grow during a call, so
+// once every instance is overloaded it stays so until the call ends.
+// The queue is a ring: entry q (0 = oldest) is at (head + q) mod capacity, qstate = {head, length}.
+// Results: instance index, -1 malformed or request table full (dropped), -2 waits, -3 turned away;
+// for the entries that were waiting at entry in qchoice[q], for the arrivals in choice[k].
+// fast != 0 keeps running maxima and overload counts instead of rescanning (same decisions,
+// admitted by tests only after it equals the literal mode).
+void orc_route_admit(const int32_t* aP, const int32_t* aD, int64_t A, int32_t I, int32_t H, int64_t M,
+                     double t_mem, double beta, double overload_level, double overload_share,
+                     int32_t* qP, int32_t* qD, int64_t* qstate, int64_t qcap, int32_t* qchoice,
+                     int64_t* curves, int64_t* queued_p, int64_t* current_d, int32_t* P, int32_t* g,
+                     int32_t* D, int32_t* inst, int64_t* n_requests, int64_t max_requests,
+                     int32_t* choice, double* score, int32_t fast) {
+    const double theta = t_mem * (double)M;
+    const double hot = overload_level * (double)M;
+    const double many = overload_share * (double)H;
+    const int64_t head = qstate[0], len0 = qstate[1];
+    std::vector<int64_t> PM, SM;
+    std::vector<int32_t> over;
+    auto rebuild = [&](int32_t i) {
+        const int64_t* c = curves + (size_t)i * H;
+        int64_t* pm = PM.data() + (size_t)i * H;
+        int64_t* sm = SM.data() + (size_t)i * H;
+        int64_t m = INT64_MIN;
+        int32_t cnt = 0;
+        for (int32_t j = 0; j < H; ++j) {
+            int64_t v = c[j] + j; if (v > m) m = v; pm[j] = m;
+            if ((double)c[j] > hot) ++cnt;
+        }
+        m = INT64_MIN;
+        for (int32_t j = H - 1; j >= 0; --j) { if (c[j] > m) m = c[j]; sm[j] = m; }
+        over[i] = cnt;
+    };
+    if (fast) {
+        PM.resize((size_t)I * H); SM.resize((size_t)I * H); over.resize((size_t)I);
+        for (int32_t i = 0; i < I; ++i) rebuild(i);
+    }
+    auto all_overloaded = [&]() {
+        for (int32_t i = 0; i < I; ++i) {
+            int32_t cnt = 0;
+            if (fast) cnt = over[i];
+            else {
+                const int64_t* c = curves + (size_t)i * H;
+                for (int32_t j = 0; j < H; ++j) if ((double)c[j] > hot) ++cnt;
+            }
+            if (!((double)cnt > many)) return false;
+        }
+        return true;
+    };
+    bool blocked = false;
+    int64_t left = 0;       // waiting entries that stay
+    int64_t joined = 0;     // arrivals that joined the queue
+    for (int64_t k = 0; k < len0 + A; ++k) {
+        const bool waiting = k < len0;
+        const int32_t rP = waiting ? qP[(head + k) % qcap] : aP[k - len0];
+        const int32_t rD = waiting ? qD[(head + k) % qcap] : aD[k - len0];
+        int32_t* out = waiting ? &qchoice[k] : &choice[k - len0];
+        double* sc = (!waiting && score) ? &score[k - len0] : nullptr;
+        if (sc) *sc = 0.0;
+        if (blocked && waiting) { *out = -2; ++left; continue; }      // keeps its place, not looked at
+        if (rP < 0 || rD < 1) { *out = -1; continue; }                // malformed: dropped
+        if (!blocked) {
+            if (*n_requests >= max_requests) { *out = -1; continue; } // request table full: dropped
+            if (all_overloaded()) blocked = true;
+        }
+        if (blocked) {
+            if (waiting) { *out = -2; ++left; }
+            else if (left + joined < qcap) {
+                const int64_t pos = (head + len0 + joined) % qcap;    // behind the last waiting entry
+                qP[pos] = rP; qD[pos] = rD;
+                ++joined;
+                *out = -2;
+            } else {
+                *out = -3;
+            }
+            continue;
+        }
+        const int32_t Dc = rD < H ? rD : H;
+        int32_t best = -1;
+        double best_l = 0.0;
+        for (int32_t i = 0; i < I; ++i) {
+            int64_t peak;
+            if (fast) {
+                peak = (int64_t)rP + PM[(size_t)i * H + (Dc - 1)];
+                if (Dc < H && SM[(size_t)i * H + Dc] > peak) peak = SM[(size_t)i * H + Dc];
+            } else {
+                peak = peak_with(curves + (size_t)i * H, H, rP, rD);
+            }
+            double l = score_of(queued_p[i], current_d[i], peak, rP, rD, theta, beta);
+            if (best < 0 || l < best_l) { best = i; best_l = l; }
+        }
+        int64_t* c = curves + (size_t)best * H;
+        for (int32_t j = 0; j < Dc; ++j) c[j] += (int64_t)rP + j;
+        if (fast) rebuild(best);
+        queued_p[best] += rP;
+        current_d[best] += rD;
+        int64_t slot = (*n_requests)++;
+        P[slot] = rP; g[slot] = 0; D[slot] = rD; inst[slot] = best;
+        *out = best;
+        if (sc) *sc = best_l;
+    }
+    // entries that left are a prefix of the old queue
+    qstate[0] = qcap > 0 ? (head + (len0 - left)) % qcap : 0;
+    qstate[1] = left + joined;
 }
 
 }  // extern "C"

@@ -58,3 +58,41 @@ def load_worked_example(path):
         else:
             out[key] = vals
     return out
+
+
+def exact_admit(curves, queued_p, current_d, waiting, arrivals, capacity, queue_capacity, level, share,
+                t_mem=Fraction(4, 5), beta=Fraction(1)):
+    """Router with the admission queue in exact arithmetic: waiting requests (oldest first) then
+    arrivals; a request waits when every instance is overloaded (more than share*H steps above
+    level*capacity), joins the queue while there is room, is turned away otherwise.
+    Returns (results for the waiting ones, results for the arrivals, new queue, curves, queued_p, current_d)."""
+    c = np.array(curves, dtype=np.int64)
+    q = np.array(queued_p, dtype=np.int64)
+    cd = np.array(current_d, dtype=np.int64)
+    horizon = c.shape[1]
+
+    def everyone_overloaded():
+        for row in c:
+            steps = sum(1 for v in row if Fraction(int(v)) > Fraction(level) * capacity)
+            if not Fraction(steps) > Fraction(share) * horizon:
+                return False
+        return True
+
+    stay, joined, res_wait, res_arr = [], [], [], []
+    blocked = False
+    for k, (p, d) in enumerate(list(waiting) + list(arrivals)):
+        is_waiting = k < len(waiting)
+        out = res_wait if is_waiting else res_arr
+        if not blocked and everyone_overloaded():
+            blocked = True
+        if blocked:
+            if is_waiting:
+                stay.append((p, d)); out.append(-2)
+            elif len(stay) + len(joined) < queue_capacity:
+                joined.append((p, d)); out.append(-2)
+            else:
+                out.append(-3)
+            continue
+        ch, _, c, q, cd = exact_route(c, q, cd, [p], [d], capacity, t_mem, beta)
+        out.append(ch[0])
+    return res_wait, res_arr, stay + joined, c, q, cd
