@@ -289,6 +289,30 @@ def main():
     B.check(st.status(), "end-to-end steps")
     routed_ok = int((host_choice >= 0).sum())
 
+    # the same batch through the router with its admission queue (Sec. 4.3.3), the paper's overload
+    # levels; a separate call, not part of the step
+    reset()
+    B.check(B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, n0, st.curves,
+                             st.current_d), "pre_anticipate")
+    st.make_queue(4096)
+    e0, e1 = ev(), ev()
+    e0.record()
+    _, adm_choice, _ = st.route_admit(arr_p, arr_d, overload_level=0.95, overload_share=0.10)
+    e1.record()
+    torch.cuda.synchronize()
+    t_admit = e0.elapsed_time(e1)
+    adm = {"routed": int((adm_choice >= 0).sum()), "waiting": int((adm_choice == -2).sum()),
+           "turned_away": int((adm_choice == -3).sum())}
+    B.check(st.status(), "admission call")
+    # leave the state as the step leaves it (the calls below continue from there)
+    reset()
+    B.check(B.pre_anticipate(st.ctx, st.prompt, st.generated, st.predicted, st.instance, n0, st.curves,
+                             st.current_d), "pre_anticipate")
+    B.check(B.pre_route_batch(st.ctx, arr_p, arr_d, a, st.curves, st.queued_p, st.current_d, st.prompt,
+                              st.generated, st.predicted, st.instance, st.n_requests, choice, score),
+            "pre_route_batch")
+    st.step()
+
     # scaler signals over the maps (Sec. 4.3.2): a separate, HBM-bound call, not part of the step
     flush.zero_()
     sc_ev = []
@@ -358,6 +382,9 @@ def main():
         "roofline_step": dict(roof(b_step, t_dstep, 2), kernel="pre_step_requests + pre_step_shift"),
         "roofline_scaler_signals": dict(roof(8 * wl.n_instances * wl.horizon + 12 * wl.n_instances, t_scaler, 1),
                                         kernel="pre_scaler_rows", note="separate call, not part of the step"),
+        "route_admit": dict(adm, ms=t_admit, decided_per_s=a / (t_admit * 1e-3), kernel="pre_route_persistent<admit>",
+                            overload_level=0.95, overload_share=0.10, queue_capacity=4096,
+                            note="separate call, not part of the step; same batch, same maps"),
         "roofline_refine": dict(roof(20 * n_after, t_refine, 1), kernel="pre_refine_requests",
                                 events_last_tick={"early_finish": rf_counts[0], "extended": rf_counts[1]},
                                 note="separate call, not part of the step; bytes = five int32 columns of the "

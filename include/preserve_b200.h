@@ -146,6 +146,38 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
              int32_t* d_instance, const int64_t* d_n_requests, int64_t* d_curves,
              int64_t* d_queued_p, int64_t* d_current_d, void* stream);
 
+/* Values of d_choice / d_queue_choice below zero. */
+#define PRE_CHOICE_DROPPED     (-1)  /* malformed request, or the request table is full */
+#define PRE_CHOICE_WAITS       (-2)  /* every instance overloaded: the request is in the queue */
+#define PRE_CHOICE_TURNED_AWAY (-3)  /* every instance overloaded and the queue is full */
+
+/* Router with its admission queue (Sec. 4.3.3: an incoming request is held back while all
+ * instances are overloaded and is turned away once the queue is full).  The paper does not
+ * define "overloaded" for the router; the scaler's criterion of Sec. 4.3.2 is used, on the maps
+ * as they stand, without the request:
+ *     instance i is overloaded  <=>  #{ j in [0,H) : curves[i][j] > overload_level * M } > overload_share * H
+ * (binary64 products; the paper's values are 0.95 and 0.10).
+ * One call decides, in this order, the requests that were waiting at entry (oldest first) and
+ * then the n_arrivals new ones.  While some instance is not overloaded a request is routed
+ * exactly as by pre_route_batch (score, argmin, update of the winner, append to the table).
+ * The first request that finds every instance overloaded is not routed, and neither is any
+ * request after it (maps only grow during a call): a waiting request keeps its place, an
+ * arrival joins the tail of the queue while it has room and is turned away otherwise.
+ * The queue is a ring owned by the caller, all DEVICE memory: d_queue_prompt/d_queue_predicted
+ * (int32[queue_capacity]), d_queue_state (int64[2] = {head, length}; entry q, 0 = oldest, is at
+ * (head + q) mod queue_capacity; start with {0, 0}).  queue_capacity may be 0 (nobody waits).
+ * Results: d_queue_choice[q] (int32[queue_capacity], written for the entries waiting at entry) and
+ * d_choice[k] for the arrivals receive the instance index or one of the PRE_CHOICE_* values;
+ * d_score[k] (may be NULL) the winning L of a routed arrival, 0 otherwise.  Entries that leave
+ * the queue are a prefix of it.  Other arguments, errors and the status word as for
+ * pre_route_batch; n_arrivals and queue_capacity below 2^30. */
+int pre_route_admit(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted, int64_t n_arrivals,
+                    double overload_level, double overload_share, int32_t* d_queue_prompt,
+                    int32_t* d_queue_predicted, int64_t* d_queue_state, int64_t queue_capacity,
+                    int32_t* d_queue_choice, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
+                    int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                    int64_t* d_n_requests, int32_t* d_choice, double* d_score, void* stream);
+
 /* Refinement of the maps against real response lengths (Sec. 4.3.1, the paragraph after the
  * map update).  d_actual[r] (DEVICE int32, >= 1) is the real response length of table row r as
  * the serving engine learns it; call once per tick, after pre_step.  For every row r below

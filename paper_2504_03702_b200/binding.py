@@ -16,7 +16,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
-           "pre_refine")
+           "pre_refine", "pre_route_admit")
 
 
 class pre_config(C.Structure):
@@ -38,6 +38,7 @@ def _load():
     lib.pre_route_batch.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_refine.argtypes = [vp] * 11
+    lib.pre_route_admit.argtypes = [vp, vp, vp, i64, C.c_double, C.c_double, vp, vp, vp, i64] + [vp] * 12
     lib.pre_scaler_signals.argtypes = [vp, vp, C.c_double, C.c_double, C.c_double, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
     lib.pre_last_cuda_error.argtypes = [vp]
@@ -110,6 +111,16 @@ def pre_route_batch(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p
                                _ptr(queued_p), _ptr(current_d), _ptr(prompt), _ptr(generated), _ptr(predicted),
                                _ptr(instance), _ptr(n_requests), _ptr(choice), _ptr(score),
                                _stream() if stream is None else stream)
+
+
+def pre_route_admit(ctx, arr_prompt, arr_predicted, n_arrivals, overload_level, overload_share, queue_prompt,
+                    queue_predicted, queue_state, queue_capacity, queue_choice, curves, queued_p, current_d, prompt,
+                    generated, predicted, instance, n_requests, choice, score, stream=None):
+    return lib.pre_route_admit(ctx, _ptr(arr_prompt), _ptr(arr_predicted), int(n_arrivals), float(overload_level),
+                               float(overload_share), _ptr(queue_prompt), _ptr(queue_predicted), _ptr(queue_state),
+                               int(queue_capacity), _ptr(queue_choice), _ptr(curves), _ptr(queued_p),
+                               _ptr(current_d), _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance),
+                               _ptr(n_requests), _ptr(choice), _ptr(score), _stream() if stream is None else stream)
 
 
 def pre_step(ctx, prompt, generated, predicted, instance, n_requests, curves, queued_p, current_d, stream=None):

@@ -29,6 +29,7 @@ void release(pre_ctx* c) {
     cudaFree(c->d_active);
     cudaFree(c->d_scaler_partial);
     cudaFree(c->d_scaler_done);
+    cudaFree(c->d_queue_entry);
     delete c;
 }
 
@@ -86,6 +87,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_done, 1);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_queue_entry, 2);
     if (e == cudaSuccess) e = pre_anticipate_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
     if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)32 * c->route_blocks);
@@ -136,6 +138,34 @@ int pre_route_batch(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_
     cudaError_t e = pre_launch_route(ctx, d_arr_prompt, d_arr_predicted, n_arrivals, d_curves, d_queued_p,
                                      d_current_d, d_prompt, d_generated, d_predicted, d_instance, d_n_requests,
                                      d_choice, d_score, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_route_admit(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted, int64_t n_arrivals,
+                    double overload_level, double overload_share, int32_t* d_queue_prompt,
+                    int32_t* d_queue_predicted, int64_t* d_queue_state, int64_t queue_capacity,
+                    int32_t* d_queue_choice, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
+                    int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                    int64_t* d_n_requests, int32_t* d_choice, double* d_score, void* stream) {
+    if (!ctx || n_arrivals < 0 || n_arrivals >= (1LL << 30)) return PRE_EINVAL;
+    if (queue_capacity < 0 || queue_capacity >= (1LL << 30) || !d_queue_state) return PRE_EINVAL;
+    if (queue_capacity > 0 && (!d_queue_prompt || !d_queue_predicted || !d_queue_choice)) return PRE_EINVAL;
+    if (!std::isfinite(overload_level) || !std::isfinite(overload_share)) return PRE_EINVAL;
+    if (!d_curves || !d_queued_p || !d_current_d || !d_prompt || !d_generated || !d_predicted || !d_instance ||
+        !d_n_requests)
+        return PRE_EINVAL;
+    if (n_arrivals > 0 && (!d_arr_prompt || !d_arr_predicted || !d_choice)) return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_queued_p, 8) || !aligned(d_current_d, 8) || !aligned(d_n_requests, 8) ||
+        !aligned(d_score, 8) || !aligned(d_choice, 4) || !aligned(d_arr_prompt, 4) || !aligned(d_arr_predicted, 4) ||
+        !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) || !aligned(d_instance, 4) ||
+        !aligned(d_queue_prompt, 4) || !aligned(d_queue_predicted, 4) || !aligned(d_queue_choice, 4) ||
+        !aligned(d_queue_state, 8))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_route_admit(ctx, d_arr_prompt, d_arr_predicted, n_arrivals, overload_level,
+                                           overload_share, d_queue_prompt, d_queue_predicted, d_queue_state,
+                                           queue_capacity, d_queue_choice, d_curves, d_queued_p, d_current_d, d_prompt,
+                                           d_generated, d_predicted, d_instance, d_n_requests, d_choice, d_score,
+                                           static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
 }
 

@@ -28,12 +28,15 @@ struct pre_ctx {
     int route_threads;
     size_t route_smem;
     size_t route_resident_bytes;  // shared memory per routing block left for resident rows
+    size_t route_smem_admit;            // the same two for the kernel with the admission queue
+    size_t route_resident_bytes_admit;
     double theta;        // t_mem * M in binary64
     int last_cuda_error;
     // device scratch
     int* d_status;            // status word
     int* d_abort;             // routing kernel gives up when set
     unsigned int* d_epoch;    // running exchange counter of the routing kernel (tags of the exchange slots)
+    int64_t* d_queue_entry;   // {head, length} of the admission queue as they were when the call was made
     unsigned int* d_chunk_off;   // [(n_tiles+1) x chunks] where each tile starts inside each sorted chunk
     unsigned int* d_bin_count;   // slow path [n_tiles]   zero between calls
     unsigned int* d_bin_base;    // slow path [n_tiles+1]
@@ -54,6 +57,13 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
                              int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
                              int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
                              int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s);
+cudaError_t pre_launch_route_admit(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                   int64_t n_arrivals, double overload_level, double overload_share,
+                                   int32_t* queue_prompt, int32_t* queue_predicted, int64_t* queue_state,
+                                   int64_t queue_capacity, int32_t* queue_choice, int64_t* curves,
+                                   int64_t* queued_p, int64_t* current_d, int32_t* prompt, int32_t* generated,
+                                   int32_t* predicted, int32_t* instance, int64_t* n_requests, int32_t* choice,
+                                   double* score, cudaStream_t s);
 cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
                             int32_t* instance, const int64_t* n_requests, int64_t* curves,
                             int64_t* queued_p, int64_t* current_d, cudaStream_t s);

@@ -29,6 +29,8 @@
 
 #include <math_constants.h>
 
+#include <cmath>
+
 namespace {
 
 constexpr int ROUTE_THREADS = 1024;
@@ -130,7 +132,18 @@ struct RouteArgs {
     int* abort_flag;
     int max_rows;       // ceil(I / G)
     size_t resident_bytes;  // shared memory per block left for resident rows
+    // admission queue (ADMIT kernels only): a ring of waiting requests, entry q at (head + q) mod capacity
+    int32_t* queue_prompt;
+    int32_t* queue_predicted;
+    int64_t* queue_state;          // {head, length}, rewritten by block 0 at the end
+    const int64_t* queue_entry;    // the same two words as they were when the call was made
+    long long queue_capacity;
+    int32_t* queue_choice;         // results for the entries that were waiting at entry
+    long long hot;                 // floor(overload_level * M): a cell counts when it is above
+    double many;                   // overload_share * H: overloaded when more cells than this count
 };
+
+constexpr int CHOICE_DROPPED = -1, CHOICE_WAITS = -2, CHOICE_TURNED_AWAY = -3;
 
 // Peak over 64-cell chunks [q0, q1) of one row with the arrival (P, Dc) virtually added
 // (chunk q covers steps 64q .. 64q+63, two per lane); the result is per lane.
@@ -323,6 +336,11 @@ __device__ __forceinline__ void inspect_row_chunks(const int64_t* __restrict__ r
     *max_lo = m;
 }
 
+// ADMIT adds the admission queue of Sec. 4.3.3: every block keeps, for its rows, the number of
+// steps above the overload level (the scaler's criterion of Sec. 4.3.2) and publishes with its
+// best row whether all its rows are overloaded; when all blocks say so the request that was
+// being decided is not routed and the batch stops there: what is left waits or is turned away.
+template <bool ADMIT>
 __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const RouteArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     long long* pk = reinterpret_cast<long long*>(smem_raw);  // [2][max_rows] peaks, by exchange parity
@@ -337,7 +355,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     // rstate[r]: RS_RESIDENT while the row's shared-memory copy is in use, RS_WIDE once the row
     // is known to need 64 bits
     int* rstate = order + a.max_rows;
-    unsigned char* res = reinterpret_cast<unsigned char*>(rstate + a.max_rows);  // 48*max_rows bytes in: 16-byte aligned
+    // over[r] (ADMIT): steps of row r above the overload level; 64 bytes of fixed words per row then, else 48
+    int* over = rstate + a.max_rows;
+    unsigned char* res = reinterpret_cast<unsigned char*>(rstate + (ADMIT ? 5 : 1) * a.max_rows);  // 16-byte aligned
     __shared__ int sh_winner;
     __shared__ double sh_score;
     __shared__ int sh_dead;
@@ -345,6 +365,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     __shared__ long long sh_part[ROUTE_WARPS];  // per-warp peaks of the row that was just folded and re-scored
     __shared__ double sh_best_s[2];  // the block's best and second-best score for the arrival being scored
     __shared__ int sh_best_i[2];     // ... and their rows
+    __shared__ int sh_cnt[ROUTE_WARPS];   // ADMIT: per-warp change of the folded row's overload count
+    __shared__ int sh_n_over;             // ADMIT: rows of this block that are overloaded
+    __shared__ int sh_all_over;           // ADMIT: every block reported all its rows overloaded
     constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
 
     const int G = gridDim.x, b = blockIdx.x;
@@ -445,12 +468,55 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         }
     }
     __syncthreads();
+    if (ADMIT) {   // overload counts of the owned rows, one warp per row and trip
+        for (int r = warp; r < nrows; r += ROUTE_WARPS) {
+            const int64_t* gp = a.curves + (size_t)(row0 + r) * H;
+            int cnt = 0;
+            for (int j = lane; j < H; j += 32) cnt += __ldcg(gp + j) > a.hot;
+            cnt = __reduce_add_sync(0xffffffffu, cnt);
+            if (lane == 0) over[r] = cnt;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int n = 0;
+            for (int r = 0; r < nrows; ++r) n += (double)over[r] > a.many;
+            sh_n_over = n;
+            sh_all_over = 0;
+        }
+        __syncthreads();
+    }
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
     if (room < 0) room = 0;
+    // ADMIT: the requests that were waiting when the call was made come first, then the arrivals
+    long long q_head = 0, q_len = 0;
+    if (ADMIT && a.queue_capacity > 0) {   // kept inside the ring whatever the two words hold
+        q_head = a.queue_entry[0];
+        q_len = a.queue_entry[1];
+        if (q_head < 0 || q_head >= a.queue_capacity) q_head = 0;
+        if (q_len < 0) q_len = 0;
+        if (q_len > a.queue_capacity) q_len = a.queue_capacity;
+    }
+    const long long n_items = q_len + a.n_arrivals;
+    auto item_prompt = [&](long long k) {
+        return (ADMIT && k < q_len) ? a.queue_prompt[(q_head + k) % a.queue_capacity] : a.arr_prompt[k - q_len];
+    };
+    auto item_predicted = [&](long long k) {
+        return (ADMIT && k < q_len) ? a.queue_predicted[(q_head + k) % a.queue_capacity] : a.arr_predicted[k - q_len];
+    };
+    // where the result of item k goes (block 0, one thread)
+    auto put_result = [&](long long k, int c, double sc) {
+        if (ADMIT && k < q_len) a.queue_choice[k] = c;
+        else {
+            a.choice[k - q_len] = c;
+            if (a.score) a.score[k - q_len] = sc;
+        }
+    };
+    bool blocked = false;         // ADMIT: the pending request found every instance overloaded
     // Identical in every thread of every block: all take the same decisions.
     long long seq = 0;            // exchanges started so far (= requests appended or pending)
     bool saw_bad = false, saw_full = false;
+    long long first_bad = I64_MAX, first_full = I64_MAX;   // the first items dropped as malformed / for a full table
     bool pending = false;         // an arrival has been published but not yet folded
     int pP = 0, pD = 0;           // ... its prompt and predicted lengths
     long long pidx = 0;           // ... its index in the batch
@@ -467,6 +533,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         const unsigned long long tag16 = (unsigned long long)(tag & 0xffffu);
         const unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * SLOT_WORDS;
         bool lost = false;
+        bool all_over = true;
         double bs = CUDART_INF;
         int bi = 0x7fffffff;
         for (int base = 0; base < G && !lost; base += 32 * GATHER_ILP) {
@@ -495,7 +562,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 if (cta < G) {
                     const unsigned long long bits = (w[i][0] << 16) | ((w[i][1] >> 32) & 0xffffull);
                     const double sc = __longlong_as_double((long long)bits);
-                    const int idx = (int)(unsigned int)(w[i][1] & 0xffffffffu);
+                    const int idx = (int)(unsigned int)(w[i][1] & (ADMIT ? 0x7fffffffu : 0xffffffffu));
+                    if (ADMIT) all_over &= ((w[i][1] >> 31) & 1ull) != 0;   // bit 31 of the row word
                     if (better(sc, idx, bs, bi)) { bs = sc; bi = idx; }
                 }
             }
@@ -515,6 +583,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             sh_winner = bi;
             sh_score = bs;
         }
+        if (ADMIT) {
+            all_over = __all_sync(0xffffffffu, all_over) && !lost;
+            if (lane == 0) sh_all_over = all_over;
+        }
     };
 
     // The winner w of the pending arrival is known: the owner really adds it to row w
@@ -532,10 +604,13 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             uint32_t* sp32 = reinterpret_cast<uint32_t*>(res) + (size_t)r * H;
             int64_t* sp64 = reinterpret_cast<int64_t*>(res) + (size_t)r * H;
             long long pkv = I64_MIN;
+            int crossed = 0;   // ADMIT: cells the fold takes above the overload level
             for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
                 long long c = !in_smem ? __ldcg(gp + j) : packed ? (long long)sp32[j] : sp64[j];
                 if (j < pDc) {
+                    if (ADMIT) crossed -= c > a.hot;
                     c += (long long)pP + j;
+                    if (ADMIT) crossed += c > a.hot;
                     gp[j] = c;
                     if (in_smem) {
                         if (!packed) sp64[j] = c;
@@ -548,8 +623,19 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 pkv = warp_max64(pkv);
                 if (lane == 0) sh_part[warp] = pkv;
             }
+            if (ADMIT) {
+                crossed = __reduce_add_sync(0xffffffffu, crossed);
+                if (lane == 0) sh_cnt[warp] = crossed;
+            }
             __syncthreads();   // block-uniform branch; every thread has read rstate/bound above
             if (tid == 0) {
+                if (ADMIT) {
+                    int d = 0;
+                    for (int x = 0; x < ROUTE_WARPS; ++x) d += sh_cnt[x];
+                    const bool was = (double)over[r] > a.many;
+                    over[r] += d;
+                    if (!was && (double)over[r] > a.many) sh_n_over += 1;
+                }
                 if (evict) rstate[r] = st & ~RS_RESIDENT;
                 if (bound[r] != I64_MAX) bound[r] += (long long)pP + pDc;  // the ramp adds less than this
                 sq[r] += pP;
@@ -564,21 +650,22 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             a.generated[slot] = 0;
             a.predicted[slot] = pD;
             a.instance[slot] = w;
-            a.choice[pidx] = w;
-            if (a.score) a.score[pidx] = sh_score;
+            put_result(pidx, w, sh_score);
         }
     };
 
-    for (long long k = 0; k < a.n_arrivals; ++k) {
-        const int P = a.arr_prompt[k], D = a.arr_predicted[k];
+    for (long long k = 0; k < n_items; ++k) {
+        const int P = item_prompt(k), D = item_predicted(k);
         if (P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX) {
             saw_bad = true;
-            if (b == 0 && tid == 0) { a.choice[k] = -1; if (a.score) a.score[k] = 0.0; }
+            if (ADMIT && k < first_bad) first_bad = k;
+            if (b == 0 && tid == 0) put_result(k, CHOICE_DROPPED, 0.0);
             continue;
         }
         if (seq >= room) {
             saw_full = true;
-            if (b == 0 && tid == 0) { a.choice[k] = -1; if (a.score) a.score[k] = 0.0; }
+            if (ADMIT && k < first_full) first_full = k;
+            if (b == 0 && tid == 0) put_result(k, CHOICE_DROPPED, 0.0);
             continue;
         }
         const int Dc = D < H ? D : H;
@@ -665,6 +752,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         }
         __syncthreads();  // B: winner of the pending arrival known to the block
         if (sh_dead) break;
+        if (ADMIT && pending && sh_all_over) { blocked = true; break; }   // the pending request is not routed
 
         // ---- 3. fold the pending arrival (owner only), publish the block's best row for arrival k
         const int w = sh_winner;
@@ -687,7 +775,10 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 const unsigned long long tag16 = (unsigned long long)(tag & 0xffffu) << 48;
                 unsigned long long* slot = a.slots + ((size_t)(tag & 1u) * G + b) * SLOT_WORDS;
                 const unsigned long long bits = (unsigned long long)__double_as_longlong(b1s);
-                st_relaxed_v2(slot, tag16 | (bits >> 16), tag16 | ((bits & 0xffffull) << 32) | (unsigned int)b1i);
+                // ADMIT: bit 31 of the row word says that every row of this block is overloaded (lane 0 is the
+                // thread that keeps sh_n_over, so it sees its own latest update)
+                const unsigned int flag = (ADMIT && sh_n_over == nrows) ? 0x80000000u : 0u;
+                st_relaxed_v2(slot, tag16 | (bits >> 16), tag16 | ((bits & 0xffffull) << 32) | flag | (unsigned int)b1i);
             }
         }
         if (owner) __syncthreads();  // C: nobody scans the folded row before the fold is complete
@@ -698,65 +789,136 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     }
 
     // ---- the last arrival is still pending
-    if (pending && !sh_dead) {
+    if (pending && !sh_dead && !blocked) {
         __syncthreads();
         if (warp == 0) gather(seq - 1);
         __syncthreads();
-        if (!sh_dead) settle(sh_winner, false, 0, 0);
+        if (ADMIT && !sh_dead && sh_all_over) blocked = true;
+        if (!sh_dead && !blocked) settle(sh_winner, false, 0, 0);
     }
 
     if (b == 0 && tid == 0) {
-        // after a lost wait the pending arrival was never settled
-        *a.n_requests = n0 + (sh_dead && pending ? seq - 1 : seq);
+        // after a lost wait, or when it found every instance overloaded, the pending request was never settled
+        *a.n_requests = n0 + ((sh_dead || blocked) && pending ? seq - 1 : seq);
         *a.epoch_ptr = epoch + (unsigned int)seq;
-        if (saw_bad) atomicOr(a.status, PRE_ST_BADREQ);
-        if (saw_full) atomicOr(a.status, PRE_ST_CAPACITY);
+        // what the loop noted beyond a blocked request is decided again below and does not count here
+        const long long decided = (ADMIT && blocked) ? pidx : n_items;
+        if (saw_bad && (!ADMIT || first_bad < decided)) atomicOr(a.status, PRE_ST_BADREQ);
+        if (saw_full && (!ADMIT || first_full < decided)) atomicOr(a.status, PRE_ST_CAPACITY);
+    }
+
+    if (ADMIT && b == 0) {
+        // Everything from the blocked request on: a request that was waiting keeps its place; an
+        // arrival joins the tail of the queue while there is room and is turned away otherwise
+        // (a malformed arrival is dropped).  Nothing else reads or writes these arrays any more:
+        // the other blocks only look at items up to the one they are scanning, whose fields they
+        // read before the exchange that stopped the batch.
+        __syncthreads();
+        const bool lost = sh_dead != 0;
+        const long long stop = blocked ? pidx : n_items;
+        const long long left = stop < q_len ? q_len - stop : 0;          // waiting entries that stay
+        for (long long k = stop + tid; k < q_len; k += ROUTE_THREADS) a.queue_choice[k] = CHOICE_WAITS;
+        __shared__ long long sh_joined;
+        __shared__ int sh_warp_ok[ROUTE_WARPS];
+        __shared__ int sh_any_bad;
+        if (tid == 0) { sh_joined = 0; sh_any_bad = 0; }
+        __syncthreads();
+        const long long a0 = (stop > q_len ? stop : q_len) - q_len;      // first arrival that was not decided
+        for (long long base = a0; base < a.n_arrivals && !lost; base += ROUTE_THREADS) {
+            const long long i = base + tid;
+            int P = -1, D = 0;
+            if (i < a.n_arrivals) { P = a.arr_prompt[i]; D = a.arr_predicted[i]; }
+            const bool ok = i < a.n_arrivals && !(P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX);
+            const unsigned int vote = __ballot_sync(0xffffffffu, ok);
+            if (lane == 0) sh_warp_ok[warp] = __popc(vote);
+            __syncthreads();
+            long long rank = sh_joined + __popc(vote & ((1u << lane) - 1u));
+            int total = 0;
+            for (int x = 0; x < ROUTE_WARPS; ++x) { if (x < warp) rank += sh_warp_ok[x]; total += sh_warp_ok[x]; }
+            if (i < a.n_arrivals) {
+                int c = CHOICE_DROPPED;
+                if (ok) {
+                    if (left + rank < a.queue_capacity) {
+                        const long long pos = (q_head + q_len + rank) % a.queue_capacity;   // behind the last one waiting
+                        a.queue_prompt[pos] = P;
+                        a.queue_predicted[pos] = D;
+                        c = CHOICE_WAITS;
+                    } else {
+                        c = CHOICE_TURNED_AWAY;
+                    }
+                } else {
+                    sh_any_bad = 1;
+                }
+                a.choice[i] = c;
+                if (a.score) a.score[i] = 0.0;
+            }
+            __syncthreads();
+            if (tid == 0) sh_joined += total;
+            __syncthreads();
+        }
+        if (tid == 0 && !lost) {
+            long long joined = sh_joined;
+            if (left + joined > a.queue_capacity) joined = a.queue_capacity - left;
+            a.queue_state[0] = a.queue_capacity > 0 ? (q_head + (q_len - left)) % a.queue_capacity : 0;
+            a.queue_state[1] = left + joined;
+            if (blocked && sh_any_bad) atomicOr(a.status, PRE_ST_BADREQ);
+        }
     }
 }
 
 }  // namespace
 
-cudaError_t pre_route_configure(pre_ctx* ctx) {
-    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
-    const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
-    const int max_rows = (I + G - 1) / G;
-    const size_t fixed = (size_t)max_rows * 48;  // five 8-byte and two 4-byte words per row
-    cudaDeviceProp prop;
-    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
-    if (e != cudaSuccess) return e;
+// Shared-memory split of one instantiation: `fixed_per_row` bytes of per-row words, the rest for resident rows.
+template <bool ADMIT>
+static cudaError_t configure_one(pre_ctx* ctx, int G, int max_rows, size_t limit, size_t* smem_out,
+                                 size_t* resident_out) {
+    const int H = ctx->cfg.horizon;
+    const size_t fixed = (size_t)max_rows * (ADMIT ? 64 : 48);  // five 8-byte and two 4-byte words per row (+ the overload count)
     cudaFuncAttributes attr;
-    e = cudaFuncGetAttributes(&attr, pre_route_persistent);
+    cudaError_t e = cudaFuncGetAttributes(&attr, pre_route_persistent<ADMIT>);
     if (e != cudaSuccess) return e;
-    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
-    if (fixed + attr.sharedSizeBytes + 1024 > limit) return cudaErrorInvalidConfiguration;
+    const size_t spare = 256;   // left unused; the occupancy query below confirms that the block still fits
+    if (fixed + attr.sharedSizeBytes + spare > limit) return cudaErrorInvalidConfiguration;
     // what is left beside the fixed part holds resident rows (the kernel decides how many)
-    size_t resident_bytes = limit - attr.sharedSizeBytes - 1024 - fixed;
+    size_t resident_bytes = limit - attr.sharedSizeBytes - spare - fixed;
     if (resident_bytes > (size_t)max_rows * H * sizeof(int64_t)) resident_bytes = (size_t)max_rows * H * sizeof(int64_t);
     resident_bytes &= ~(size_t)15;
     const size_t smem = fixed + resident_bytes;
     // (the limit is shared by every context of the process: always the device maximum)
-    e = cudaFuncSetAttribute(pre_route_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(pre_route_persistent<ADMIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(limit - attr.sharedSizeBytes));
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pre_route_persistent, ROUTE_THREADS, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pre_route_persistent<ADMIT>, ROUTE_THREADS, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) return cudaErrorInvalidConfiguration;
-    ctx->route_blocks = G;
-    ctx->route_threads = ROUTE_THREADS;
-    ctx->route_smem = smem;
-    ctx->route_resident_bytes = resident_bytes;
+    (void)G;
+    *smem_out = smem;
+    *resident_out = resident_bytes;
     return cudaSuccess;
 }
 
-cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
-                             int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
-                             int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
-                             int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
-    if (n_arrivals == 0) return cudaSuccess;
-    cudaError_t e = cudaMemsetAsync(ctx->d_abort, 0, sizeof(int), s);
+cudaError_t pre_route_configure(pre_ctx* ctx) {
+    const int I = ctx->cfg.n_instances;
+    const int G = ctx->n_sm < I ? ctx->n_sm : I;  // one block per SM, never more blocks than rows
+    const int max_rows = (I + G - 1) / G;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
     if (e != cudaSuccess) return e;
-    RouteArgs a;
+    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+    e = configure_one<false>(ctx, G, max_rows, limit, &ctx->route_smem, &ctx->route_resident_bytes);
+    if (e != cudaSuccess) return e;
+    e = configure_one<true>(ctx, G, max_rows, limit, &ctx->route_smem_admit, &ctx->route_resident_bytes_admit);
+    if (e != cudaSuccess) return e;
+    ctx->route_blocks = G;
+    ctx->route_threads = ROUTE_THREADS;
+    return cudaSuccess;
+}
+
+static void fill_route_args(RouteArgs& a, pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                            int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                            int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                            int64_t* n_requests, int32_t* choice, double* score) {
     a.arr_prompt = arr_prompt; a.arr_predicted = arr_predicted; a.n_arrivals = n_arrivals;
     a.curves = curves; a.queued_p = queued_p; a.current_d = current_d;
     a.prompt = prompt; a.generated = generated; a.predicted = predicted; a.instance = instance;
@@ -768,7 +930,51 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
     a.status = ctx->d_status; a.abort_flag = ctx->d_abort;
     a.max_rows = (a.I + ctx->route_blocks - 1) / ctx->route_blocks;
     a.resident_bytes = ctx->route_resident_bytes;
+    a.queue_prompt = nullptr; a.queue_predicted = nullptr; a.queue_state = nullptr; a.queue_entry = nullptr;
+    a.queue_capacity = 0; a.queue_choice = nullptr; a.hot = 0; a.many = 0.0;
+}
+
+cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                             int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                             int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                             int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
+    if (n_arrivals == 0) return cudaSuccess;
+    cudaError_t e = cudaMemsetAsync(ctx->d_abort, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    RouteArgs a;
+    fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
+                    predicted, instance, n_requests, choice, score);
     void* params[] = {(void*)&a};
-    return cudaLaunchCooperativeKernel((const void*)pre_route_persistent, dim3(ctx->route_blocks),
+    return cudaLaunchCooperativeKernel((const void*)pre_route_persistent<false>, dim3(ctx->route_blocks),
                                        dim3(ROUTE_THREADS), params, ctx->route_smem, s);
+}
+
+cudaError_t pre_launch_route_admit(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                   int64_t n_arrivals, double overload_level, double overload_share,
+                                   int32_t* queue_prompt, int32_t* queue_predicted, int64_t* queue_state,
+                                   int64_t queue_capacity, int32_t* queue_choice, int64_t* curves,
+                                   int64_t* queued_p, int64_t* current_d, int32_t* prompt, int32_t* generated,
+                                   int32_t* predicted, int32_t* instance, int64_t* n_requests, int32_t* choice,
+                                   double* score, cudaStream_t s) {
+    // The kernel's blocks read the queue's head and length while block 0 may already be writing the
+    // new ones: they read a copy taken here, in stream order.
+    cudaError_t e = cudaMemcpyAsync(ctx->d_queue_entry, queue_state, 2 * sizeof(int64_t), cudaMemcpyDeviceToDevice, s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(ctx->d_abort, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    RouteArgs a;
+    fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
+                    predicted, instance, n_requests, choice, score);
+    a.resident_bytes = ctx->route_resident_bytes_admit;
+    a.queue_prompt = queue_prompt; a.queue_predicted = queue_predicted; a.queue_state = queue_state;
+    a.queue_entry = ctx->d_queue_entry; a.queue_capacity = queue_capacity; a.queue_choice = queue_choice;
+    // For a whole number c, c > x holds exactly when c > floor(x): the per-cell test is done on integers.
+    double hot = floor(overload_level * (double)ctx->cfg.capacity_tokens);
+    if (hot > 9.2e18) hot = 9.2e18;
+    if (hot < -9.2e18) hot = -9.2e18;
+    a.hot = (long long)hot;
+    a.many = overload_share * (double)a.H;
+    void* params[] = {(void*)&a};
+    return cudaLaunchCooperativeKernel((const void*)pre_route_persistent<true>, dim3(ctx->route_blocks),
+                                       dim3(ROUTE_THREADS), params, ctx->route_smem_admit, s);
 }

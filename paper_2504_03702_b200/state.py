@@ -61,6 +61,29 @@ class DeviceState:
                                   self.n_requests, choice, score), "pre_route_batch")
         return choice, score
 
+    def make_queue(self, capacity):
+        """Empty admission queue (a ring in device memory) of the given capacity."""
+        self.queue_capacity = int(capacity)
+        n = max(self.queue_capacity, 1)
+        self.queue_prompt = torch.zeros(n, dtype=torch.int32, device=self.device)
+        self.queue_predicted = torch.zeros(n, dtype=torch.int32, device=self.device)
+        self.queue_choice = torch.zeros(n, dtype=torch.int32, device=self.device)
+        self.queue_state = torch.zeros(2, dtype=torch.int64, device=self.device)     # head, length
+
+    def route_admit(self, arr_prompt, arr_predicted, overload_level=0.95, overload_share=0.10, want_score=True):
+        """Router with the admission queue. Returns device tensors (queue_choice int32[capacity],
+        choice int32[A], score float64[A] or None); queue_choice is meaningful for the entries that
+        were waiting when the call was made."""
+        a = int(arr_prompt.shape[0])
+        choice = torch.empty(a, dtype=torch.int32, device=self.device)
+        score = torch.empty(a, dtype=torch.float64, device=self.device) if want_score else None
+        B.check(B.pre_route_admit(self.ctx, arr_prompt, arr_predicted, a, overload_level, overload_share,
+                                  self.queue_prompt, self.queue_predicted, self.queue_state, self.queue_capacity,
+                                  self.queue_choice, self.curves, self.queued_p, self.current_d, self.prompt,
+                                  self.generated, self.predicted, self.instance, self.n_requests, choice, score),
+                "pre_route_admit")
+        return self.queue_choice, choice, score
+
     def step(self):
         B.check(B.pre_step(self.ctx, self.prompt, self.generated, self.predicted, self.instance,
                            self.n_requests, self.curves, self.queued_p, self.current_d), "pre_step")

@@ -502,3 +502,119 @@ def test_refine_streaming_ticks():
         filled += len(ap)
     assert_state_equal(st, ref, "at the end of the stream")
     st.close()
+
+
+# ------------------------------------------------------------------ router with admission queue (Sec. 4.3.3)
+
+def both_with_queue(wl, capacity):
+    st, ref = both(wl)
+    st.make_queue(capacity)
+    ref.make_queue(capacity)
+    return st, ref
+
+
+def admit_both(st, ref, ap, ad, level, share, what=""):
+    """One call on both sides; compares results, the queue and the whole state."""
+    waiting = int(ref.queue_state[1])
+    qc, c, s = st.route_admit(dev(ap), dev(ad), overload_level=level, overload_share=share)
+    wqc, wc, ws = ref.route_admit(ap, ad, overload_level=level, overload_share=share, fast=True)
+    c = c.cpu().numpy()
+    assert (c == wc).all(), f"{what}: first difference at arrival {int(np.argmax(c != wc))}: {c[c != wc][:4]} vs {wc[c != wc][:4]}"
+    assert (qc[:waiting].cpu().numpy() == wqc).all(), f"{what}: results of the waiting requests differ"
+    assert_scores_close(s.cpu().numpy(), ws, wc)
+    assert (s.cpu().numpy()[wc < 0] == 0).all()
+    assert st.queue_state.cpu().numpy().tolist() == ref.queue_state.tolist(), f"{what}: queue head/length differ"
+    head, n = (int(v) for v in ref.queue_state)
+    if n:
+        idx = (head + np.arange(n)) % ref.queue_capacity
+        assert (st.queue_prompt.cpu().numpy()[idx] == ref.queue_prompt[idx]).all(), f"{what}: queue contents differ"
+        assert (st.queue_predicted.cpu().numpy()[idx] == ref.queue_predicted[idx]).all(), f"{what}: queue contents differ"
+    assert_state_equal(st, ref, what)
+    return wc
+
+
+@pytest.mark.parametrize("idx,level,first_blocked", [(0, 0.6, 25), (1, 0.6, 335), (2, 0.3, 5979), (1, 0.95, None),
+                                                     (0, 0.3, 0)])
+def test_admit_configs(idx, level, first_blocked):
+    wl = W.make_config(idx)
+    st, ref = both_with_queue(wl, 100)
+    ap, ad = wl.ticks[0]
+    c = admit_both(st, ref, ap, ad, level, 0.10, f"config {idx}")
+    if first_blocked is None:
+        assert (c >= 0).all()
+    else:
+        assert (c[:first_blocked] >= 0).all() and (c[first_blocked:] < 0).all()
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+def test_admit_never_blocking_equals_route_batch():
+    wl = W.make_config(1)
+    st, ref = both_with_queue(wl, 10)
+    plain = DeviceState.from_workload(wl)
+    plain.anticipate()
+    ap, ad = wl.ticks[0]
+    _, c, s = st.route_admit(dev(ap), dev(ad), overload_level=1e9)
+    pc, ps = plain.route_batch(dev(ap), dev(ad))
+    assert (c == pc).all() and (s == ps).all() and (st.curves == plain.curves).all()
+    st.close()
+    plain.close()
+
+
+@pytest.mark.parametrize("seed,n_inst,h,n,a,qcap,level", [(11, 3, 8, 30, 40, 5, 0.7), (12, 2, 5, 10, 30, 0, 0.7),
+                                                          (13, 5, 16, 80, 60, 100, 0.5), (14, 1, 4, 6, 12, 3, 0.9),
+                                                          (15, 4, 12, 50, 64, 7, 0.7), (16, 300, 64, 4000, 900, 64, 0.8),
+                                                          (17, 149, 128, 3000, 700, 1000, 0.75)])
+def test_admit_shapes_over_several_calls(seed, n_inst, h, n, a, qcap, level):
+    """Calls alternate with decode steps: requests wait, are routed later, the ring's head moves on."""
+    wl = W.make_random(seed, n_inst, h, n, a, max_prompt=30, max_output=20)
+    st, ref = both_with_queue(wl, qcap)
+    ap, ad = wl.ticks[0]
+    seen = set()
+    for call in range(4):
+        lo, hi = call * a // 4, (call + 1) * a // 4
+        c = admit_both(st, ref, ap[lo:hi], ad[lo:hi], level, 0.25, f"call {call}")
+        seen |= set(np.sign(c).tolist()) | set(c[c < 0].tolist())
+        for _ in range(3):
+            st.step()
+            ref.step()
+    assert_state_equal(st, ref, "at the end")
+    if seed < 16:
+        assert 1 in seen or 0 in seen
+        assert -2 in seen or -3 in seen
+    st.close()
+
+
+def test_admit_long_tail_after_the_block_and_malformed_arrivals():
+    """Thousands of arrivals behind the blocked one: they join the queue in order until it is full."""
+    wl = W.make_config(2)
+    st, ref = both_with_queue(wl, 1500)
+    ap, ad = (x.copy() for x in wl.ticks[0])
+    ap[6000] = -5                       # malformed, beyond the point where the batch blocks
+    ad[7000] = 0
+    ap[17] = -1                         # malformed, before it
+    c = admit_both(st, ref, ap, ad, 0.3, 0.10, "first call")
+    assert c[17] == -1 and c[6000] == -1 and c[7000] == -1
+    assert (c == -2).sum() == 1500 and (c == -3).sum() > 0
+    assert st.status() == B.PRE_EBADREQ
+    # nothing drains: a second call changes nothing but the results
+    c = admit_both(st, ref, ap[:10], ad[:10], 0.3, 0.10, "second call")
+    assert (c == -3).all()
+    # 200 steps later the queue drains (in order) before the new arrivals
+    for _ in range(200):
+        st.step()
+        ref.step()
+    admit_both(st, ref, ap[:64], ad[:64], 0.3, 0.10, "third call")
+    st.close()
+
+
+def test_admit_table_full_and_empty_call():
+    wl = W.make_random(31, 4, 16, 20, 12)
+    wl.max_requests = 25
+    st, ref = both_with_queue(wl, 8)
+    ap, ad = wl.ticks[0]
+    c = admit_both(st, ref, ap, ad, 1e9, 0.1, "table fills")
+    assert (c[:5] >= 0).all() and (c[5:] == -1).all()
+    assert st.status() == B.PRE_ECAPACITY
+    admit_both(st, ref, ap[:0], ad[:0], 1e9, 0.1, "empty call")
+    st.close()
