@@ -9,30 +9,52 @@
 // so each request costs one shared-memory update and column 0 is not a hot spot.
 //
 // Pipeline (all on the caller's stream, no host synchronisation).  A tile is T
-// consecutive instance rows, built by one block in shared memory.
-//   1. pre_chunk_sort   each block takes a contiguous chunk of the table, packs every live
-//                       request into 8 bytes, orders them by tile inside the chunk (counting
-//                       sort in shared memory) and records where each tile starts in it
-//   2. pre_tile_build   one block per tile: gathers the tile's requests from every chunk,
+// consecutive instance rows (T a power of two), built by one block in shared memory.
+//   1. pre_chunk_sort   each block takes a contiguous chunk of the table and turns every live
+//                       request into an 8-byte record {where its update goes inside the tile's
+//                       shared memory, B}; records are ordered by tile inside the chunk (the
+//                       rank of a request is what its counting atomic returns) and the block
+//                       records where each tile starts in the chunk
+//   2. pre_tile_build   one block per tile: gathers the tile's records from every chunk,
 //                       accumulates (count, sum B) per (row, R-1) with shared-memory atomics,
-//                       suffix-scans over the horizon and writes the rows
-// No global atomics, no counting pass.  When there are more tiles than a block can count in
-// shared memory, a slower path is taken: pre_bin_count, pre_bin_scan, pre_bin_scatter
-// (global per-tile cursors) feed the same pre_tile_build.
+//                       suffix-scans over the horizon in registers and writes the rows
+// No counting pass over the table.  When there are more tiles than a block can count in
+// shared memory, or more chunks than the offset table is wide, a slower path is taken:
+// pre_bin_count, pre_bin_scan, pre_bin_scatter (global per-tile cursors) feed the same
+// pre_tile_build.
+//
+// The part of a request's remaining length that lies beyond the window, (D - g - H)+, only
+// matters for current_d; the first pass adds it to a per-instance scratch array (a global
+// reduction, a few percent of the requests), the tile kernel adds it in and clears it again.
+#include <cuda.h>   // CUtensorMap (types only; the encoder is fetched through the runtime)
+
+#include <cstring>
+
 #include "pre_common.cuh"
 
 namespace {
 
 constexpr int BIN_THREADS = 512;
+constexpr int RUN = 16;                 // consecutive cells of a row that one thread scans: 128 bytes
+
+// Shape of the build, the same for every kernel of a call.
+struct BuildShape {
+    int I, H;
+    int tile_shift;   // log2 of the rows per tile
+    int n_tiles;
+    int rpr;          // runs per row
+    int hp;           // rpr * RUN: cells of a padded row
+};
 
 // Slow path only.  Per-tile request counts.  Finished and malformed requests may be counted
 // too: the counts only reserve room, the scatter pass decides what is written.
 __global__ void __launch_bounds__(BIN_THREADS)
-pre_bin_count(const int32_t* __restrict__ instance, int64_t n, int I, int T, unsigned int* __restrict__ bin_count) {
+pre_bin_count(const int32_t* __restrict__ instance, int64_t n, int I, int tile_shift,
+              unsigned int* __restrict__ bin_count) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += stride) {
         const int32_t v = instance[r];
-        if ((uint32_t)v < (uint32_t)I) atomicAdd(&bin_count[v / T], 1u);
+        if ((uint32_t)v < (uint32_t)I) atomicAdd(&bin_count[v >> tile_shift], 1u);
     }
 }
 
@@ -64,147 +86,170 @@ pre_bin_scan(const unsigned int* __restrict__ bin_count, int n_tiles, unsigned i
     }
 }
 
-struct Packed { bool live; bool bad; int tile; unsigned long long rec; };
-
-__device__ __forceinline__ Packed pack_request(int32_t P, int32_t g, int32_t D, int32_t inst, int I, int T) {
-    Packed o;
-    o.live = false; o.bad = false; o.tile = 0; o.rec = 0;
-    if (!pre_request_ok(P, g, D, inst, I)) { o.bad = true; return o; }
-    if (g >= D) return o;  // finished: tombstone
-    const int64_t B = (int64_t)P + g;
-    const int32_t rem = D - g;
-    if (B > PRE_FIELD_MAX || rem > PRE_FIELD_MAX) { o.bad = true; return o; }
-    o.live = true;
-    o.tile = inst / T;
-    const unsigned long long local = (unsigned long long)(inst - o.tile * T);
-    o.rec = (local << (2 * PRE_FIELD_BITS)) | ((unsigned long long)B << PRE_FIELD_BITS) |
-            (unsigned long long)rem;
-    return o;
+// Where cell c of a tile (row within tile * hp + column) lies in the tile's shared memory.  Run
+// c/16 occupies 128 consecutive bytes; inside them the 16-byte piece p is stored at position
+// p ^ (run & 7).  This is the 128-byte swizzle of the tensor copy unit, so a finished tile can
+// leave shared memory in one bulk tensor store, and it lets 32 threads that each own a run
+// read and write their runs 16 bytes at a time without bank conflicts.
+__host__ __device__ __forceinline__ unsigned int cell_bytes(unsigned int c) {
+    const unsigned int run = c >> 4, k = c & 15u;
+    return (run << 7) | ((((k >> 1) ^ (run & 7u)) << 4)) | ((k & 1u) << 3);
 }
 
-// Calls f(P, g, D, inst) for every request of [r0, r1); 16-byte loads when the four arrays
-// allow it (r0 is then a multiple of 4, or the range is empty).
-template <class F>
-__device__ __forceinline__ void for_each_request(const int32_t* __restrict__ prompt,
-                                                 const int32_t* __restrict__ generated,
-                                                 const int32_t* __restrict__ predicted,
-                                                 const int32_t* __restrict__ instance, int64_t r0, int64_t r1,
-                                                 bool vec, F f) {
-    if (vec) {
-        const int64_t q1 = r1 >> 2;  // full quads end here
-        for (int64_t q = (r0 >> 2) + threadIdx.x; q < q1; q += blockDim.x) {
-            const int4 p = __ldg(reinterpret_cast<const int4*>(prompt) + q);
-            const int4 g = __ldg(reinterpret_cast<const int4*>(generated) + q);
-            const int4 d = __ldg(reinterpret_cast<const int4*>(predicted) + q);
-            const int4 i = __ldg(reinterpret_cast<const int4*>(instance) + q);
-            f(p.x, g.x, d.x, i.x); f(p.y, g.y, d.y, i.y); f(p.z, g.z, d.z, i.z); f(p.w, g.w, d.w, i.w);
-        }
-        for (int64_t r = (q1 << 2) + threadIdx.x; r < r1; r += blockDim.x)
-            if (r >= r0) f(prompt[r], generated[r], predicted[r], instance[r]);
-    } else {
-        for (int64_t r = r0 + threadIdx.x; r < r1; r += blockDim.x)
-            f(prompt[r], generated[r], predicted[r], instance[r]);
-    }
+// A request as the tile kernel wants it: {byte offset of its cell word in the tile's shared
+// memory : 32 | B : 32}.  The cell of a request is (row within tile, R - 1).
+struct Packed {
+    bool live, bad;
+    int tile;
+    unsigned int excess;        // (D - g - H)+
+    unsigned long long rec;
+};
+
+__device__ __forceinline__ Packed pack_request(int32_t P, int32_t g, int32_t D, int32_t inst, const BuildShape& sh) {
+    Packed o;
+    const unsigned int B = (unsigned int)P + (unsigned int)g;              // exact when P, g >= 0
+    const int32_t rem = (int32_t)((unsigned int)D - (unsigned int)g);
+    const bool ok = ((P | g) >= 0) & (D >= 1) & ((unsigned int)inst < (unsigned int)sh.I);
+    const bool fits = (B <= (unsigned int)PRE_FIELD_MAX) & (rem <= PRE_FIELD_MAX);
+    const bool alive = ok & (rem > 0);                                     // g >= D: finished, a tombstone
+    o.bad = !ok | (alive & !fits);
+    o.live = alive & fits;
+    o.tile = inst >> sh.tile_shift;
+    const int local = inst & ((1 << sh.tile_shift) - 1);
+    const int R = rem < sh.H ? rem : sh.H;
+    o.excess = rem > sh.H ? (unsigned int)(rem - sh.H) : 0u;
+    o.rec = ((unsigned long long)cell_bytes((unsigned int)(local * sh.hp + R - 1)) << 32) | B;
+    return o;
 }
 
 // Slow path only: one global atomic per live request on its tile's cursor.
 __global__ void __launch_bounds__(BIN_THREADS)
 pre_bin_scatter(const int32_t* __restrict__ prompt, const int32_t* __restrict__ generated,
                 const int32_t* __restrict__ predicted, const int32_t* __restrict__ instance, int64_t n,
-                int I, int T, const unsigned int* __restrict__ bin_base, unsigned int* __restrict__ bin_cursor,
-                unsigned long long* __restrict__ records, int* __restrict__ status) {
-    int64_t chunk = (n + gridDim.x - 1) / gridDim.x;
-    chunk = (chunk + 3) & ~(int64_t)3;
-    const int64_t r0 = (int64_t)blockIdx.x * chunk < n ? (int64_t)blockIdx.x * chunk : n;
-    const int64_t r1 = r0 + chunk < n ? r0 + chunk : n;
-    const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
-                       reinterpret_cast<uintptr_t>(predicted) | reinterpret_cast<uintptr_t>(instance)) & 15) == 0;
+                const BuildShape sh, const unsigned int* __restrict__ bin_base,
+                unsigned int* __restrict__ bin_cursor, unsigned long long* __restrict__ records,
+                unsigned long long* __restrict__ excess, int* __restrict__ status) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     bool any_bad = false;
-    for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
-                     [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
-                         const Packed p = pack_request(P, g, D, inst, I, T);
-                         any_bad |= p.bad;
-                         if (p.live) records[bin_base[p.tile] + atomicAdd(&bin_cursor[p.tile], 1u)] = p.rec;
-                     });
+    for (int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; r < n; r += stride) {
+        const int32_t inst = instance[r];
+        const Packed p = pack_request(prompt[r], generated[r], predicted[r], inst, sh);
+        any_bad |= p.bad;
+        if (p.live) {
+            records[bin_base[p.tile] + atomicAdd(&bin_cursor[p.tile], 1u)] = p.rec;
+            if (p.excess) atomicAdd(&excess[inst], (unsigned long long)p.excess);
+        }
+    }
     if (any_bad) atomicOr(status, PRE_ST_BADREQ);
 }
 
 // ---------------------------------------------------------------------------------------
-// Fast path, step 1.  Block `ch` owns table rows [ch*chunk, (ch+1)*chunk) and the same span
-// of `records`.  It writes its live requests there ordered by tile and stores, for every
-// tile t, the offset of t's first record inside the span: chunk_off[t*NC + ch]
-// (chunk_off[n_tiles*NC + ch] = number of live requests of the chunk).
+// Fast path, step 1.  Block `ch` owns table rows [ch*chunk, (ch+1)*chunk), chunk <= SORT_CHUNK,
+// and the same span of `records`.  Every thread keeps its (at most eight) records in
+// registers: all table loads are issued before the first is used, the per-tile rank of a
+// request is the value its counting atomic returns, and after one scan of the per-tile counts
+// each record is stored at (tile start + rank).  The chunk's records end up ordered by tile;
+// chunk_off[ch*n_tiles + t] = {start of tile t inside the span : 16 | number of its records : 16}
+// (a chunk has at most 4,096 rows, so both fit); chunk_max[ch] = largest B of the chunk.
 constexpr int SORT_THREADS = 512;
-constexpr int SORT_CHUNK = 6144;   // requests a block can stage in shared memory
-constexpr int SORT_MAX_CHUNKS = 1024;
+constexpr int SORT_QUADS = 2;                                  // 16-byte loads per thread and array
+constexpr int SORT_SLOTS = 4 * SORT_QUADS;                     // requests a thread holds
+constexpr int SORT_CHUNK = SORT_THREADS * SORT_SLOTS;          // 4,096
+constexpr int SORT_MAX_CHUNKS = 4096;                          // widest offset table (16.7 M requests)
 
-__global__ void __launch_bounds__(SORT_THREADS)
+__global__ void __launch_bounds__(SORT_THREADS, 2)
 pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ generated,
                const int32_t* __restrict__ predicted, const int32_t* __restrict__ instance, int64_t n,
-               int I, int T, int n_tiles, int64_t chunk, int staged, unsigned long long* __restrict__ records,
-               unsigned int* __restrict__ chunk_off, int* __restrict__ status) {
-    extern __shared__ __align__(16) unsigned char sort_smem[];
+               const BuildShape sh, int64_t chunk, unsigned long long* __restrict__ records,
+               unsigned int* __restrict__ chunk_off, unsigned int* __restrict__ chunk_max,
+               unsigned long long* __restrict__ excess, int* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned int hist[];    // [n_tiles + 1], rounded up to whole 16-byte groups
     __shared__ unsigned int warp_tot[SORT_THREADS / 32];
-    // layout: [stage: u64 x SORT_CHUNK][tile_of: u16 x SORT_CHUNK] (only when staged) [hist: u32 x (n_tiles+1)]
-    unsigned long long* stage = reinterpret_cast<unsigned long long*>(sort_smem);
-    unsigned short* tile_of = reinterpret_cast<unsigned short*>(stage + (staged ? SORT_CHUNK : 0));
-    unsigned int* hist = reinterpret_cast<unsigned int*>(tile_of + (staged ? SORT_CHUNK : 0));
+    __shared__ unsigned int block_max;
 
-    const int ch = blockIdx.x, NC = gridDim.x;
+    const int n_tiles = sh.n_tiles;
+    const int ch = blockIdx.x;
     const int64_t r0 = (int64_t)ch * chunk < n ? (int64_t)ch * chunk : n;
     const int64_t r1 = r0 + chunk < n ? r0 + chunk : n;
+    const int cnt = (int)(r1 - r0);
     const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
                        reinterpret_cast<uintptr_t>(predicted) | reinterpret_cast<uintptr_t>(instance)) & 15) == 0;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    bool any_bad = false;
 
-    for (int i = tid; i <= n_tiles; i += SORT_THREADS) hist[i] = 0;
-    __syncthreads();
-
-    // ---- pass A: pack, count per tile (and keep the packed request when it fits)
-    if (staged) {
-        // one request per (thread, slot): slot li = r - r0 < SORT_CHUNK
-        auto take = [&](int64_t r, int32_t P, int32_t g, int32_t D, int32_t inst) {
-            const Packed p = pack_request(P, g, D, inst, I, T);
-            any_bad |= p.bad;
-            const int li = (int)(r - r0);
-            stage[li] = p.rec;
-            tile_of[li] = p.live ? (unsigned short)p.tile : (unsigned short)0xFFFF;
-            if (p.live) atomicAdd(&hist[p.tile], 1u);
-        };
-        if (vec) {
-            const int64_t q1 = r1 >> 2;
-            for (int64_t q = (r0 >> 2) + tid; q < q1; q += SORT_THREADS) {
-                const int4 p = __ldg(reinterpret_cast<const int4*>(prompt) + q);
-                const int4 g = __ldg(reinterpret_cast<const int4*>(generated) + q);
-                const int4 d = __ldg(reinterpret_cast<const int4*>(predicted) + q);
-                const int4 i = __ldg(reinterpret_cast<const int4*>(instance) + q);
-                const int64_t r = q << 2;
-                take(r, p.x, g.x, d.x, i.x); take(r + 1, p.y, g.y, d.y, i.y);
-                take(r + 2, p.z, g.z, d.z, i.z); take(r + 3, p.w, g.w, d.w, i.w);
-            }
-            for (int64_t r = (q1 << 2) + tid; r < r1; r += SORT_THREADS)
-                if (r >= r0) take(r, prompt[r], generated[r], predicted[r], instance[r]);
-        } else {
-            for (int64_t r = r0 + tid; r < r1; r += SORT_THREADS)
-                take(r, prompt[r], generated[r], predicted[r], instance[r]);
+    // ---- load: slot u of this thread is table row r0 + (u/4 * SORT_THREADS + tid) * 4 + u%4
+    int32_t P[SORT_SLOTS], G[SORT_SLOTS], D[SORT_SLOTS], N[SORT_SLOTS];
+    unsigned int present = 0;
+    if (vec && (SORT_QUADS - 1) * SORT_THREADS * 4 + tid * 4 + 4 <= cnt) {   // r0 is a multiple of 4
+        #pragma unroll
+        for (int h = 0; h < SORT_QUADS; ++h) {
+            const int64_t q = (r0 >> 2) + h * SORT_THREADS + tid;
+            const int4 p = __ldg(reinterpret_cast<const int4*>(prompt) + q);
+            const int4 g = __ldg(reinterpret_cast<const int4*>(generated) + q);
+            const int4 d = __ldg(reinterpret_cast<const int4*>(predicted) + q);
+            const int4 i = __ldg(reinterpret_cast<const int4*>(instance) + q);
+            P[4 * h] = p.x; P[4 * h + 1] = p.y; P[4 * h + 2] = p.z; P[4 * h + 3] = p.w;
+            G[4 * h] = g.x; G[4 * h + 1] = g.y; G[4 * h + 2] = g.z; G[4 * h + 3] = g.w;
+            D[4 * h] = d.x; D[4 * h + 1] = d.y; D[4 * h + 2] = d.z; D[4 * h + 3] = d.w;
+            N[4 * h] = i.x; N[4 * h + 1] = i.y; N[4 * h + 2] = i.z; N[4 * h + 3] = i.w;
         }
+        present = (1u << SORT_SLOTS) - 1;
     } else {
-        for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
-                         [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
-                             const Packed p = pack_request(P, g, D, inst, I, T);
-                             any_bad |= p.bad;
-                             if (p.live) atomicAdd(&hist[p.tile], 1u);
-                         });
+        #pragma unroll
+        for (int u = 0; u < SORT_SLOTS; ++u) {
+            const int li = ((u >> 2) * SORT_THREADS + tid) * 4 + (u & 3);
+            P[u] = G[u] = D[u] = N[u] = 0;
+            if (li < cnt) {
+                const int64_t r = r0 + li;
+                P[u] = __ldg(prompt + r); G[u] = __ldg(generated + r);
+                D[u] = __ldg(predicted + r); N[u] = __ldg(instance + r);
+                present |= 1u << u;
+            }
+        }
     }
+    // hist is cleared 16 bytes at a time (it is padded to whole groups)
+    const int groups = (n_tiles + 4) >> 2;                    // 16-byte groups that cover n_tiles + 1 counts
+    for (int i = tid; i < groups; i += SORT_THREADS) reinterpret_cast<uint4*>(hist)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) block_max = 0;
     __syncthreads();
 
-    // ---- exclusive scan of the per-tile counts, in place (each thread a contiguous run)
+    // ---- pack and count: the counting atomic hands back the request's rank inside its tile
+    unsigned long long rec[SORT_SLOTS];
+    int tile_of[SORT_SLOTS];                 // -1 when there is nothing to place
+    unsigned int rank[SORT_SLOTS];
+    bool any_bad = false;
+    unsigned int max_b = 0;
+    #pragma unroll
+    for (int u = 0; u < SORT_SLOTS; ++u) {
+        const Packed p = pack_request(P[u], G[u], D[u], N[u], sh);
+        const bool here = (present >> u) & 1u;
+        const bool live = here & p.live;
+        any_bad |= here & p.bad;
+        rec[u] = p.rec;
+        tile_of[u] = live ? p.tile : -1;
+        const unsigned int b = live ? (unsigned int)p.rec : 0u;
+        max_b = b > max_b ? b : max_b;
+        if (live && p.excess) atomicAdd(&excess[N[u]], (unsigned long long)p.excess);
+    }
+    #pragma unroll
+    for (int u = 0; u < SORT_SLOTS; ++u) {
+        rank[u] = 0;
+        if (tile_of[u] >= 0) rank[u] = atomicAdd(&hist[tile_of[u]], 1u);
+    }
+    max_b = __reduce_max_sync(0xffffffffu, max_b);
+    if (lane == 0 && max_b) atomicMax(&block_max, max_b);
+    __syncthreads();
+
+    // ---- exclusive scan of the per-tile counts, in place; a thread owns whole 16-byte groups
     {
-        const int per = (n_tiles + SORT_THREADS) / SORT_THREADS;  // covers n_tiles + 1 entries
-        const int b0 = tid * per;
+        const int per = (groups + SORT_THREADS - 1) / SORT_THREADS;
+        const int g0 = tid * per;
         unsigned int local = 0;
-        for (int k = 0; k < per; ++k) if (b0 + k <= n_tiles) local += hist[b0 + k];
+        for (int k = 0; k < per; ++k) {
+            if (g0 + k < groups) {
+                const uint4 v = reinterpret_cast<const uint4*>(hist)[g0 + k];
+                local += v.x + v.y + v.z + v.w;
+            }
+        }
         unsigned int x = local;
         #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -213,270 +258,608 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
         }
         if (lane == 31) warp_tot[warp] = x;
         __syncthreads();
-        unsigned int run = x - local;
-        for (int w = 0; w < warp; ++w) run += warp_tot[w];
+        // what the warps before this one hold: a 16-lane scan of the warp totals
+        unsigned int w = lane < SORT_THREADS / 32 ? warp_tot[lane] : 0u;
+        #pragma unroll
+        for (int off = 1; off < SORT_THREADS / 32; off <<= 1) {
+            const unsigned int y = __shfl_up_sync(0xffffffffu, w, off);
+            if (lane >= off) w += y;
+        }
+        const unsigned int before = __shfl_sync(0xffffffffu, w, warp > 0 ? warp - 1 : 0);
+        unsigned int run = x - local + (warp > 0 ? before : 0u);
         for (int k = 0; k < per; ++k) {
-            const int i = b0 + k;
-            if (i <= n_tiles) {
-                const unsigned int c = hist[i];
-                hist[i] = run;                              // becomes the tile's write cursor
-                chunk_off[(size_t)i * NC + ch] = run;       // entry n_tiles receives the total
-                run += c;
+            if (g0 + k < groups) {
+                const uint4 v = reinterpret_cast<const uint4*>(hist)[g0 + k];
+                uint4 o;
+                o.x = run; run += v.x;
+                o.y = run; run += v.y;
+                o.z = run; run += v.z;
+                o.w = run; run += v.w;
+                reinterpret_cast<uint4*>(hist)[g0 + k] = o;   // entries past n_tiles hold the chunk's total
             }
         }
     }
     __syncthreads();
 
-    // ---- pass B: place
-    unsigned long long* out = records + r0;
-    if (staged) {
-        const int cnt = (int)(r1 - r0);
-        for (int l0 = tid; l0 < cnt; l0 += 4 * SORT_THREADS) {   // four independent cursor bumps in flight
-            unsigned int t[4], pos[4];
-            #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int li = l0 + u * SORT_THREADS;
-                t[u] = li < cnt ? tile_of[li] : 0xFFFFu;
-            }
-            #pragma unroll
-            for (int u = 0; u < 4; ++u) pos[u] = t[u] != 0xFFFFu ? atomicAdd(&hist[t[u]], 1u) : 0u;
-            #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (t[u] != 0xFFFFu) out[pos[u]] = stage[l0 + u * SORT_THREADS];
-        }
-    } else {
-        for_each_request(prompt, generated, predicted, instance, r0, r1, vec,
-                         [&](int32_t P, int32_t g, int32_t D, int32_t inst) {
-                             const Packed p = pack_request(P, g, D, inst, I, T);
-                             if (p.live) out[atomicAdd(&hist[p.tile], 1u)] = p.rec;
-                         });
+    // ---- offsets {start, length} (consecutive threads, consecutive tiles) and records
+    unsigned int* my_off = chunk_off + (size_t)ch * n_tiles;
+    for (int i = tid; i < n_tiles; i += SORT_THREADS) {
+        const unsigned int a = hist[i];
+        my_off[i] = a | ((hist[i + 1] - a) << 16);
     }
+    if (tid == 0) chunk_max[ch] = block_max;
+    unsigned long long* out = records + r0;
+    #pragma unroll
+    for (int u = 0; u < SORT_SLOTS; ++u)
+        if (tile_of[u] >= 0) out[hist[tile_of[u]] + rank[u]] = rec[u];
     if (any_bad) atomicOr(status, PRE_ST_BADREQ);
 }
 
 // ---------------------------------------------------------------------------------------
-// Step 2.  One block per tile.  Shared memory holds, per cell (row, j) of the tile, one
-// 64-bit word {low: sum of B mod 2^32, high: count} plus a rarely used 32-bit carry word
-// (so that only 32-bit shared atomics are needed).  Rows are padded to a multiple of RUN
-// cells; a run of RUN consecutive cells is scanned by one thread, and every run is
-// followed by 16 bytes of padding so that the threads' 16-byte loads fall in different banks.
-constexpr int TILE_THREADS = 256;
-constexpr int TILE_WARPS = TILE_THREADS / 32;
-constexpr int RUN = 16;
+// Step 2.  A persistent grid of blocks; a block builds one tile after another.  Shared memory
+// holds one 64-bit word per cell (row, j) of the tile, {low: sum of B, high: count}, updated
+// with two 32-bit atomics whose results are not needed, in the swizzled layout of cell_bytes().
+// A run of RUN consecutive cells of a row belongs to one thread, which keeps it in registers
+// for the whole scan.  A warp serves 32 consecutive runs of one row, or, when a row has fewer
+// than 32 runs, several rows side by side (W lanes each).  The finished tile, int64 values in
+// the same layout, leaves shared memory in bulk tensor stores issued by one thread while the
+// block already works on its next tile in the second cell buffer.
+//
+// Latency is hidden by looking ahead: a lane holds the offsets of its two chunks for the next
+// tile a whole tile early, and issues the loads of this tile's records before it waits for
+// the cell buffer and clears it.
+//
+// All sums, and the map values themselves, fit 32 bits as long as
+//     (records of the tile) * (max(largest B, 32) + H) < 2^32,
+// which the block checks once it has accumulated.  Otherwise it works in wide mode: the counts
+// stay in shared memory, the sums of B are accumulated with 64-bit atomics in the tile's own
+// rows of `curves` (cleared first), and the scan runs in 64 bits.
+constexpr int TILE_MAX_THREADS = 512;
+constexpr int TILE_BUFFERS = 2;
+constexpr int TMA_BOX_RUNS = 256;      // rows (runs of 128 bytes) of one bulk tensor store
 
-__device__ __forceinline__ int cell_slot(int c) { return c + ((c >> 4) << 1); }  // index in 8-byte words
+struct TileGeom {
+    int rpr;      // runs per row
+    int W;        // lanes that serve one row piece: 32, or the power of two >= rpr when rpr < 32
+    int w_shift;  // log2(W)
+    int cpw;      // 32-run pieces per row (1 when rpr <= 32)
+    int rpw;      // rows per warp (1 when rpr >= 32)
+};
 
-struct TileShape { int hp, rpr, cpw; };  // padded row length, runs per row, 32-run chunks per row
-
-__host__ __device__ inline TileShape tile_shape(int H) {
-    TileShape t;
-    t.rpr = (H + RUN - 1) / RUN;
-    t.hp = t.rpr * RUN;
-    t.cpw = (t.rpr + 31) / 32;
-    return t;
+inline TileGeom tile_geom(int H) {
+    TileGeom g;
+    g.rpr = (H + RUN - 1) / RUN;
+    if (g.rpr >= 32) {
+        g.W = 32; g.w_shift = 5; g.cpw = (g.rpr + 31) / 32; g.rpw = 1;
+    } else {
+        g.W = 1; g.w_shift = 0;
+        while (g.W < g.rpr) { g.W <<= 1; ++g.w_shift; }
+        g.cpw = 1; g.rpw = 32 / g.W;
+    }
+    return g;
 }
 
-__global__ void __launch_bounds__(TILE_THREADS, 3)
-pre_tile_build(const unsigned long long* __restrict__ records,
-               const unsigned int* __restrict__ chunk_off, int NC, int64_t chunk,          // fast path
-               const unsigned int* __restrict__ bin_base, unsigned int* __restrict__ bin_cursor,
-               unsigned int* __restrict__ bin_count,                                        // slow path
-               int I, int H, int T, int64_t* __restrict__ curves, int64_t* __restrict__ current_d) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const TileShape sh = tile_shape(H);
-    const int cells = T * sh.hp;            // padded cells of a full tile
-    const int n_runs_max = T * sh.rpr;
-    unsigned long long* cl = reinterpret_cast<unsigned long long*>(smem_raw);        // [cells * 9/8]
-    unsigned long long* run_s = cl + (cells + (cells >> 3));                          // [n_runs_max]
-    unsigned long long* run_w = run_s + n_runs_max;                                   // [n_runs_max]
-    unsigned long long* chk_s = run_w + n_runs_max;                                   // [T * cpw]
-    unsigned long long* excess = chk_s + T * sh.cpw;                                  // [T]
-    unsigned long long* sum_n = excess + T;                                           // [T]
-    uint32_t* run_n = reinterpret_cast<uint32_t*>(sum_n + T);                         // [n_runs_max]
-    uint32_t* chk_n = run_n + n_runs_max;                                             // [T * cpw]
-    uint32_t* hi = chk_n + T * sh.cpw;                                                // [cells]
-    __shared__ int any_hi;
+inline int tile_warps(int T, const TileGeom& g) {
+    return g.rpr >= 32 ? T * g.cpw : (T + g.rpw - 1) / g.rpw;
+}
 
-    const int tile = blockIdx.x;
-    const int row0 = tile * T;
-    const int rows = (I - row0) < T ? (I - row0) : T;
-    const int n_runs = rows * sh.rpr;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+struct TileArgs {
+    BuildShape sh;
+    TileGeom g;
+    const unsigned long long* records;
+    const unsigned int* chunk_off;     // fast path (else null)
+    const unsigned int* chunk_max;
+    int NC;
+    unsigned int chunk;
+    const unsigned int* bin_base;      // slow path
+    unsigned int* bin_cursor;
+    unsigned int* bin_count;
+    unsigned long long* excess;
+    int64_t* curves;
+    int64_t* current_d;
+    int buffer_runs;                   // runs of 128 bytes in one cell buffer (a multiple of 8)
+    int use_tma;                       // the tensor map describes `curves` as runs of 128 bytes
+};
 
-    {   // clear the cell words, the carry words and the per-row sums
-        uint4* z = reinterpret_cast<uint4*>(cl);
-        const int nz = (cells + (cells >> 3)) >> 1;
-        for (int i = tid; i < nz; i += TILE_THREADS) z[i] = make_uint4(0, 0, 0, 0);
-        for (int i = tid; i < cells; i += TILE_THREADS) hi[i] = 0;
-        for (int i = tid; i < 2 * T; i += TILE_THREADS) excess[i] = 0;
-        if (tid == 0) any_hi = 0;
+constexpr int GATHER_AHEAD = 4;   // records of a chunk's piece that a lane loads before using any
+
+// The pieces of the tile's records that this lane is responsible for in one trip over the
+// chunks: chunk c0 = first + lane and c1 = c0 + 32.
+struct Pieces {
+    const unsigned long long* p0;
+    const unsigned long long* p1;
+    unsigned int len0, len1;
+};
+
+__device__ __forceinline__ void load_offsets(const TileArgs& a, int tile, int first, unsigned int& w0,
+                                             unsigned int& w1) {
+    const int lane = threadIdx.x & 31;
+    const int c0 = first + lane, c1 = c0 + 32;
+    const bool in = tile < a.sh.n_tiles;
+    w0 = in && c0 < a.NC ? __ldg(a.chunk_off + ((unsigned int)c0 * (unsigned int)a.sh.n_tiles + tile)) : 0u;
+    w1 = in && c1 < a.NC ? __ldg(a.chunk_off + ((unsigned int)c1 * (unsigned int)a.sh.n_tiles + tile)) : 0u;
+}
+
+__device__ __forceinline__ Pieces pieces_of(const TileArgs& a, int first, unsigned int w0, unsigned int w1) {
+    const int lane = threadIdx.x & 31;
+    Pieces s;
+    s.len0 = w0 >> 16; s.len1 = w1 >> 16;
+    s.p0 = a.records + ((unsigned int)(first + lane) * a.chunk + (w0 & 0xFFFFu));
+    s.p1 = a.records + ((unsigned int)(first + lane + 32) * a.chunk + (w1 & 0xFFFFu));
+    return s;
+}
+
+__device__ __forceinline__ void load_ahead(const Pieces& s, unsigned long long (&x0)[GATHER_AHEAD],
+                                           unsigned long long (&x1)[GATHER_AHEAD]) {
+    #pragma unroll
+    for (int u = 0; u < GATHER_AHEAD; ++u) {
+        x0[u] = (unsigned int)u < s.len0 ? __ldg(s.p0 + u) : 0ull;
+        x1[u] = (unsigned int)u < s.len1 ? __ldg(s.p1 + u) : 0ull;
     }
-    __syncthreads();
+}
 
-    // ---- accumulate: one update per request at (row, R-1)
-    auto add_record = [&](unsigned long long rec) {
-        const uint32_t rem = (uint32_t)(rec & PRE_FIELD_MAX);
-        const uint32_t B = (uint32_t)((rec >> PRE_FIELD_BITS) & PRE_FIELD_MAX);
-        const int local = (int)(rec >> (2 * PRE_FIELD_BITS));
-        const uint32_t R = rem < (uint32_t)H ? rem : (uint32_t)H;
-        const int c = local * sh.hp + (int)R - 1;
-        uint32_t* w = reinterpret_cast<uint32_t*>(cl + cell_slot(c));
-        atomicAdd(w + 1, 1u);
-        const uint32_t old = atomicAdd(w, B);
-        if (old + B < old) { atomicAdd(&hi[c], 1u); any_hi = 1; }  // exactly one thread sees each wrap
-        if (rem > (uint32_t)H) atomicAdd(&excess[local], (unsigned long long)(rem - (uint32_t)H));
-    };
-    if (chunk_off != nullptr) {
-        const unsigned int* o0 = chunk_off + (size_t)tile * NC;
-        const unsigned int* o1 = o0 + NC;
-        // A tile has a few records per chunk (about n / (tiles * chunks)): take up to four with
-        // independent loads, then whatever is left one by one.
-        for (int ch = tid; ch < NC; ch += TILE_THREADS) {
-            const unsigned int a = o0[ch], b = o1[ch];
-            const unsigned long long* src = records + (size_t)ch * chunk + a;
-            const unsigned int len = b - a;
-            unsigned long long rec[4];
-            #pragma unroll
-            for (int u = 0; u < 4; ++u) rec[u] = (unsigned int)u < len ? src[u] : 0ull;
-            #pragma unroll
-            for (int u = 0; u < 4; ++u) if ((unsigned int)u < len) add_record(rec[u]);
-            for (unsigned int r = 4; r < len; ++r) add_record(src[r]);
-        }
+// f(record) for the records of one trip: the loaded ones, then up to the eighth of each piece
+// lane by lane, and what lies beyond (a skewed or instance-ordered table) with the whole warp.
+template <class F>
+__device__ __forceinline__ void apply_pieces(const Pieces& s, const unsigned long long (&x0)[GATHER_AHEAD],
+                                             const unsigned long long (&x1)[GATHER_AHEAD], F f) {
+    const int lane = threadIdx.x & 31;
+    #pragma unroll
+    for (int u = 0; u < GATHER_AHEAD; ++u) {
+        if ((unsigned int)u < s.len0) f(x0[u]);
+        if ((unsigned int)u < s.len1) f(x1[u]);
+    }
+    const unsigned int near0 = s.len0 < 8u ? s.len0 : 8u, near1 = s.len1 < 8u ? s.len1 : 8u;
+    for (unsigned int u = GATHER_AHEAD; u < near0; ++u) f(__ldg(s.p0 + u));
+    for (unsigned int u = GATHER_AHEAD; u < near1; ++u) f(__ldg(s.p1 + u));
+    unsigned int long0 = __ballot_sync(0xffffffffu, s.len0 > 8u);
+    unsigned int long1 = __ballot_sync(0xffffffffu, s.len1 > 8u);
+    while (long0 | long1) {
+        const bool first = long0 != 0;
+        const int src = __ffs(first ? long0 : long1) - 1;
+        if (first) long0 &= long0 - 1; else long1 &= long1 - 1;
+        const unsigned long long pp =
+            __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(first ? s.p0 : s.p1), src);
+        const unsigned int ll = __shfl_sync(0xffffffffu, first ? s.len0 : s.len1, src);
+        const unsigned long long* p = reinterpret_cast<const unsigned long long*>(pp);
+        for (unsigned int u = 8u + lane; u < ll; u += 32) f(__ldg(p + u));
+    }
+}
+
+// Where this thread's run is: a warp serves one 32-run piece of a row, or several short rows.
+struct RunPlace { int row, q, piece, sub; unsigned int seg_mask; };
+
+__device__ __forceinline__ RunPlace run_place(const TileGeom& g) {
+    RunPlace p;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (g.W == 32) {
+        p.row = warp / g.cpw; p.piece = warp - p.row * g.cpw; p.q = p.piece * 32 + lane;
+        p.sub = lane; p.seg_mask = 0xffffffffu;
     } else {
-        const unsigned int rec0 = bin_base[tile];
-        const unsigned int rec1 = rec0 + bin_cursor[tile];
-        for (unsigned int r = rec0 + tid; r < rec1; r += TILE_THREADS) add_record(records[r]);
+        p.row = warp * g.rpw + (lane >> g.w_shift); p.piece = 0; p.q = lane & (g.W - 1);
+        p.sub = p.q; p.seg_mask = ((1u << g.W) - 1u) << (lane & ~(g.W - 1));
     }
-    __syncthreads();
-    if (chunk_off == nullptr && tid == 0) { bin_cursor[tile] = 0; bin_count[tile] = 0; }  // for the next call
-    const bool with_hi = any_hi != 0;
+    return p;
+}
 
-    // ---- phase 1: totals of every run
-    for (int run = tid; run < n_runs; run += TILE_THREADS) {
-        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(cl + run * (RUN + 2));
-        const int j0 = (run % sh.rpr) * RUN;
-        uint32_t tn = 0;
-        unsigned long long ts = 0, tw = 0;
-        #pragma unroll
-        for (int i = 0; i < RUN / 2; ++i) {
-            const ulonglong2 v = src[i];
-            const uint32_t n0 = (uint32_t)(v.x >> 32), n1 = (uint32_t)(v.y >> 32);
-            tn += n0 + n1;
-            ts += (v.x & 0xffffffffull) + (v.y & 0xffffffffull);
-            tw += (unsigned long long)n0 * (uint32_t)(j0 + 2 * i + 1) + (unsigned long long)n1 * (uint32_t)(j0 + 2 * i + 2);
-        }
-        if (with_hi) {
-            for (int k = 0; k < RUN; ++k) ts += (unsigned long long)hi[run * RUN + k] << 32;
-        }
-        run_n[run] = tn; run_s[run] = ts; run_w[run] = tw;
+// Sum of v over the lanes of a row piece (v < 2^31 each; the sum may need 37 bits).
+__device__ __forceinline__ unsigned long long piece_sum(unsigned int v, unsigned int seg_mask) {
+    const unsigned int lo = __reduce_add_sync(seg_mask, v & 0xFFFFu);
+    const unsigned int hi = __reduce_add_sync(seg_mask, v >> 16);
+    return ((unsigned long long)hi << 16) + lo;
+}
+
+// The scan of one tile in 32 bits; results overwrite the cell words (int64 map values).
+__device__ __forceinline__ void tile_scan_narrow(const TileArgs& a, int rows, unsigned char* cells,
+                                                 unsigned long long* cur, unsigned int* piece_n,
+                                                 unsigned int* piece_s) {
+    const TileGeom& g = a.g;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const RunPlace at = run_place(g);
+    const bool valid = at.row < rows && at.q < g.rpr;
+    const unsigned int j0 = (unsigned int)at.q * RUN;
+    const unsigned int run = (unsigned int)(at.row * g.rpr + at.q);
+    unsigned char* mine = cells + ((size_t)run << 7);
+    const unsigned int sw = (run & 7u) << 4;          // piece i of the run lies at byte (i*16) ^ sw
+
+    uint4 v[RUN / 2];     // {sum, count, sum, count} of two cells
+    #pragma unroll
+    for (int i = 0; i < RUN / 2; ++i)
+        v[i] = valid ? *reinterpret_cast<const uint4*>(mine + ((i * 16) ^ sw)) : make_uint4(0, 0, 0, 0);
+    unsigned int tn = 0, ts = 0;
+    #pragma unroll
+    for (int i = 0; i < RUN / 2; ++i) { ts += v[i].x + v[i].z; tn += v[i].y + v[i].w; }
+
+    // suffix sums over the runs of the piece: what lies above this run
+    unsigned int xn = tn, xs = ts;
+    for (int off = 1; off < g.W; off <<= 1) {
+        const unsigned int yn = __shfl_down_sync(0xffffffffu, xn, off, g.W);
+        const unsigned int ys = __shfl_down_sync(0xffffffffu, xs, off, g.W);
+        if (at.sub + off < g.W) { xn += yn; xs += ys; }
     }
-    __syncthreads();
-
-    // ---- phase 2: suffix over the runs of each row, 32 runs per warp task
-    for (int task = warp; task < rows * sh.cpw; task += TILE_WARPS) {
-        const int row = task / sh.cpw, k = task - row * sh.cpw;
-        const int q = k * 32 + lane;
-        const bool valid = q < sh.rpr;
-        const int run = row * sh.rpr + q;
-        const uint32_t n = valid ? run_n[run] : 0u;
-        const unsigned long long s = valid ? run_s[run] : 0ull;
-        unsigned long long w = valid ? run_w[run] : 0ull;
-        uint32_t xn = n;
-        unsigned long long xs = s;
-        #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t yn = __shfl_down_sync(0xffffffffu, xn, off);
-            const unsigned long long ys = __shfl_down_sync(0xffffffffu, xs, off);
-            if (lane + off < 32) { xn += yn; xs += ys; }
-            w += __shfl_xor_sync(0xffffffffu, w, off);
-        }
-        if (valid) { run_n[run] = xn - n; run_s[run] = xs - s; }  // what lies above, inside the chunk
-        if (lane == 0) {
-            chk_n[task] = xn; chk_s[task] = xs;
-            // sum over j of N[j] = sum over requests of R: each request is counted on R steps
-            if (w) atomicAdd(&sum_n[row], w);
+    unsigned int N = xn - tn, A = xs - ts;
+    if (g.cpw > 1) {     // the same for every thread of the block
+        if (lane == 0) { piece_n[warp] = xn; piece_s[warp] = xs; }
+        __syncthreads();
+        for (int kk = at.piece + 1; kk < g.cpw; ++kk) {
+            N += piece_n[at.row * g.cpw + kk];
+            A += piece_s[at.row * g.cpw + kk];
         }
     }
-    __syncthreads();
+    // from the run's last cell down: N[j], A[j], c[j] = A[j] + j * N[j]
+    unsigned int sn = 0;
+    #pragma unroll
+    for (int i = RUN / 2 - 1; i >= 0; --i) {
+        uint4 o;
+        N += v[i].w; A += v[i].z; sn += N;
+        o.z = A + N * (j0 + 2 * i + 1); o.w = 0;
+        N += v[i].y; A += v[i].x; sn += N;
+        o.x = A + N * (j0 + 2 * i); o.y = 0;
+        if (valid) *reinterpret_cast<uint4*>(mine + ((i * 16) ^ sw)) = o;
+    }
+    // sum over j of N[j] = sum over the row's requests of R: each is counted on R steps
+    const unsigned long long sum_n = piece_sum(sn, at.seg_mask);
+    if (at.sub == 0 && at.row < rows && sum_n) atomicAdd(&cur[at.row], sum_n);
+}
 
-    // ---- phase 3: every run from its last cell down; results overwrite the cell words
-    for (int run = tid; run < n_runs; run += TILE_THREADS) {
-        const int row = run / sh.rpr, q = run - row * sh.rpr;
-        const int k = q >> 5;
-        uint32_t N = run_n[run];
-        unsigned long long A = run_s[run];
-        for (int kk = k + 1; kk < sh.cpw; ++kk) { N += chk_n[row * sh.cpw + kk]; A += chk_s[row * sh.cpw + kk]; }
-        ulonglong2* io = reinterpret_cast<ulonglong2*>(cl + run * (RUN + 2));
-        const int j0 = q * RUN;
-        #pragma unroll
-        for (int i = RUN / 2 - 1; i >= 0; --i) {
-            const ulonglong2 v = io[i];
-            unsigned long long s1 = v.y & 0xffffffffull, s0 = v.x & 0xffffffffull;
-            if (with_hi) {
-                s1 |= (unsigned long long)hi[run * RUN + 2 * i + 1] << 32;
-                s0 |= (unsigned long long)hi[run * RUN + 2 * i] << 32;
+// The same in 64 bits, with the sums of B in the tile's rows of `curves`; writes the rows itself.
+__device__ __forceinline__ void tile_scan_wide(const TileArgs& a, int row0, int rows, const unsigned char* cells,
+                                               unsigned long long* cur, unsigned int* piece_n,
+                                               unsigned long long* piece_s) {
+    const TileGeom& g = a.g;
+    const int H = a.sh.H;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const RunPlace at = run_place(g);
+    const bool valid = at.row < rows && at.q < g.rpr;
+    const int j0 = at.q * RUN;
+    const unsigned int c0 = (unsigned int)(at.row * g.rpr + at.q) * RUN;     // first cell of the run
+    unsigned long long* grow = reinterpret_cast<unsigned long long*>(a.curves) + (size_t)(row0 + at.row) * H;
+    auto count_at = [&](int k) { return *reinterpret_cast<const unsigned int*>(cells + cell_bytes(c0 + k) + 4); };
+
+    unsigned int tn = 0;
+    unsigned long long ts = 0;
+    if (valid) {
+        for (int k = 0; k < RUN; ++k) {
+            if (j0 + k < H) { tn += count_at(k); ts += __ldcg(grow + j0 + k); }
+        }
+    }
+    unsigned int xn = tn;
+    unsigned long long xs = ts;
+    for (int off = 1; off < g.W; off <<= 1) {
+        const unsigned int yn = __shfl_down_sync(0xffffffffu, xn, off, g.W);
+        const unsigned long long ys = __shfl_down_sync(0xffffffffu, xs, off, g.W);
+        if (at.sub + off < g.W) { xn += yn; xs += ys; }
+    }
+    unsigned int N = xn - tn;
+    unsigned long long A = xs - ts;
+    if (g.cpw > 1) {
+        if (lane == 0) { piece_n[warp] = xn; piece_s[warp] = xs; }
+        __syncthreads();
+        for (int kk = at.piece + 1; kk < g.cpw; ++kk) {
+            N += piece_n[at.row * g.cpw + kk];
+            A += piece_s[at.row * g.cpw + kk];
+        }
+    }
+    unsigned long long sum_n = 0;
+    if (valid) {
+        for (int k = RUN - 1; k >= 0; --k) {
+            if (j0 + k < H) {
+                N += count_at(k);
+                A += __ldcg(grow + j0 + k);
+                sum_n += N;
+                grow[j0 + k] = A + (unsigned long long)N * (unsigned int)(j0 + k);
             }
-            ulonglong2 o;
-            N += (uint32_t)(v.y >> 32); A += s1;
-            o.y = A + (unsigned long long)(uint32_t)(j0 + 2 * i + 1) * N;
-            N += (uint32_t)(v.x >> 32); A += s0;
-            o.x = A + (unsigned long long)(uint32_t)(j0 + 2 * i) * N;
-            io[i] = o;
         }
     }
-    __syncthreads();
+    for (int off = g.W >> 1; off > 0; off >>= 1) sum_n += __shfl_down_sync(0xffffffffu, sum_n, off, g.W);
+    if (at.sub == 0 && at.row < rows && sum_n) atomicAdd(&cur[at.row], sum_n);
+}
 
-    // ---- phase 4: copy the rows out with consecutive lanes on consecutive 16 bytes
-    {
-        const int half = sh.hp >> 1;  // cell pairs per padded row
-        const int total = rows * half;
-        const bool vec_gl = (H & 1) == 0;
-        const int shift = (half & (half - 1)) == 0 ? 31 - __clz(half) : -1;  // log2 when a power of two
-        for (int p = tid; p < total; p += TILE_THREADS) {
-            const int row = shift >= 0 ? p >> shift : p / half;
-            const int j = (p - row * half) << 1;
-            if (j < H) {
-                const int c = row * sh.hp + j;
-                const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(cl + cell_slot(c));
-                int64_t* dst = curves + ((size_t)(row0 + row) * H + j);
-                if (vec_gl) {
-                    *reinterpret_cast<ulonglong2*>(dst) = v;
+// One thread: bulk tensor stores of a finished tile (runs [run0, run0 + n_runs) of the map).
+__device__ __forceinline__ void store_tile_tma(const CUtensorMap* map, const unsigned char* cells, int run0, int n_runs) {
+    for (int r = 0; r < n_runs; r += TMA_BOX_RUNS) {
+        const unsigned int src = (unsigned int)__cvta_generic_to_shared(cells + ((size_t)r << 7));
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                     :: "l"(map), "r"(0), "r"(run0 + r), "r"(src) : "memory");
+    }
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+__global__ void __maxnreg__(80)
+pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
+    extern __shared__ unsigned char smem_raw[];
+    const TileGeom& g = a.g;
+    const int H = a.sh.H, T = 1 << a.sh.tile_shift, hp = a.sh.hp, n_tiles = a.sh.n_tiles;
+    const int nwarps = blockDim.x >> 5;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    // carve: cell buffers (1024-byte aligned: the swizzle pattern repeats every 1024 bytes), backlog
+    // sums, piece sums, piece counts
+    const unsigned int raw = (unsigned int)__cvta_generic_to_shared(smem_raw);
+    unsigned char* cells0 = smem_raw + ((1024u - (raw & 1023u)) & 1023u);
+    const size_t buffer_bytes = (size_t)a.buffer_runs << 7;
+    unsigned long long* cur = reinterpret_cast<unsigned long long*>(cells0 + TILE_BUFFERS * buffer_bytes);   // [T]
+    unsigned long long* piece_s = cur + T;                                                                   // [nwarps]
+    unsigned int* piece_n = reinterpret_cast<unsigned int*>(piece_s + nwarps);                               // [nwarps]
+    __shared__ unsigned int tile_records, tile_max_b, table_max_b;
+
+    const bool fast = a.chunk_off != nullptr;
+    const bool tma = a.use_tma != 0;
+    const int trip = nwarps * 64;                 // chunks the block covers in one trip
+    const int first = warp * 64;                  // this warp's chunks in trip 0
+
+    // ---- once: an upper bound of every B of the table (the largest of the chunks' maxima)
+    if (tid == 0) table_max_b = 0;
+    __syncthreads();
+    if (fast) {
+        unsigned int m = 0;
+        for (int c = tid; c < a.NC; c += nthr) { const unsigned int x = __ldg(a.chunk_max + c); m = x > m ? x : m; }
+        m = __reduce_max_sync(0xffffffffu, m);
+        if (lane == 0 && m) atomicMax(&table_max_b, m);
+    }
+
+    unsigned int w0 = 0, w1 = 0;                  // offsets of this lane's two chunks, trip 0, next tile
+    if (fast) load_offsets(a, blockIdx.x, first, w0, w1);
+
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+        unsigned char* cells = cells0 + (it & (TILE_BUFFERS - 1)) * buffer_bytes;
+        const int row0 = tile << a.sh.tile_shift;
+        const int rows = (a.sh.I - row0) < T ? (a.sh.I - row0) : T;
+
+        // ---- look ahead: this tile's first records, the next tile's offsets, the backlog beyond the window
+        Pieces s;
+        unsigned long long x0[GATHER_AHEAD], x1[GATHER_AHEAD];
+        if (fast) {
+            s = pieces_of(a, first, w0, w1);
+            load_ahead(s, x0, x1);
+            load_offsets(a, tile + gridDim.x, first, w0, w1);
+        }
+        const unsigned long long beyond = tid < rows ? a.excess[row0 + tid] : 0ull;
+
+        // ---- the cell buffer is free once the store of the tile before the last has read it
+        if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(TILE_BUFFERS - 1) : "memory");
+        __syncthreads();
+        {
+            uint4* z = reinterpret_cast<uint4*>(cells);
+            const int nz = a.buffer_runs << 3;
+            for (int i = tid; i < nz; i += nthr) z[i] = make_uint4(0, 0, 0, 0);
+            for (int i = tid; i < T; i += nthr) cur[i] = 0ull;
+            if (tid == 0) { tile_records = 0; tile_max_b = 0; }
+        }
+        __syncthreads();
+
+        // ---- accumulate: one update per request at (row, R-1)
+        unsigned int cnt = 0, max_b = 0;
+        auto add = [&](unsigned long long rec) {
+            unsigned int* w = reinterpret_cast<unsigned int*>(cells + (unsigned int)(rec >> 32));
+            atomicAdd(w, (unsigned int)rec);
+            atomicAdd(w + 1, 1u);
+        };
+        if (fast) {
+            cnt = s.len0 + s.len1;
+            apply_pieces(s, x0, x1, add);
+            for (int base = trip; base < a.NC; base += trip) {      // tables of more than `trip` chunks
+                unsigned int v0, v1;
+                load_offsets(a, tile, base + first, v0, v1);
+                const Pieces more = pieces_of(a, base + first, v0, v1);
+                unsigned long long y0[GATHER_AHEAD], y1[GATHER_AHEAD];
+                load_ahead(more, y0, y1);
+                cnt += more.len0 + more.len1;
+                apply_pieces(more, y0, y1, add);
+            }
+        } else {
+            const unsigned int rec0 = a.bin_base[tile];
+            const unsigned int rec1 = rec0 + a.bin_cursor[tile];
+            for (unsigned int r = rec0 + tid; r < rec1; r += nthr) {
+                const unsigned long long rec = a.records[r];
+                const unsigned int b = (unsigned int)rec;
+                max_b = b > max_b ? b : max_b;
+                ++cnt;
+                add(rec);
+            }
+            max_b = __reduce_max_sync(0xffffffffu, max_b);
+            if (lane == 0 && max_b) atomicMax(&tile_max_b, max_b);
+        }
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (lane == 0 && cnt) atomicAdd(&tile_records, cnt);
+        __syncthreads();
+        const unsigned int largest = fast ? table_max_b : tile_max_b;
+        const unsigned long long bound =
+            (unsigned long long)tile_records * ((largest > 32u ? largest : 32u) + (unsigned long long)H);
+
+        if (bound < (1ull << 32)) {
+            tile_scan_narrow(a, rows, cells, cur, piece_n, reinterpret_cast<unsigned int*>(piece_s));
+            if (tma) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stores above, for the copy unit
+                __syncthreads();
+                if (tid == 0) store_tile_tma(&out_map, cells, tile * (T * g.rpr), T * g.rpr);
+            } else {
+                __syncthreads();
+                // consecutive lanes on consecutive 16 bytes: the pair p of cells of the tile lies
+                // at 16-byte word p ^ ((p >> 3) & 7) of the buffer
+                const int half = hp >> 1;               // cell pairs per padded row
+                const int total = rows * half;
+                const uint4* src = reinterpret_cast<const uint4*>(cells);
+                if (hp == H) {
+                    ulonglong2* dst = reinterpret_cast<ulonglong2*>(a.curves + (size_t)row0 * H);
+                    for (int p = tid; p < total; p += nthr) {
+                        const uint4 v = src[p ^ ((p >> 3) & 7)];
+                        dst[p] = make_ulonglong2(v.x, v.z);
+                    }
                 } else {
-                    dst[0] = (int64_t)v.x;
-                    if (j + 1 < H) dst[1] = (int64_t)v.y;
+                    const bool vec_gl = (H & 1) == 0;
+                    for (int p = tid; p < total; p += nthr) {
+                        const int row = p / half;
+                        const int j = (p - row * half) << 1;
+                        if (j < H) {
+                            const uint4 v = src[p ^ ((p >> 3) & 7)];
+                            int64_t* dst = a.curves + ((size_t)(row0 + row) * H + j);
+                            if (vec_gl) {
+                                *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(v.x, v.z);
+                            } else {
+                                dst[0] = (int64_t)v.x;
+                                if (j + 1 < H) dst[1] = (int64_t)v.z;
+                            }
+                        }
+                    }
                 }
             }
+        } else {
+            // ---- wide mode: start over with the sums of B in the tile's rows of `curves`
+            __syncthreads();
+            {
+                uint4* z = reinterpret_cast<uint4*>(cells);
+                const int nz = a.buffer_runs << 3;
+                for (int i = tid; i < nz; i += nthr) z[i] = make_uint4(0, 0, 0, 0);
+            }
+            unsigned long long* gsum = reinterpret_cast<unsigned long long*>(a.curves) + (size_t)row0 * H;
+            for (int i = tid; i < rows * H; i += nthr) gsum[i] = 0ull;
+            __threadfence();
+            __syncthreads();
+            auto add_wide = [&](unsigned long long rec) {
+                const unsigned int at = (unsigned int)(rec >> 32);
+                atomicAdd(reinterpret_cast<unsigned int*>(cells + at) + 1, 1u);
+                const unsigned int run = at >> 7;
+                const unsigned int k = ((((at >> 4) & 7u) ^ (run & 7u)) << 1) | ((at >> 3) & 1u);
+                const unsigned int c = (run << 4) | k;                          // cell index in the padded tile
+                const unsigned int local = c / (unsigned int)hp;
+                atomicAdd(gsum + (size_t)local * H + (c - local * hp), (unsigned long long)(unsigned int)rec);
+            };
+            if (fast) {
+                for (int base = 0; base < a.NC; base += trip) {
+                    unsigned int v0, v1;
+                    load_offsets(a, tile, base + first, v0, v1);
+                    const Pieces more = pieces_of(a, base + first, v0, v1);
+                    unsigned long long y0[GATHER_AHEAD], y1[GATHER_AHEAD];
+                    load_ahead(more, y0, y1);
+                    apply_pieces(more, y0, y1, add_wide);
+                }
+            } else {
+                const unsigned int rec0 = a.bin_base[tile];
+                const unsigned int rec1 = rec0 + a.bin_cursor[tile];
+                for (unsigned int r = rec0 + tid; r < rec1; r += nthr) add_wide(a.records[r]);
+            }
+            __threadfence();
+            __syncthreads();
+            tile_scan_wide(a, row0, rows, cells, cur, piece_n, piece_s);
+            __syncthreads();
+            // an empty group keeps "one group per tile", which the wait at the top counts on
+            if (tma && tid == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
+        // current_d = sum over j of N[j] + what lies beyond the window (left there by the first
+        // pass; cleared for the next call).  cur[] is complete: a barrier followed the scan.
+        if (tid < rows) {
+            a.current_d[row0 + tid] = (int64_t)(cur[tid] + beyond);
+            if (beyond) a.excess[row0 + tid] = 0ull;
+        }
+        if (!fast && tid == 0) { a.bin_cursor[tile] = 0; a.bin_count[tile] = 0; }   // for the next call
     }
-    for (int i = tid; i < rows; i += TILE_THREADS) current_d[row0 + i] = (int64_t)(sum_n[i] + excess[i]);
+    // shared memory must outlive the copy unit's reads of it
+    if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
 }  // namespace
 
-size_t pre_tile_smem_bytes(int tile_rows, int horizon) {
-    const TileShape sh = tile_shape(horizon);
-    const size_t cells = (size_t)tile_rows * sh.hp;
-    const size_t runs = (size_t)tile_rows * sh.rpr;
-    const size_t chunks = (size_t)tile_rows * sh.cpw;
-    return (cells + cells / 8) * 8 + runs * (8 + 8 + 4) + chunks * (8 + 4) + (size_t)tile_rows * 16 + cells * 4;
+// ---------------------------------------------------------------------------------------
+// Host side.
+
+static TileArgs tile_args(int I, int H, int T) {
+    TileArgs a;
+    a.g = tile_geom(H);
+    a.sh.I = I; a.sh.H = H; a.sh.rpr = a.g.rpr; a.sh.hp = a.g.rpr * RUN;
+    a.sh.tile_shift = 0;
+    while ((1 << a.sh.tile_shift) < T) ++a.sh.tile_shift;
+    a.sh.n_tiles = (I + T - 1) / T;
+    a.records = nullptr; a.chunk_off = nullptr; a.chunk_max = nullptr; a.NC = 0; a.chunk = 0;
+    a.bin_base = nullptr; a.bin_cursor = nullptr; a.bin_count = nullptr;
+    a.excess = nullptr; a.curves = nullptr; a.current_d = nullptr;
+    a.buffer_runs = (T * a.g.rpr + 7) & ~7;
+    a.use_tma = 0;
+    return a;
 }
 
+size_t pre_tile_smem_bytes(int tile_rows, int horizon) {
+    const TileGeom g = tile_geom(horizon);
+    const size_t warps = (size_t)tile_warps(tile_rows, g);
+    const size_t buffer = (size_t)((tile_rows * g.rpr + 7) & ~7) * 128;
+    // alignment slack, cell buffers, backlog sums, piece sums, piece counts
+    return 1024 + TILE_BUFFERS * buffer + (size_t)tile_rows * 8 + warps * 12 + 16;
+}
+
+int pre_tile_threads(int tile_rows, int horizon) { return 32 * tile_warps(tile_rows, tile_geom(horizon)); }
+
+// Rows per tile: a power of two, about eight warps of runs, but several tiles per SM when the
+// number of instances allows it.
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm) {
-    const TileShape sh = tile_shape(horizon);
-    int t = 4096 / sh.hp;                       // about 4096 cells (16 per thread) per tile
+    const TileGeom g = tile_geom(horizon);
+    int t = g.rpr >= 32 ? 8 / g.cpw : 8 * g.rpw;
     if (t < 1) t = 1;
     if (t > PRE_MAX_TILE_ROWS) t = PRE_MAX_TILE_ROWS;
-    int by_grid = n_instances / (8 * n_sm);     // but keep the grid at several blocks per SM
-    if (by_grid < 1) by_grid = 1;
-    return t < by_grid ? t : by_grid;
+    int p = 1;
+    while (p * 2 <= t) p *= 2;
+    while (p > 1 && n_instances / p < 8 * n_sm) p >>= 1;
+    return p;
 }
 
-// How the table is cut into chunks: enough chunks that each fits the staging buffer, and, when
-// the table allows it, as many as the GPU runs blocks at once (`slots`), so that the sort is a
-// single wave; never more than `max_chunks` (the width of the offset table).
-static void sort_geometry(int64_t n, int slots, int max_chunks, int* n_chunks, int64_t* chunk, int* staged) {
+// Blocks of the persistent tile kernel: as many as are resident at once, at most one per tile.
+int pre_tile_grid(int tile_rows, int horizon, int n_tiles, int n_sm) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pre_tile_build, pre_tile_threads(tile_rows, horizon),
+                                                      pre_tile_smem_bytes(tile_rows, horizon)) != cudaSuccess ||
+        per_sm < 1)
+        per_sm = 1;
+    const long long resident = (long long)per_sm * n_sm;
+    return (int)(n_tiles < resident ? n_tiles : resident);
+}
+
+// The map as a matrix of runs for the copy unit: [I * H/16 runs][16 int64], stored from
+// shared memory in boxes of `box_runs` runs with the 128-byte swizzle.  Only when a row is a
+// whole number of runs and a tile a whole number of boxes; otherwise the kernel stores with
+// ordinary instructions.  The encoder is a driver entry point, fetched through the runtime so
+// that the library does not link against the driver.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static encode_tiled_fn tensor_map_encoder() {
+    static encode_tiled_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+static bool make_out_map(CUtensorMap* map, int64_t* curves, int I, int H, int T) {
+    memset(map, 0, sizeof(*map));
+    if (H % RUN != 0) return false;
+    const int runs_per_tile = T * (H / RUN);
+    if (runs_per_tile > TMA_BOX_RUNS && runs_per_tile % TMA_BOX_RUNS != 0) return false;
+    encode_tiled_fn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)RUN, (cuuint64_t)I * (cuuint64_t)(H / RUN)};
+    const cuuint64_t strides[1] = {(cuuint64_t)RUN * sizeof(int64_t)};
+    const cuuint32_t box[2] = {(cuuint32_t)RUN, (cuuint32_t)(runs_per_tile < TMA_BOX_RUNS ? runs_per_tile : TMA_BOX_RUNS)};
+    const cuuint32_t elem[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_INT64, 2, curves, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// How the table is cut into chunks: no chunk above SORT_CHUNK rows, and, when the table allows
+// it, as many chunks as the GPU runs blocks at once (`slots`) but none below ~1024 rows.
+// Returns false when the table needs more than `max_chunks` chunks.
+static bool sort_geometry(int64_t n, int slots, int max_chunks, int* n_chunks, int64_t* chunk) {
     int64_t nc = (n + SORT_CHUNK - 1) / SORT_CHUNK;
-    int64_t wave = (n + 1023) / 1024;            // but no chunk below ~1024 requests
+    if (nc > max_chunks) return false;
+    int64_t wave = (n + 1023) / 1024;
     if (wave > slots) wave = slots;
     if (nc < wave) nc = wave;
     if (nc > max_chunks) nc = max_chunks;
@@ -486,15 +869,23 @@ static void sort_geometry(int64_t n, int slots, int max_chunks, int* n_chunks, i
     if (c < 4) c = 4;
     *n_chunks = (int)nc;
     *chunk = c;
-    *staged = c <= SORT_CHUNK;
+    return true;
 }
 
-static size_t sort_smem_bytes(int n_tiles, int staged) {
-    return (staged ? (size_t)SORT_CHUNK * (8 + 2) : 0) + ((size_t)n_tiles + 1) * 4;
+static size_t sort_smem_bytes(int n_tiles) { return ((size_t)n_tiles + 4) * 4; }
+
+int pre_sort_max_chunks(int64_t max_requests, int n_sm) {
+    int64_t need = (max_requests + SORT_CHUNK - 1) / SORT_CHUNK;
+    int64_t wave = (max_requests + 1023) / 1024;
+    if (wave > 2 * n_sm) wave = 2 * n_sm;
+    if (need < wave) need = wave;
+    if (need > SORT_MAX_CHUNKS) need = SORT_MAX_CHUNKS;
+    return (int)need;
 }
 
-size_t pre_chunk_off_words(int n_tiles) {
-    return n_tiles <= PRE_SMEM_BINS ? ((size_t)n_tiles + 1) * SORT_MAX_CHUNKS : 0;
+// Words of the offset table (n_tiles per chunk) followed by one word per chunk (its largest B).
+size_t pre_chunk_table_words(int n_tiles, int max_chunks) {
+    return n_tiles <= PRE_SMEM_BINS ? ((size_t)n_tiles + 1) * (size_t)max_chunks : 0;
 }
 
 cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
@@ -502,31 +893,35 @@ cudaError_t pre_launch_anticipate(pre_ctx* ctx, const int32_t* prompt, const int
                                   int64_t* curves, int64_t* current_d, cudaStream_t s) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon, T = ctx->tile_rows, nt = ctx->n_tiles;
     const size_t tile_smem = pre_tile_smem_bytes(T, H);
-    if (nt <= PRE_SMEM_BINS) {
-        int nc = 1, staged = 1;
-        int64_t chunk = 4;
-        sort_geometry(n, 3 * ctx->n_sm, SORT_MAX_CHUNKS, &nc, &chunk, &staged);
+    const int tile_threads = pre_tile_threads(T, H);
+    TileArgs a = tile_args(I, H, T);
+    a.records = ctx->d_records; a.excess = ctx->d_excess; a.curves = curves; a.current_d = current_d;
+    CUtensorMap out_map;
+    a.use_tma = make_out_map(&out_map, curves, I, H, T) ? 1 : 0;
+    int nc = 1;
+    int64_t chunk = 4;
+    if (nt <= PRE_SMEM_BINS && sort_geometry(n, 2 * ctx->n_sm, ctx->max_chunks, &nc, &chunk)) {
         // With n == 0 the single chunk is empty: its offsets are all zero and every tile writes zero rows.
-        pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(nt, staged), s>>>(
-            prompt, generated, predicted, instance, n, I, T, nt, chunk, staged, ctx->d_records, ctx->d_chunk_off,
-            ctx->d_status);
-        pre_tile_build<<<nt, TILE_THREADS, tile_smem, s>>>(ctx->d_records, ctx->d_chunk_off, nc, chunk, nullptr,
-                                                         nullptr, nullptr, I, H, T, curves, current_d);
+        unsigned int* chunk_max = ctx->d_chunk_off + (size_t)nt * ctx->max_chunks;
+        pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(nt), s>>>(
+            prompt, generated, predicted, instance, n, a.sh, chunk, ctx->d_records, ctx->d_chunk_off, chunk_max,
+            ctx->d_excess, ctx->d_status);
+        a.chunk_off = ctx->d_chunk_off; a.chunk_max = chunk_max; a.NC = nc; a.chunk = (unsigned int)chunk;
+        pre_tile_build<<<ctx->tile_grid, tile_threads, tile_smem, s>>>(a, out_map);
     } else {
         int grid = (int)((n + BIN_THREADS * 8 - 1) / (BIN_THREADS * 8));
         if (grid > 2 * ctx->n_sm) grid = 2 * ctx->n_sm;
         if (grid < 1) grid = 1;
         if (n > 0) {
-            pre_bin_count<<<grid, BIN_THREADS, 0, s>>>(instance, n, I, T, ctx->d_bin_count);
+            pre_bin_count<<<grid, BIN_THREADS, 0, s>>>(instance, n, I, a.sh.tile_shift, ctx->d_bin_count);
             pre_bin_scan<<<1, 1024, 0, s>>>(ctx->d_bin_count, nt, ctx->d_bin_base);
-            pre_bin_scatter<<<grid, BIN_THREADS, 0, s>>>(prompt, generated, predicted, instance, n, I, T,
+            pre_bin_scatter<<<grid, BIN_THREADS, 0, s>>>(prompt, generated, predicted, instance, n, a.sh,
                                                        ctx->d_bin_base, ctx->d_bin_cursor, ctx->d_records,
-                                                       ctx->d_status);
+                                                       ctx->d_excess, ctx->d_status);
         }
         // With n == 0 the cursors are zero (every build clears them): every tile sees an empty span.
-        pre_tile_build<<<nt, TILE_THREADS, tile_smem, s>>>(ctx->d_records, nullptr, 0, 0, ctx->d_bin_base,
-                                                         ctx->d_bin_cursor, ctx->d_bin_count, I, H, T, curves,
-                                                         current_d);
+        a.bin_base = ctx->d_bin_base; a.bin_cursor = ctx->d_bin_cursor; a.bin_count = ctx->d_bin_count;
+        pre_tile_build<<<ctx->tile_grid, tile_threads, tile_smem, s>>>(a, out_map);
     }
     return cudaGetLastError();
 }
@@ -545,8 +940,11 @@ cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
     if (e != cudaSuccess) return e;
     e = cudaFuncGetAttributes(&attr, pre_tile_build);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                optin - (int)attr.sharedSizeBytes);
+    e = cudaFuncSetAttribute(pre_tile_build, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             optin - (int)attr.sharedSizeBytes);
+    if (e != cudaSuccess) return e;
+    ctx->tile_grid = pre_tile_grid(ctx->tile_rows, ctx->cfg.horizon, ctx->n_tiles, ctx->n_sm);
+    return cudaSuccess;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -558,10 +956,15 @@ cudaError_t pre_anticipate_configure(pre_ctx* ctx) {
 constexpr int PRE_STATIC_MAX_REQUESTS = 262144;   // table rows one call may cover
 constexpr int PRE_STATIC_MAX_TILES = 2048;        // build tiles one call may need
 constexpr int PRE_STATIC_MAX_CHUNKS = 64;          // chunks of at most 4,096 requests
+constexpr int PRE_STATIC_MAX_INSTANCES = 65536;    // rows of the map
 constexpr size_t PRE_STATIC_STATUS_BYTES = 256;
 constexpr size_t PRE_STATIC_OFF_BYTES = (size_t)(PRE_STATIC_MAX_TILES + 1) * PRE_STATIC_MAX_CHUNKS * sizeof(unsigned int);
 constexpr size_t PRE_STATIC_REC_BYTES = (size_t)PRE_STATIC_MAX_REQUESTS * sizeof(unsigned long long);
-constexpr size_t PRE_STATIC_BYTES = PRE_STATIC_STATUS_BYTES + ((PRE_STATIC_OFF_BYTES + 255) & ~(size_t)255) + PRE_STATIC_REC_BYTES;
+constexpr size_t PRE_STATIC_EXCESS_BYTES = (size_t)PRE_STATIC_MAX_INSTANCES * sizeof(unsigned long long);
+constexpr size_t PRE_STATIC_OFF_AT = PRE_STATIC_STATUS_BYTES;
+constexpr size_t PRE_STATIC_REC_AT = PRE_STATIC_OFF_AT + ((PRE_STATIC_OFF_BYTES + 255) & ~(size_t)255);
+constexpr size_t PRE_STATIC_EXCESS_AT = PRE_STATIC_REC_AT + PRE_STATIC_REC_BYTES;
+constexpr size_t PRE_STATIC_BYTES = PRE_STATIC_EXCESS_AT + PRE_STATIC_EXCESS_BYTES;
 
 static __device__ __align__(256) unsigned char pre_static_scratch[PRE_STATIC_BYTES];
 
@@ -621,7 +1024,7 @@ extern "C" int pre_anticipate_static(int32_t n_instances, int32_t horizon, const
         (reinterpret_cast<uintptr_t>(d_generated) & 3) || (reinterpret_cast<uintptr_t>(d_predicted) & 3) ||
         (reinterpret_cast<uintptr_t>(d_instance) & 3))
         return PRE_EINVAL;
-    if (n_requests > PRE_STATIC_MAX_REQUESTS) return PRE_ESIZE;
+    if (n_requests > PRE_STATIC_MAX_REQUESTS || n_instances > PRE_STATIC_MAX_INSTANCES) return PRE_ESIZE;
 
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess) return PRE_ECUDA;
@@ -635,21 +1038,28 @@ extern "C" int pre_anticipate_static(int32_t n_instances, int32_t horizon, const
     const size_t tile_smem = pre_tile_smem_bytes(T, horizon);
     if (tile_smem > (size_t)st->smem_optin) return PRE_EINVAL;
 
-    int nc = 1, staged = 1;
+    int nc = 1;
     int64_t chunk = 4;
-    sort_geometry(n_requests, 3 * st->n_sm, PRE_STATIC_MAX_CHUNKS, &nc, &chunk, &staged);  // staged: chunk <= 4096
+    if (!sort_geometry(n_requests, 2 * st->n_sm, PRE_STATIC_MAX_CHUNKS, &nc, &chunk)) return PRE_ESIZE;
 
     int* status = d_flags ? d_flags : reinterpret_cast<int*>(st->base);
-    unsigned int* chunk_off = reinterpret_cast<unsigned int*>(st->base + PRE_STATIC_STATUS_BYTES);
-    unsigned long long* records = reinterpret_cast<unsigned long long*>(
-        st->base + PRE_STATIC_STATUS_BYTES + ((PRE_STATIC_OFF_BYTES + 255) & ~(size_t)255));
+    unsigned int* chunk_off = reinterpret_cast<unsigned int*>(st->base + PRE_STATIC_OFF_AT);
+    unsigned int* chunk_max = chunk_off + (size_t)PRE_STATIC_MAX_TILES * PRE_STATIC_MAX_CHUNKS;
+    unsigned long long* records = reinterpret_cast<unsigned long long*>(st->base + PRE_STATIC_REC_AT);
+    unsigned long long* excess = reinterpret_cast<unsigned long long*>(st->base + PRE_STATIC_EXCESS_AT);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // Nothing in the scratch has to start at zero: pre_chunk_sort writes every offset that
+    // Nothing in the scratch has to be cleared here.  pre_chunk_sort writes every offset that
     // pre_tile_build reads, and a record is read only where an offset says one was written.
-    pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(n_tiles, staged), s>>>(
-        d_prompt, d_generated, d_predicted, d_instance, n_requests, n_instances, T, n_tiles, chunk, staged, records,
-        chunk_off, status);
-    pre_tile_build<<<n_tiles, TILE_THREADS, tile_smem, s>>>(records, chunk_off, nc, chunk, nullptr, nullptr, nullptr,
-                                                          n_instances, horizon, T, d_curves, d_current_d);
+    // The per-instance words for what lies beyond the window start as zeros (the array is part of
+    // the library image) and pre_tile_build clears each word again after reading it.
+    TileArgs a = tile_args(n_instances, horizon, T);
+    a.records = records; a.excess = excess; a.curves = d_curves; a.current_d = d_current_d;
+    CUtensorMap out_map;
+    a.use_tma = make_out_map(&out_map, d_curves, n_instances, horizon, T) ? 1 : 0;
+    pre_chunk_sort<<<nc, SORT_THREADS, sort_smem_bytes(n_tiles), s>>>(
+        d_prompt, d_generated, d_predicted, d_instance, n_requests, a.sh, chunk, records, chunk_off, chunk_max, excess,
+        status);
+    a.chunk_off = chunk_off; a.chunk_max = chunk_max; a.NC = nc; a.chunk = (unsigned int)chunk;
+    pre_tile_build<<<pre_tile_grid(T, horizon, n_tiles, st->n_sm), pre_tile_threads(T, horizon), tile_smem, s>>>(a, out_map);
     return cudaGetLastError() == cudaSuccess ? PRE_OK : PRE_ECUDA;
 }

@@ -20,6 +20,7 @@ void release(pre_ctx* c) {
     if (!c) return;
     cudaFree(c->d_status);
     cudaFree(c->d_chunk_off);
+    cudaFree(c->d_excess);
     cudaFree(c->d_bin_count);
     cudaFree(c->d_bin_base);
     cudaFree(c->d_bin_cursor);
@@ -77,8 +78,10 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
         const unsigned int first = 2;
         e = cudaMemcpy(c->d_epoch, &first, sizeof(first), cudaMemcpyHostToDevice);
     }
-    if (e == cudaSuccess && pre_chunk_off_words(c->n_tiles))
-        e = alloc_zero(&c->d_chunk_off, pre_chunk_off_words(c->n_tiles));
+    c->max_chunks = pre_sort_max_chunks(cfg->max_requests, c->n_sm);
+    if (e == cudaSuccess && pre_chunk_table_words(c->n_tiles, c->max_chunks))
+        e = alloc_zero(&c->d_chunk_off, pre_chunk_table_words(c->n_tiles, c->max_chunks));
+    if (e == cudaSuccess) e = alloc_zero(&c->d_excess, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_base, (size_t)c->n_tiles + 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_cursor, (size_t)c->n_tiles);

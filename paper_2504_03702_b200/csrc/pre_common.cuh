@@ -24,6 +24,8 @@ struct pre_ctx {
     int n_sm;
     int tile_rows;       // T: instance rows per build tile
     int n_tiles;         // ceil(I / T)
+    int max_chunks;      // width of the offset table: chunks the sorting pass may cut the table into
+    int tile_grid;       // blocks of the persistent tile kernel
     int route_blocks;    // G: blocks of the persistent routing kernel
     int route_threads;
     size_t route_smem;
@@ -37,7 +39,9 @@ struct pre_ctx {
     int* d_abort;             // routing kernel gives up when set
     unsigned int* d_epoch;    // running exchange counter of the routing kernel (tags of the exchange slots)
     int64_t* d_queue_entry;   // {head, length} of the admission queue as they were when the call was made
-    unsigned int* d_chunk_off;   // [(n_tiles+1) x chunks] where each tile starts inside each sorted chunk
+    unsigned int* d_chunk_off;   // [max_chunks x n_tiles] {start : 16 | length : 16} of each tile inside each
+                                 // sorted chunk, then [max_chunks] the largest B of each chunk
+    unsigned long long* d_excess;   // [I] remaining tokens beyond the window, per instance (zero between calls)
     unsigned int* d_bin_count;   // slow path [n_tiles]   zero between calls
     unsigned int* d_bin_base;    // slow path [n_tiles+1]
     unsigned int* d_bin_cursor;  // slow path [n_tiles]   zero between calls
@@ -76,7 +80,9 @@ cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overlo
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
 size_t pre_tile_smem_bytes(int tile_rows, int horizon);
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm);
-size_t pre_chunk_off_words(int n_tiles);
+int pre_tile_threads(int tile_rows, int horizon);
+int pre_sort_max_chunks(int64_t max_requests, int n_sm);
+size_t pre_chunk_table_words(int n_tiles, int max_chunks);
 cudaError_t pre_anticipate_configure(pre_ctx* ctx);
 
 __device__ __forceinline__ bool pre_request_ok(int32_t P, int32_t g, int32_t D, int32_t inst, int32_t I) {

@@ -73,6 +73,32 @@ def test_anticipate_all_on_one_instance_and_long_requests():
     st.close()
 
 
+def test_anticipate_sums_beyond_32_bits():
+    """Prompts near the field limit: a tile's sum of B passes 2^32, so the build works in 64 bits."""
+    wl = W.make_random(19, 3, 40, 500, 0, max_prompt=2 ** 27, max_output=90)
+    st, ref = both(wl)
+    assert int(ref.curves.max()) > 2 ** 32
+    assert_state_equal(st, ref)
+    wl = W.make_random(20, 70, 2048, 4000, 0, max_prompt=2 ** 27, max_output=5000)
+    wl.instance[:] = wl.instance % 3 + 66           # a ragged last tile, all of it wide
+    st2, ref2 = both(wl)
+    assert_state_equal(st2, ref2)
+    assert st.status() == B.PRE_OK and st2.status() == B.PRE_OK
+    st.close()
+    st2.close()
+
+
+def test_anticipate_table_ordered_by_instance():
+    """A table kept in instance order: every chunk holds long pieces of a few tiles."""
+    wl = W.make_random(21, 64, 256, 60000, 0, max_prompt=3000, max_output=700)
+    order = np.argsort(wl.instance, kind="stable")
+    for name in ("prompt", "generated", "predicted", "instance"):
+        setattr(wl, name, np.ascontiguousarray(getattr(wl, name)[order]))
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    st.close()
+
+
 def test_anticipate_tombstones_and_malformed():
     wl = W.make_random(13, 5, 40, 600, 0)
     wl.generated[::7] = wl.predicted[::7]          # finished: silently ignored
