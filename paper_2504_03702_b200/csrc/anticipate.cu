@@ -163,7 +163,8 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
                const BuildShape sh, int64_t chunk, unsigned long long* __restrict__ records,
                unsigned int* __restrict__ chunk_off, unsigned int* __restrict__ chunk_max,
                unsigned long long* __restrict__ excess, int* __restrict__ status) {
-    extern __shared__ __align__(16) unsigned int hist[];    // [n_tiles + 1], rounded up to whole 16-byte groups
+    extern __shared__ __align__(16) unsigned int hist[];    // [n_tiles + 1], rounded up to whole 16-byte groups;
+                                                             // then the chunk's records in tile order
     __shared__ unsigned int warp_tot[SORT_THREADS / 32];
     __shared__ unsigned int block_max;
 
@@ -288,11 +289,25 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
         my_off[i] = a | ((hist[i + 1] - a) << 16);
     }
     if (tid == 0) chunk_max[ch] = block_max;
-    unsigned long long* out = records + r0;
+    // the records are put in order in shared memory (a scattered store there costs little) and
+    // leave in one bulk copy: scattered 8-byte stores to global memory would each touch a sector
+    unsigned long long* stage = reinterpret_cast<unsigned long long*>(hist + 4 * groups);
     #pragma unroll
     for (int u = 0; u < SORT_SLOTS; ++u)
-        if (tile_of[u] >= 0) out[hist[tile_of[u]] + rank[u]] = rec[u];
+        if (tile_of[u] >= 0) stage[hist[tile_of[u]] + rank[u]] = rec[u];
     if (any_bad) atomicOr(status, PRE_ST_BADREQ);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int bytes = ((hist[n_tiles] + 1u) & ~1u) * 8u;   // whole 16 bytes; the span has room (chunk is even)
+        if (bytes) {
+            const unsigned int src = (unsigned int)__cvta_generic_to_shared(stage);
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         :: "l"(records + r0), "r"(src), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory must outlive the copy
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -302,12 +317,14 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
 // A run of RUN consecutive cells of a row belongs to one thread, which keeps it in registers
 // for the whole scan.  A warp serves 32 consecutive runs of one row, or, when a row has fewer
 // than 32 runs, several rows side by side (W lanes each).  The finished tile, int64 values in
-// the same layout, leaves shared memory in bulk tensor stores issued by one thread while the
-// block already works on its next tile in the second cell buffer.
+// the same layout, leaves shared memory in bulk tensor stores issued by one thread.
 //
-// Latency is hidden by looking ahead: a lane holds the offsets of its two chunks for the next
-// tile a whole tile early, and issues the loads of this tile's records before it waits for
-// the cell buffer and clears it.
+// A tile has a few records in every chunk, each piece somewhere else in memory, so the gather
+// is bound by the number of separate 32-byte sectors it touches: a lane reads its piece in
+// aligned 32-byte windows (one load each).  The first windows of the NEXT tile are copied into
+// a per-thread slot of shared memory asynchronously while this tile is scanned and stored, and
+// the offset word they need is loaded one tile earlier still, so the accumulation of a tile
+// does not wait for global memory.
 //
 // All sums, and the map values themselves, fit 32 bits as long as
 //     (records of the tile) * (max(largest B, 32) + H) < 2^32,
@@ -315,7 +332,7 @@ pre_chunk_sort(const int32_t* __restrict__ prompt, const int32_t* __restrict__ g
 // stay in shared memory, the sums of B are accumulated with 64-bit atomics in the tile's own
 // rows of `curves` (cleared first), and the scan runs in 64 bits.
 constexpr int TILE_MAX_THREADS = 512;
-constexpr int TILE_BUFFERS = 2;
+constexpr int TILE_BUFFERS = 1;
 constexpr int TMA_BOX_RUNS = 256;      // rows (runs of 128 bytes) of one bulk tensor store
 
 struct TileGeom {
@@ -361,68 +378,84 @@ struct TileArgs {
     int use_tma;                       // the tensor map describes `curves` as runs of 128 bytes
 };
 
-constexpr int GATHER_AHEAD = 4;   // records of a chunk's piece that a lane loads before using any
+constexpr int WINDOW = 4;          // records of one 32-byte load
+constexpr int WINDOWS_AHEAD = 2;   // windows of a chunk's piece that a lane loads before using any
+constexpr int WINDOWS_ALONE = 8;   // beyond this many, the whole warp shares a lane's piece
 
-// The pieces of the tile's records that this lane is responsible for in one trip over the
-// chunks: chunk c0 = first + lane and c1 = c0 + 32.
-struct Pieces {
-    const unsigned long long* p0;
-    const unsigned long long* p1;
-    unsigned int len0, len1;
+// This lane's piece of the tile's records in one trip over the chunks (chunk c = first + lane):
+// records [s, s + len) of the chunk's span, read in aligned windows of four starting at `win`.
+struct Piece {
+    const unsigned long long* win;   // 32-byte aligned
+    unsigned int skip;               // records of the first window that belong to the previous tile
+    unsigned int len;
+    unsigned int n_win;
 };
 
-__device__ __forceinline__ void load_offsets(const TileArgs& a, int tile, int first, unsigned int& w0,
-                                             unsigned int& w1) {
-    const int lane = threadIdx.x & 31;
-    const int c0 = first + lane, c1 = c0 + 32;
-    const bool in = tile < a.sh.n_tiles;
-    w0 = in && c0 < a.NC ? __ldg(a.chunk_off + ((unsigned int)c0 * (unsigned int)a.sh.n_tiles + tile)) : 0u;
-    w1 = in && c1 < a.NC ? __ldg(a.chunk_off + ((unsigned int)c1 * (unsigned int)a.sh.n_tiles + tile)) : 0u;
+__device__ __forceinline__ unsigned int load_offset(const TileArgs& a, int tile, int c) {
+    return tile < a.sh.n_tiles && c < a.NC
+               ? __ldg(a.chunk_off + ((unsigned int)c * (unsigned int)a.sh.n_tiles + tile)) : 0u;
 }
 
-__device__ __forceinline__ Pieces pieces_of(const TileArgs& a, int first, unsigned int w0, unsigned int w1) {
-    const int lane = threadIdx.x & 31;
-    Pieces s;
-    s.len0 = w0 >> 16; s.len1 = w1 >> 16;
-    s.p0 = a.records + ((unsigned int)(first + lane) * a.chunk + (w0 & 0xFFFFu));
-    s.p1 = a.records + ((unsigned int)(first + lane + 32) * a.chunk + (w1 & 0xFFFFu));
-    return s;
+__device__ __forceinline__ Piece piece_of(const TileArgs& a, int c, unsigned int w) {
+    Piece p;
+    const unsigned int s = w & 0xFFFFu;
+    p.len = w >> 16;
+    p.skip = s & (WINDOW - 1);
+    p.win = a.records + ((unsigned int)c * a.chunk + (s - p.skip));
+    p.n_win = p.len ? (p.skip + p.len + WINDOW - 1) / WINDOW : 0u;
+    return p;
 }
 
-__device__ __forceinline__ void load_ahead(const Pieces& s, unsigned long long (&x0)[GATHER_AHEAD],
-                                           unsigned long long (&x1)[GATHER_AHEAD]) {
-    #pragma unroll
-    for (int u = 0; u < GATHER_AHEAD; ++u) {
-        x0[u] = (unsigned int)u < s.len0 ? __ldg(s.p0 + u) : 0ull;
-        x1[u] = (unsigned int)u < s.len1 ? __ldg(s.p1 + u) : 0ull;
-    }
+struct Window { unsigned long long r[WINDOW]; };
+
+// One 32-byte load (the span of a chunk starts on a 32-byte boundary and is a whole number of windows).
+__device__ __forceinline__ Window load_window(const unsigned long long* p) {
+    Window x;
+    asm volatile("ld.global.nc.v4.u64 {%0, %1, %2, %3}, [%4];"
+                 : "=l"(x.r[0]), "=l"(x.r[1]), "=l"(x.r[2]), "=l"(x.r[3]) : "l"(p));
+    return x;
 }
 
-// f(record) for the records of one trip: the loaded ones, then up to the eighth of each piece
-// lane by lane, and what lies beyond (a skewed or instance-ordered table) with the whole warp.
+// The same window copied into shared memory behind the thread's back (two 16-byte pieces).
+__device__ __forceinline__ void copy_window_async(unsigned char* dst_shared, const unsigned long long* p) {
+    const unsigned int d = (unsigned int)__cvta_generic_to_shared(dst_shared);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d), "l"(p) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(d + 16u), "l"(p + 2) : "memory");
+}
+
+__device__ __forceinline__ Window read_window(const unsigned char* src_shared) {
+    Window x;
+    const ulonglong2 lo = *reinterpret_cast<const ulonglong2*>(src_shared);
+    const ulonglong2 hi = *reinterpret_cast<const ulonglong2*>(src_shared + 16);
+    x.r[0] = lo.x; x.r[1] = lo.y; x.r[2] = hi.x; x.r[3] = hi.y;
+    return x;
+}
+
+// f(record) for the records of window k of a piece.
 template <class F>
-__device__ __forceinline__ void apply_pieces(const Pieces& s, const unsigned long long (&x0)[GATHER_AHEAD],
-                                             const unsigned long long (&x1)[GATHER_AHEAD], F f) {
-    const int lane = threadIdx.x & 31;
+__device__ __forceinline__ void apply_window(const Window& x, unsigned int k, unsigned int skip, unsigned int len, F f) {
     #pragma unroll
-    for (int u = 0; u < GATHER_AHEAD; ++u) {
-        if ((unsigned int)u < s.len0) f(x0[u]);
-        if ((unsigned int)u < s.len1) f(x1[u]);
-    }
-    const unsigned int near0 = s.len0 < 8u ? s.len0 : 8u, near1 = s.len1 < 8u ? s.len1 : 8u;
-    for (unsigned int u = GATHER_AHEAD; u < near0; ++u) f(__ldg(s.p0 + u));
-    for (unsigned int u = GATHER_AHEAD; u < near1; ++u) f(__ldg(s.p1 + u));
-    unsigned int long0 = __ballot_sync(0xffffffffu, s.len0 > 8u);
-    unsigned int long1 = __ballot_sync(0xffffffffu, s.len1 > 8u);
-    while (long0 | long1) {
-        const bool first = long0 != 0;
-        const int src = __ffs(first ? long0 : long1) - 1;
-        if (first) long0 &= long0 - 1; else long1 &= long1 - 1;
-        const unsigned long long pp =
-            __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(first ? s.p0 : s.p1), src);
-        const unsigned int ll = __shfl_sync(0xffffffffu, first ? s.len0 : s.len1, src);
-        const unsigned long long* p = reinterpret_cast<const unsigned long long*>(pp);
-        for (unsigned int u = 8u + lane; u < ll; u += 32) f(__ldg(p + u));
+    for (int i = 0; i < WINDOW; ++i)
+        if (k * WINDOW + i - skip < len) f(x.r[i]);      // unsigned: also false in front of the piece
+}
+
+// f(record) for what a lane has not loaded ahead: its windows up to WINDOWS_ALONE by itself, and
+// the rest of a long piece (a skewed or instance-ordered table) with all lanes of the warp.
+template <class F>
+__device__ __forceinline__ void apply_rest(const Piece& p, F f) {
+    const int lane = threadIdx.x & 31;
+    const unsigned int alone = p.n_win < (unsigned int)WINDOWS_ALONE ? p.n_win : (unsigned int)WINDOWS_ALONE;
+    for (unsigned int k = WINDOWS_AHEAD; k < alone; ++k) apply_window(load_window(p.win + k * WINDOW), k, p.skip, p.len, f);
+    unsigned int longs = __ballot_sync(0xffffffffu, p.n_win > (unsigned int)WINDOWS_ALONE);
+    while (longs) {
+        const int src = __ffs(longs) - 1;
+        longs &= longs - 1;
+        const unsigned long long* win =
+            reinterpret_cast<const unsigned long long*>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(p.win), src));
+        const unsigned int skip = __shfl_sync(0xffffffffu, p.skip, src);
+        const unsigned int len = __shfl_sync(0xffffffffu, p.len, src);
+        const unsigned int n_win = __shfl_sync(0xffffffffu, p.n_win, src);
+        for (unsigned int k = WINDOWS_ALONE + lane; k < n_win; k += 32) apply_window(load_window(win + k * WINDOW), k, skip, len, f);
     }
 }
 
@@ -565,7 +598,7 @@ __device__ __forceinline__ void store_tile_tma(const CUtensorMap* map, const uns
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-__global__ void __maxnreg__(80)
+__global__ void __launch_bounds__(TILE_MAX_THREADS, 2)
 pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
     extern __shared__ unsigned char smem_raw[];
     const TileGeom& g = a.g;
@@ -580,12 +613,13 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
     unsigned long long* cur = reinterpret_cast<unsigned long long*>(cells0 + TILE_BUFFERS * buffer_bytes);   // [T]
     unsigned long long* piece_s = cur + T;                                                                   // [nwarps]
     unsigned int* piece_n = reinterpret_cast<unsigned int*>(piece_s + nwarps);                               // [nwarps]
+    // [WINDOWS_AHEAD][nthr] windows of 32 bytes: where the next tile's first records arrive
+    unsigned char* stage = reinterpret_cast<unsigned char*>(cur) + (((size_t)T * 8 + (size_t)nwarps * 12 + 31) & ~(size_t)31);
     __shared__ unsigned int tile_records, tile_max_b, table_max_b;
 
     const bool fast = a.chunk_off != nullptr;
     const bool tma = a.use_tma != 0;
-    const int trip = nwarps * 64;                 // chunks the block covers in one trip
-    const int first = warp * 64;                  // this warp's chunks in trip 0
+    const int trip = nthr;                        // chunks the block covers in one trip: one per thread
 
     // ---- once: an upper bound of every B of the table (the largest of the chunks' maxima)
     if (tid == 0) table_max_b = 0;
@@ -597,8 +631,18 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         if (lane == 0 && m) atomicMax(&table_max_b, m);
     }
 
-    unsigned int w0 = 0, w1 = 0;                  // offsets of this lane's two chunks, trip 0, next tile
-    if (fast) load_offsets(a, blockIdx.x, first, w0, w1);
+    // this thread's piece of the block's first tile is on its way; the offset word of the second is loaded
+    Piece mine;
+    unsigned int w = 0;
+    mine.win = a.records; mine.skip = 0; mine.len = 0; mine.n_win = 0;
+    if (fast) {
+        mine = piece_of(a, tid, load_offset(a, blockIdx.x, tid));
+        #pragma unroll
+        for (int k = 0; k < WINDOWS_AHEAD; ++k)
+            if ((unsigned int)k < mine.n_win) copy_window_async(stage + ((size_t)(k * nthr + tid) << 5), mine.win + k * WINDOW);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        w = load_offset(a, blockIdx.x + gridDim.x, tid);
+    }
 
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
@@ -606,14 +650,6 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         const int row0 = tile << a.sh.tile_shift;
         const int rows = (a.sh.I - row0) < T ? (a.sh.I - row0) : T;
 
-        // ---- look ahead: this tile's first records, the next tile's offsets, the backlog beyond the window
-        Pieces s;
-        unsigned long long x0[GATHER_AHEAD], x1[GATHER_AHEAD];
-        if (fast) {
-            s = pieces_of(a, first, w0, w1);
-            load_ahead(s, x0, x1);
-            load_offsets(a, tile + gridDim.x, first, w0, w1);
-        }
         const unsigned long long beyond = tid < rows ? a.excess[row0 + tid] : 0ull;
 
         // ---- the cell buffer is free once the store of the tile before the last has read it
@@ -636,16 +672,21 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
             atomicAdd(w + 1, 1u);
         };
         if (fast) {
-            cnt = s.len0 + s.len1;
-            apply_pieces(s, x0, x1, add);
+            cnt = mine.len;
+            asm volatile("cp.async.wait_all;" ::: "memory");       // this thread's own copies
+            #pragma unroll
+            for (int k = 0; k < WINDOWS_AHEAD; ++k)
+                if ((unsigned int)k < mine.n_win)
+                    apply_window(read_window(stage + ((size_t)(k * nthr + tid) << 5)), k, mine.skip, mine.len, add);
+            apply_rest(mine, add);
             for (int base = trip; base < a.NC; base += trip) {      // tables of more than `trip` chunks
-                unsigned int v0, v1;
-                load_offsets(a, tile, base + first, v0, v1);
-                const Pieces more = pieces_of(a, base + first, v0, v1);
-                unsigned long long y0[GATHER_AHEAD], y1[GATHER_AHEAD];
-                load_ahead(more, y0, y1);
-                cnt += more.len0 + more.len1;
-                apply_pieces(more, y0, y1, add);
+                const Piece more = piece_of(a, base + tid, load_offset(a, tile, base + tid));
+                cnt += more.len;
+                #pragma unroll
+                for (int k = 0; k < WINDOWS_AHEAD; ++k)
+                    if ((unsigned int)k < more.n_win)
+                        apply_window(load_window(more.win + k * WINDOW), k, more.skip, more.len, add);
+                apply_rest(more, add);
             }
         } else {
             const unsigned int rec0 = a.bin_base[tile];
@@ -662,6 +703,16 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         }
         cnt = __reduce_add_sync(0xffffffffu, cnt);
         if (lane == 0 && cnt) atomicAdd(&tile_records, cnt);
+        if (fast) {
+            // look ahead: the next tile's first windows start their way into this thread's slots (it
+            // has read them), and the offset word of the tile after that is loaded
+            mine = piece_of(a, tid, w);
+            #pragma unroll
+            for (int k = 0; k < WINDOWS_AHEAD; ++k)
+                if ((unsigned int)k < mine.n_win) copy_window_async(stage + ((size_t)(k * nthr + tid) << 5), mine.win + k * WINDOW);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            w = load_offset(a, tile + 2 * gridDim.x, tid);
+        }
         __syncthreads();
         const unsigned int largest = fast ? table_max_b : tile_max_b;
         const unsigned long long bound =
@@ -727,12 +778,12 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
             };
             if (fast) {
                 for (int base = 0; base < a.NC; base += trip) {
-                    unsigned int v0, v1;
-                    load_offsets(a, tile, base + first, v0, v1);
-                    const Pieces more = pieces_of(a, base + first, v0, v1);
-                    unsigned long long y0[GATHER_AHEAD], y1[GATHER_AHEAD];
-                    load_ahead(more, y0, y1);
-                    apply_pieces(more, y0, y1, add_wide);
+                    const Piece more = piece_of(a, base + tid, load_offset(a, tile, base + tid));
+                    #pragma unroll
+                    for (int k = 0; k < WINDOWS_AHEAD; ++k)
+                        if ((unsigned int)k < more.n_win)
+                            apply_window(load_window(more.win + k * WINDOW), k, more.skip, more.len, add_wide);
+                    apply_rest(more, add_wide);
                 }
             } else {
                 const unsigned int rec0 = a.bin_base[tile];
@@ -778,26 +829,32 @@ static TileArgs tile_args(int I, int H, int T) {
     return a;
 }
 
-size_t pre_tile_smem_bytes(int tile_rows, int horizon) {
-    const TileGeom g = tile_geom(horizon);
-    const size_t warps = (size_t)tile_warps(tile_rows, g);
-    const size_t buffer = (size_t)((tile_rows * g.rpr + 7) & ~7) * 128;
-    // alignment slack, cell buffers, backlog sums, piece sums, piece counts
-    return 1024 + TILE_BUFFERS * buffer + (size_t)tile_rows * 8 + warps * 12 + 16;
+// Threads of a tile block: one per run, but at least eight warps (the spare ones only help to
+// gather, which is what a heavily loaded tile spends its time on).
+int pre_tile_threads(int tile_rows, int horizon) {
+    const int warps = tile_warps(tile_rows, tile_geom(horizon));
+    return 32 * (warps < 8 ? 8 : warps);
 }
 
-int pre_tile_threads(int tile_rows, int horizon) { return 32 * tile_warps(tile_rows, tile_geom(horizon)); }
+size_t pre_tile_smem_bytes(int tile_rows, int horizon) {
+    const TileGeom g = tile_geom(horizon);
+    const size_t warps = (size_t)pre_tile_threads(tile_rows, horizon) / 32;
+    const size_t buffer = (size_t)((tile_rows * g.rpr + 7) & ~7) * 128;
+    // alignment slack, cell buffers, backlog sums + piece sums + piece counts, windows on their way
+    return 1024 + TILE_BUFFERS * buffer + (((size_t)tile_rows * 8 + warps * 12 + 31) & ~(size_t)31) +
+           (size_t)WINDOWS_AHEAD * warps * 32 * 32;
+}
 
-// Rows per tile: a power of two, about eight warps of runs, but several tiles per SM when the
+// Rows per tile: a power of two, about sixteen warps of runs, but several tiles per SM when the
 // number of instances allows it.
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm) {
     const TileGeom g = tile_geom(horizon);
-    int t = g.rpr >= 32 ? 8 / g.cpw : 8 * g.rpw;
+    int t = g.rpr >= 32 ? 16 / g.cpw : 16 * g.rpw;
     if (t < 1) t = 1;
     if (t > PRE_MAX_TILE_ROWS) t = PRE_MAX_TILE_ROWS;
     int p = 1;
     while (p * 2 <= t) p *= 2;
-    while (p > 1 && n_instances / p < 8 * n_sm) p >>= 1;
+    while (p > 1 && n_instances / p < 2 * n_sm) p >>= 1;
     return p;
 }
 
@@ -872,7 +929,7 @@ static bool sort_geometry(int64_t n, int slots, int max_chunks, int* n_chunks, i
     return true;
 }
 
-static size_t sort_smem_bytes(int n_tiles) { return ((size_t)n_tiles + 4) * 4; }
+static size_t sort_smem_bytes(int n_tiles) { return (((size_t)n_tiles + 4) >> 2) * 16 + (size_t)SORT_CHUNK * 8; }   // counts, records
 
 int pre_sort_max_chunks(int64_t max_requests, int n_sm) {
     int64_t need = (max_requests + SORT_CHUNK - 1) / SORT_CHUNK;

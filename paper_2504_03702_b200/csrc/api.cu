@@ -85,7 +85,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_base, (size_t)c->n_tiles + 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_cursor, (size_t)c->n_tiles);
-    if (e == cudaSuccess) e = alloc_zero(&c->d_records, (size_t)cfg->max_requests);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_records, (size_t)cfg->max_requests + 16);   // read in windows of four
     if (e == cudaSuccess) e = alloc_zero(&c->d_enter, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
