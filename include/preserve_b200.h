@@ -65,8 +65,9 @@ typedef struct pre_config {
     int64_t max_requests;    /* capacity of the request table arrays, >= 1, < 2^31 */
 } pre_config;
 
-/* Creates a context on the current CUDA device and allocates its scratch
- * (8 bytes per table slot plus a few MB of index words).  *out is set only on success. */
+/* Creates a context on the current CUDA device and allocates its scratch (8 bytes per
+ * table slot, 8 bytes per instance, and one index word per build tile and 4,096 table
+ * slots: a few MB).  *out is set only on success. */
 int pre_create(const pre_config* cfg, pre_ctx** out);
 
 /* Frees the scratch.  The caller must have synchronised the stream first. */
@@ -93,11 +94,11 @@ int pre_anticipate(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_gener
  * allocator, a callback that runs while the CUDA allocator's lock is held, or a latency-critical
  * control loop where a cudaMalloc (which can synchronise the device) is not acceptable.
  * pre_create allocates scratch; this call uses scratch that is part of the library image
- * instead, about 2.6 MB that every GPU which loads the library holds until the process exits.
+ * instead, about 3.1 MB that every GPU which loads the library holds until the process exits.
  *
- * Limits (PRE_ESIZE beyond them): n_requests <= 262,144; at most 2,048 build tiles, which
- * covers n_instances * horizon up to roughly 8 million cells (e.g. 4,096 x 2,048); device
- * ordinal below 64.  horizon <= 8192 as everywhere.
+ * Limits (PRE_ESIZE beyond them): n_requests <= 262,144; n_instances <= 65,536; at most 2,048
+ * build tiles, which covers n_instances * horizon up to roughly 16 million cells (4,096 x 2,048
+ * needs 1,024 tiles); device ordinal below 64.  horizon <= 8192 as everywhere.
  *
  * Arguments as for pre_anticipate, with the shape passed directly.  d_flags (DEVICE int32,
  * may be NULL, zeroed by the caller) receives a non-zero value if a malformed request was
@@ -109,7 +110,8 @@ int pre_anticipate(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_gener
  * before any stream capture begins.  All calls on a device share the one scratch area, which
  * keeps whatever the last call left in it: two calls whose work overlaps on the GPU (different
  * streams, or different host threads) race and give wrong maps - order them on one stream or
- * with events.  Nothing in the scratch needs clearing between calls.  As with the other
+ * with events.  Nothing in the scratch needs clearing between calls (the one part that must
+ * start at zero, a word per instance, is cleared again by the call that used it).  As with the other
  * entry points, do not call it from two host threads at the same time. */
 int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d_prompt,
                           const int32_t* d_generated, const int32_t* d_predicted, const int32_t* d_instance,
