@@ -30,6 +30,10 @@ def lib():
         for fn in (_lib.orc_route_batch, _lib.orc_route_batch_fast):
             fn.argtypes = route_args
             fn.restype = C.c_int64
+        _lib.orc_route_window.argtypes = [i32p, i32p, C.c_int64, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_double,
+                                          C.c_double, i64p, i64p, i64p, i32p, i32p, i32p, i32p, i64p, C.c_int64, i32p,
+                                          f64p]
+        _lib.orc_route_window.restype = C.c_int64
         _lib.orc_score_all.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int64, C.c_double,
                                        C.c_double, i64p, i64p, i64p, f64p, i64p]
         _lib.orc_score_all.restype = None
@@ -94,6 +98,21 @@ class State:
            _p(self.prompt, C.c_int32), _p(self.generated, C.c_int32), _p(self.predicted, C.c_int32),
            _p(self.instance, C.c_int32), _p(self.n, C.c_int64), self.max_requests,
            _p(choice, C.c_int32), _p(score, C.c_double) if want_score else None)
+        return choice, score
+
+    def route_window(self, arr_prompt, arr_predicted, window, want_score=True):
+        """Router on full-width maps: the state's horizon is the map width L, peaks are taken over
+        the first `window` iterations, the real update adds the whole ramp."""
+        ap, ad = _i32(arr_prompt), _i32(arr_predicted)
+        a = len(ap)
+        choice = np.full(a, -1, np.int32)
+        score = np.zeros(a, np.float64)
+        lib().orc_route_window(_p(ap, C.c_int32), _p(ad, C.c_int32), a, self.I, self.H, int(window), self.M,
+                               self.t_mem, self.beta, _p(self.curves, C.c_int64), _p(self.queued_p, C.c_int64),
+                               _p(self.current_d, C.c_int64), _p(self.prompt, C.c_int32),
+                               _p(self.generated, C.c_int32), _p(self.predicted, C.c_int32),
+                               _p(self.instance, C.c_int32), _p(self.n, C.c_int64), self.max_requests,
+                               _p(choice, C.c_int32), _p(score, C.c_double) if want_score else None)
         return choice, score
 
     def make_queue(self, capacity):

@@ -28,7 +28,9 @@
 // hand-computed example, the closed form of the removed tokens, the chain of
 // extensions and the equality with the definition on the refined table; for
 // the admission queue a hand-computed example, the plain router as the special
-// case that never blocks, and an exact-arithmetic restatement over several calls.  The capacity rule M and the
+// case that never blocks, and an exact-arithmetic restatement over several calls; for the
+// router on full-width maps the plain router as the case l = L, an exact-arithmetic
+// restatement with a window, and the equality of the maps with a rebuild.  The capacity rule M and the
 // queued_p model are this build's readings, not the paper's: parity unpinned
 // for those two (they are inputs, the arithmetic on them is pinned).
 #include <cstdint>
@@ -116,6 +118,40 @@ int64_t orc_route_batch(const int32_t* aP, const int32_t* aD, int64_t A, int32_t
         }
         int64_t* c = curves + (size_t)best * H;
         for (int32_t j = 0; j < H && j < aD[k]; ++j) c[j] += (int64_t)aP[k] + j;
+        queued_p[best] += aP[k];
+        current_d[best] += aD[k];
+        int64_t slot = (*n_requests)++;
+        P[slot] = aP[k]; g[slot] = 0; D[slot] = aD[k]; inst[slot] = best;
+        choice[k] = best;
+        if (score) score[k] = best_l;
+    }
+    for (int64_t r = k; r < A; ++r) { choice[r] = -1; if (score) score[r] = 0.0; }
+    return k;
+}
+
+// The router on full-width maps (Sec. 4.3.1: the map covers the next L iterations, L the
+// largest response the model can produce, while the anticipator projects the load "over the
+// next l iterations" for the router, Sec. 4.3.3).  The peak is taken over the first l steps of
+// a row of width L; the real update adds the whole ramp, min(D, L) steps.  Everything else is
+// orc_route_batch.  With l = L the two are the same function.
+int64_t orc_route_window(const int32_t* aP, const int32_t* aD, int64_t A, int32_t I, int32_t L, int32_t l,
+                         int64_t M, double t_mem, double beta, int64_t* maps, int64_t* queued_p,
+                         int64_t* current_d, int32_t* P, int32_t* g, int32_t* D, int32_t* inst,
+                         int64_t* n_requests, int64_t max_requests, int32_t* choice, double* score) {
+    const double theta = t_mem * (double)M;
+    int64_t k = 0;
+    for (; k < A; ++k) {
+        if (*n_requests >= max_requests) break;
+        if (aP[k] < 0 || aD[k] < 1) { choice[k] = -1; if (score) score[k] = 0.0; continue; }  // malformed
+        int32_t best = -1;
+        double best_l = 0.0;
+        for (int32_t i = 0; i < I; ++i) {
+            int64_t peak = peak_with(maps + (size_t)i * L, l, aP[k], aD[k]);      // the next l iterations
+            double sc = score_of(queued_p[i], current_d[i], peak, aP[k], aD[k], theta, beta);
+            if (best < 0 || sc < best_l) { best = i; best_l = sc; }
+        }
+        int64_t* c = maps + (size_t)best * L;
+        for (int32_t j = 0; j < L && j < aD[k]; ++j) c[j] += (int64_t)aP[k] + j;  // the whole ramp
         queued_p[best] += aP[k];
         current_d[best] += aD[k];
         int64_t slot = (*n_requests)++;

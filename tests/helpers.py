@@ -18,8 +18,9 @@ def brute_curves(prompt, generated, predicted, instance, n_inst, horizon):
 
 
 def exact_route(curves, queued_p, current_d, arr_prompt, arr_predicted, capacity, t_mem=Fraction(4, 5),
-                beta=Fraction(1)):
-    """Greedy router in exact rational arithmetic on Python ints. Returns choices, scores, final state."""
+                beta=Fraction(1), window=None):
+    """Greedy router in exact rational arithmetic on Python ints. Returns choices, scores, final state.
+    `window`: peaks are taken over the first `window` steps only (default: the whole row)."""
     c = [[int(v) for v in row] for row in curves]
     q = [int(v) for v in queued_p]
     cd = [int(v) for v in current_d]
@@ -30,7 +31,7 @@ def exact_route(curves, queued_p, current_d, arr_prompt, arr_predicted, capacity
         p, d = int(p), int(d)
         best, best_l = None, None
         for i in range(n_inst):
-            peak = max(c[i][j] + ((p + j) if j < d else 0) for j in range(horizon))
+            peak = max(c[i][j] + ((p + j) if j < d else 0) for j in range(horizon if window is None else window))
             l = (q[i] + p) + (cd[i] + d) + Fraction(beta) * max(Fraction(0), peak - theta)
             if best is None or l < best_l:
                 best, best_l = i, l
