@@ -218,6 +218,45 @@ int pre_scaler_signals(pre_ctx* ctx, const int64_t* d_curves, double overload_le
                        double idle_level, int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary,
                        void* stream);
 
+/* Full-width maps (Sec. 4.3.1: the load-look-ahead map covers the next L iterations, L the
+ * largest response the model can produce, e.g. 4,096; the load is projected over the next l
+ * iterations, e.g. l = 100, for the router of Sec. 4.3.3).  A row is kept as a ring over
+ * absolute iterations,
+ *     d_ring[i*width + (head + j) mod width] = tokens of instance i at j iterations from now,
+ * 0 <= j < width = L, int64, row-major; *d_head (DEVICE int64, in [0, width)) is where "now"
+ * is.  A decode iteration then moves no map data.  The three calls below take a context whose
+ * horizon is the WINDOW l (the same context routes on the window); width >= horizon, else
+ * PRE_EINVAL.  A full-width map is built by pre_anticipate on a second context whose horizon
+ * is L, into d_ring with *d_head = 0.  One scheduler tick on full-width maps is
+ *     pre_ring_step, pre_ring_window, pre_route_batch (or pre_route_admit) on the window,
+ *     pre_ring_fold with the choices the router returned,
+ * and gives the decisions of a router that takes its peaks over the first l steps of the
+ * full-width maps and really adds each routed request's whole ramp: no score of a batch
+ * depends on a step beyond the window, and the additions beyond it commute. */
+
+/* d_window[i*l + j] = d_ring[i*width + (head + j) mod width], j < l: the dense maps of width
+ * l (16-byte aligned) that pre_route_batch, pre_route_admit and pre_scaler_signals take. */
+int pre_ring_window(pre_ctx* ctx, const int64_t* d_ring, int32_t width, const int64_t* d_head, int64_t* d_window,
+                    void* stream);
+
+/* The real map update of Sec. 4.3.1 for a routed batch: for every arrival k with
+ * d_choice[k] in [0, n_instances), d_ring[choice][(head + j) mod width] += P_k + j for
+ * j < min(D_k, width).  Entries below zero (dropped, waiting, turned away) are skipped.
+ * The router has already updated the window copy, queued_p, current_d and the request
+ * table; this call only brings the ring up to date.  Integer reductions: the result does
+ * not depend on the order in which the arrivals are applied. */
+int pre_ring_fold(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted, const int32_t* d_choice,
+                  int64_t n_arrivals, int64_t* d_ring, int32_t width, const int64_t* d_head, void* stream);
+
+/* One decode iteration on ring maps: the request table, queued_p and current_d change as in
+ * pre_step; every row's slot at the head (step 0, now past) receives what enters at step
+ * width-1 (the requests with at least `width` tokens still to come; none when width is the
+ * model's largest response), and *d_head becomes (head + 1) mod width.  Afterwards the
+ * logical map equals what pre_anticipate builds from the advanced table. */
+int pre_ring_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                  const int64_t* d_n_requests, int64_t* d_ring, int32_t width, int64_t* d_head, int64_t* d_queued_p,
+                  int64_t* d_current_d, void* stream);
+
 /* Synchronises `stream`, then returns and clears the device status: the most severe of
  * PRE_ETIMEOUT, PRE_ECAPACITY, PRE_EBADREQ recorded since the last call, PRE_ECUDA if the
  * stream reports a CUDA error, else PRE_OK. */

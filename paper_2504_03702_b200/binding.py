@@ -16,7 +16,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
-           "pre_refine", "pre_route_admit")
+           "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step")
 
 
 class pre_config(C.Structure):
@@ -40,6 +40,9 @@ def _load():
     lib.pre_refine.argtypes = [vp] * 11
     lib.pre_route_admit.argtypes = [vp, vp, vp, i64, C.c_double, C.c_double, vp, vp, vp, i64] + [vp] * 12
     lib.pre_scaler_signals.argtypes = [vp, vp, C.c_double, C.c_double, C.c_double, vp, vp, vp, vp]
+    lib.pre_ring_window.argtypes = [vp, vp, C.c_int32, vp, vp, vp]
+    lib.pre_ring_fold.argtypes = [vp, vp, vp, vp, i64, vp, C.c_int32, vp, vp]
+    lib.pre_ring_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
     lib.pre_last_cuda_error.argtypes = [vp]
     lib.pre_strerror.argtypes = [C.c_int]
@@ -140,6 +143,23 @@ def pre_scaler_signals(ctx, curves, overload_level, overload_share, idle_level, 
     return lib.pre_scaler_signals(ctx, _ptr(curves), float(overload_level), float(overload_share),
                                   float(idle_level), _ptr(over_count), _ptr(row_max), _ptr(summary),
                                   _stream() if stream is None else stream)
+
+
+def pre_ring_window(ctx, ring, width, head, window, stream=None):
+    return lib.pre_ring_window(ctx, _ptr(ring), int(width), _ptr(head), _ptr(window),
+                               _stream() if stream is None else stream)
+
+
+def pre_ring_fold(ctx, arr_prompt, arr_predicted, choice, n_arrivals, ring, width, head, stream=None):
+    return lib.pre_ring_fold(ctx, _ptr(arr_prompt), _ptr(arr_predicted), _ptr(choice), int(n_arrivals), _ptr(ring),
+                             int(width), _ptr(head), _stream() if stream is None else stream)
+
+
+def pre_ring_step(ctx, prompt, generated, predicted, instance, n_requests, ring, width, head, queued_p, current_d,
+                  stream=None):
+    return lib.pre_ring_step(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(n_requests),
+                             _ptr(ring), int(width), _ptr(head), _ptr(queued_p), _ptr(current_d),
+                             _stream() if stream is None else stream)
 
 
 def pre_status(ctx, stream=None):

@@ -30,6 +30,7 @@ void release(pre_ctx* c) {
     cudaFree(c->d_active);
     cudaFree(c->d_scaler_partial);
     cudaFree(c->d_scaler_done);
+    cudaFree(c->d_ring_done);
     cudaFree(c->d_queue_entry);
     delete c;
 }
@@ -90,6 +91,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_done, 1);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_ring_done, 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_queue_entry, 2);
     if (e == cudaSuccess) e = pre_anticipate_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
@@ -211,6 +213,44 @@ int pre_scaler_signals(pre_ctx* ctx, const int64_t* d_curves, double overload_le
         return PRE_EINVAL;
     cudaError_t e = pre_launch_scaler(ctx, d_curves, overload_level, overload_share, idle_level, d_over_count,
                                       d_row_max, d_summary, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_ring_window(pre_ctx* ctx, const int64_t* d_ring, int32_t width, const int64_t* d_head, int64_t* d_window,
+                    void* stream) {
+    if (!ctx || !d_ring || !d_head || !d_window) return PRE_EINVAL;
+    if (width < ctx->cfg.horizon || (long long)ctx->cfg.n_instances * width >= (1LL << 40)) return PRE_EINVAL;
+    if (!aligned(d_ring, 8) || !aligned(d_head, 8) || !aligned(d_window, 16)) return PRE_EINVAL;
+    cudaError_t e = pre_launch_ring_window(ctx, d_ring, width, d_head, d_window, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_ring_fold(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted, const int32_t* d_choice,
+                  int64_t n_arrivals, int64_t* d_ring, int32_t width, const int64_t* d_head, void* stream) {
+    if (!ctx || !d_ring || !d_head || n_arrivals < 0 || n_arrivals >= (1LL << 31)) return PRE_EINVAL;
+    if (width < ctx->cfg.horizon || (long long)ctx->cfg.n_instances * width >= (1LL << 40)) return PRE_EINVAL;
+    if (n_arrivals > 0 && (!d_arr_prompt || !d_arr_predicted || !d_choice)) return PRE_EINVAL;
+    if (!aligned(d_ring, 8) || !aligned(d_head, 8) || !aligned(d_arr_prompt, 4) || !aligned(d_arr_predicted, 4) ||
+        !aligned(d_choice, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_ring_fold(ctx, d_arr_prompt, d_arr_predicted, d_choice, n_arrivals, d_ring, width,
+                                         d_head, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_ring_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+                  const int64_t* d_n_requests, int64_t* d_ring, int32_t width, int64_t* d_head, int64_t* d_queued_p,
+                  int64_t* d_current_d, void* stream) {
+    if (!ctx || !d_prompt || !d_generated || !d_predicted || !d_instance || !d_n_requests || !d_ring || !d_head ||
+        !d_queued_p || !d_current_d)
+        return PRE_EINVAL;
+    if (width < ctx->cfg.horizon || (long long)ctx->cfg.n_instances * width >= (1LL << 40)) return PRE_EINVAL;
+    if (!aligned(d_ring, 8) || !aligned(d_head, 8) || !aligned(d_queued_p, 8) || !aligned(d_current_d, 8) ||
+        !aligned(d_n_requests, 8) || !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) ||
+        !aligned(d_instance, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_ring_step(ctx, d_prompt, d_generated, d_predicted, d_instance, d_n_requests, d_ring,
+                                         width, d_head, d_queued_p, d_current_d, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
 }
 

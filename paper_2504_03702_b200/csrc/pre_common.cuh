@@ -51,6 +51,7 @@ struct pre_ctx {
     unsigned int* d_active;         // [I] live requests per instance (zero between calls)
     long long* d_scaler_partial;    // [8 * n_sm][3] block totals of the scaler-signal kernel
     unsigned int* d_scaler_done;    // blocks of that kernel that have finished (zero between calls)
+    unsigned int* d_ring_done;      // the same for the kernel that advances a ring of maps
 };
 
 // Launchers (defined next to their kernels).  Each returns a cudaError_t.
@@ -77,6 +78,16 @@ cudaError_t pre_launch_refine(pre_ctx* ctx, const int32_t* prompt, const int32_t
 cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overload_level, double overload_share,
                               double idle_level, int32_t* over_count, int64_t* row_max, int64_t* summary,
                               cudaStream_t s);
+cudaError_t pre_launch_step_requests(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                                     int32_t* instance, const int64_t* n_requests, int width, cudaStream_t s);
+cudaError_t pre_launch_ring_window(pre_ctx* ctx, const int64_t* ring, int width, const int64_t* head,
+                                   int64_t* window, cudaStream_t s);
+cudaError_t pre_launch_ring_fold(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                 const int32_t* choice, int64_t n_arrivals, int64_t* ring, int width,
+                                 const int64_t* head, cudaStream_t s);
+cudaError_t pre_launch_ring_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                                 int32_t* instance, const int64_t* n_requests, int64_t* ring, int width,
+                                 int64_t* head, int64_t* queued_p, int64_t* current_d, cudaStream_t s);
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
 size_t pre_tile_smem_bytes(int tile_rows, int horizon);
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm);

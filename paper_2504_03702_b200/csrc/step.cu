@@ -111,17 +111,27 @@ pre_step_shift(int64_t* __restrict__ curves, int64_t* __restrict__ queued_p, int
 
 }  // namespace
 
-cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
-                            int32_t* instance, const int64_t* n_requests, int64_t* curves,
-                            int64_t* queued_p, int64_t* current_d, cudaStream_t s) {
-    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+// The pass over the request table alone, for a map of `width` steps (the shift of a dense map,
+// or the advance of a ring, follows).
+cudaError_t pre_launch_step_requests(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                                     int32_t* instance, const int64_t* n_requests, int width, cudaStream_t s) {
+    const int I = ctx->cfg.n_instances;
     const size_t smem = I <= PRE_SMEM_BINS ? (size_t)I * sizeof(unsigned int) : 0;
     long long want = (ctx->cfg.max_requests + STEP_THREADS * 4 - 1) / (STEP_THREADS * 4);
     int grid = (int)(want < 4LL * ctx->n_sm ? want : 4LL * ctx->n_sm);
     if (grid < 1) grid = 1;
     pre_step_requests<<<grid, STEP_THREADS, smem, s>>>(prompt, generated, predicted, instance, n_requests,
-                                                     ctx->cfg.max_requests, I, H, ctx->d_active, ctx->d_enter,
+                                                     ctx->cfg.max_requests, I, width, ctx->d_active, ctx->d_enter,
                                                      ctx->d_status);
+    return cudaGetLastError();
+}
+
+cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                            int32_t* instance, const int64_t* n_requests, int64_t* curves,
+                            int64_t* queued_p, int64_t* current_d, cudaStream_t s) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    cudaError_t e = pre_launch_step_requests(ctx, prompt, generated, predicted, instance, n_requests, H, s);
+    if (e != cudaSuccess) return e;
     int sgrid = I < 16 * ctx->n_sm ? I : 16 * ctx->n_sm;
     pre_step_shift<<<sgrid, SHIFT_THREADS, 0, s>>>(curves, queued_p, current_d, ctx->d_active, ctx->d_enter, I, H);
     return cudaGetLastError();

@@ -15,6 +15,7 @@ class DeviceState:
     def __init__(self, n_instances, horizon, capacity_tokens, max_requests, t_mem=0.8, beta=1.0,
                  device="cuda:0"):
         self.I, self.H = int(n_instances), int(horizon)
+        self.capacity_tokens, self.t_mem, self.beta = int(capacity_tokens), float(t_mem), float(beta)
         self.max_requests = int(max_requests)
         self.device = torch.device(device)
         with torch.cuda.device(self.device):
@@ -104,6 +105,44 @@ class DeviceState:
         B.check(B.pre_scaler_signals(self.ctx, self.curves, overload_level, overload_share, idle_level, over,
                                      row_max, summary), "pre_scaler_signals")
         return over, row_max, summary
+
+    # ---- full-width maps kept as a ring (the state's own maps are then the window of width H = l)
+
+    def make_ring(self, width, builder=None):
+        """Allocates ring[I][width] and the head word, and builds the full-width maps from the table
+        (pre_anticipate on a context of horizon `width`; pass one as `builder` to reuse it)."""
+        self.width = int(width)
+        self.ring = torch.zeros(self.I, self.width, dtype=torch.int64, device=self.device)
+        self.head = torch.zeros(1, dtype=torch.int64, device=self.device)
+        own = builder is None
+        if own:
+            with torch.cuda.device(self.device):
+                code, builder = B.pre_create(self.I, self.width, self.capacity_tokens, self.t_mem, self.beta,
+                                             self.max_requests)
+            B.check(code, "pre_create")
+        B.check(B.pre_anticipate(builder, self.prompt, self.generated, self.predicted, self.instance, self.n_host,
+                                 self.ring, self.current_d), "pre_anticipate")
+        if own:
+            torch.cuda.synchronize(self.device)
+            B.pre_destroy(builder)
+
+    def ring_window(self):
+        B.check(B.pre_ring_window(self.ctx, self.ring, self.width, self.head, self.curves), "pre_ring_window")
+
+    def ring_fold(self, arr_prompt, arr_predicted, choice):
+        B.check(B.pre_ring_fold(self.ctx, arr_prompt, arr_predicted, choice, int(arr_prompt.shape[0]), self.ring,
+                                self.width, self.head), "pre_ring_fold")
+
+    def ring_step(self):
+        B.check(B.pre_ring_step(self.ctx, self.prompt, self.generated, self.predicted, self.instance,
+                                self.n_requests, self.ring, self.width, self.head, self.queued_p, self.current_d),
+                "pre_ring_step")
+
+    def ring_logical(self):
+        """The ring read out in logical order (column j = j iterations from now); synchronises."""
+        h = int(self.head.item())
+        idx = (h + torch.arange(self.width, device=self.device)) % self.width
+        return self.ring[:, idx]
 
     def status(self):
         return B.pre_status(self.ctx)

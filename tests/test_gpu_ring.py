@@ -1,0 +1,106 @@
+"""Full-width maps kept as a ring (pre_ring_step, pre_ring_window, pre_ring_fold) against the
+oracle's router on full-width maps, tick by tick, through the C-ABI.
+
+The device keeps ring[I][L] and routes on the window of width l; the oracle keeps the dense
+maps of width L, takes peaks over their first l steps and shifts them on every step.  Bar: ring
+(read out in logical order), backlog words, table and decisions bit-exact, scores within 1e-12.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_03702_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import assert_scores_close, dev, table  # noqa: E402
+from paper_2504_03702_b200 import binding as B  # noqa: E402
+from paper_2504_03702_b200.state import DeviceState  # noqa: E402
+
+
+def pair(wl, width, window, extra_rows):
+    """Device state whose own maps are the window, with a ring of `width`; oracle state of `width`."""
+    cap = wl.n_requests + extra_rows
+    st = DeviceState(wl.n_instances, window, wl.capacity_tokens, max(cap, 1), wl.t_mem, wl.beta)
+    st.load_requests(wl.prompt, wl.generated, wl.predicted, wl.instance)
+    st.make_ring(width)
+    ref = oracle.State(wl.n_instances, width, wl.capacity_tokens, wl.prompt, wl.generated, wl.predicted,
+                       wl.instance, max(cap, 1), wl.t_mem, wl.beta)
+    ref.anticipate()
+    return st, ref
+
+
+def same(st, ref, what):
+    assert (st.ring_logical().cpu().numpy() == ref.curves).all(), f"ring differs {what}"
+    assert (st.current_d.cpu().numpy() == ref.current_d).all(), f"current_d differs {what}"
+    assert (st.queued_p.cpu().numpy() == ref.queued_p).all(), f"queued_p differs {what}"
+    n = st.sync_count()
+    assert n == int(ref.n[0])
+    for got, want in zip(table(st), (ref.prompt, ref.generated, ref.predicted, ref.instance)):
+        assert (got == want[:n]).all(), f"table differs {what}"
+
+
+def tick(st, ref, ap, ad, window):
+    st.ring_step()
+    ref.step()
+    st.ring_window()
+    choice, score = st.route_batch(dev(ap), dev(ad))
+    st.ring_fold(dev(ap), dev(ad), choice)
+    want_c, want_s = ref.route_window(ap, ad, window)
+    assert (choice.cpu().numpy() == want_c).all()
+    assert_scores_close(score.cpu().numpy(), want_s, want_c)
+
+
+@pytest.mark.parametrize("seed,n_inst,width,window,n,a,ticks", [
+    (71, 1, 5, 2, 12, 4, 14),          # the head goes round the ring several times
+    (72, 6, 40, 7, 150, 20, 50),
+    (73, 37, 96, 96, 600, 33, 12),     # window = width
+    (74, 300, 257, 100, 4000, 150, 6),
+    (75, 9, 16, 1, 80, 10, 20),
+])
+def test_ring_ticks_match_the_oracle(seed, n_inst, width, window, n, a, ticks):
+    # responses up to twice the width: some requests reach beyond the map and enter it later
+    wl = W.make_random(seed, n_inst, width, n, 0, max_prompt=300, max_output=2 * width)
+    st, ref = pair(wl, width, window, a * ticks)
+    same(st, ref, "after the build")
+    rng = np.random.RandomState(seed)
+    for t in range(ticks):
+        ap = rng.randint(1, 300, a).astype(np.int32)
+        ad = rng.randint(1, 2 * width + 1, a).astype(np.int32)
+        if t == 1 and a > 3:
+            ap[2] = -5                                 # malformed: dropped, result -1
+        tick(st, ref, ap, ad, window)
+        same(st, ref, f"after tick {t}")
+    assert st.status() in (B.PRE_OK, B.PRE_EBADREQ)
+    # the ring still is what the definition gives for the table as it stands
+    n_rows = st.sync_count()
+    check = oracle.State(n_inst, width, wl.capacity_tokens, ref.prompt[:n_rows], ref.generated[:n_rows],
+                         ref.predicted[:n_rows], ref.instance[:n_rows], n_rows)
+    check.anticipate()
+    assert (st.ring_logical().cpu().numpy() == check.curves).all()
+    st.close()
+
+
+def test_ring_streaming_config_first_ticks():
+    """The streaming configuration on maps of its full width (1,024) with the paper's window of 100."""
+    wl = W.make_config(4, n_ticks=3)
+    st, ref = pair(wl, wl.horizon, 100, sum(len(t[0]) for t in wl.ticks))
+    for t, (ap, ad) in enumerate(wl.ticks):
+        tick(st, ref, ap, ad, 100)
+        same(st, ref, f"after tick {t}")
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
+def test_ring_argument_errors_launch_nothing():
+    wl = W.make_random(76, 4, 16, 10, 0)
+    st, _ = pair(wl, 16, 8, 4)
+    assert B.pre_ring_window(st.ctx, st.ring, 7, st.head, st.curves) == B.PRE_EINVAL      # narrower than the window
+    assert B.pre_ring_window(st.ctx, None, 16, st.head, st.curves) == B.PRE_EINVAL
+    assert B.pre_ring_fold(st.ctx, None, None, None, 3, st.ring, 16, st.head) == B.PRE_EINVAL
+    assert B.pre_ring_fold(st.ctx, None, None, None, 0, st.ring, 16, st.head) == B.PRE_OK  # an empty batch
+    assert B.pre_ring_step(st.ctx, st.prompt, st.generated, st.predicted, st.instance, st.n_requests, st.ring, 16,
+                           None, st.queued_p, st.current_d) == B.PRE_EINVAL
+    torch.cuda.synchronize()
+    st.close()
