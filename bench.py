@@ -346,6 +346,32 @@ def main():
     rf_counts = [int(v) for v in rf_counts.cpu().tolist()]
     B.check(st.status(), "refinement ticks")
 
+    # full-width maps kept as a ring (Sec. 4.3.1), routed on the paper's window of 100 iterations:
+    # a separate state on the same table and batch; one warm tick, one timed tick
+    ring_window = min(100, wl.horizon)
+    ring_st = DeviceState(wl.n_instances, ring_window, wl.capacity_tokens, n0 + 2 * a, wl.t_mem, wl.beta,
+                          device=device)
+    ring_st.load_requests(wl.prompt, wl.generated, wl.predicted, wl.instance)
+    ring_st.make_ring(wl.horizon)
+    ring_ms = None
+    for k in range(2):
+        flush.zero_()
+        e = [ev() for _ in range(5)]
+        e[0].record()
+        ring_st.ring_step()
+        e[1].record()
+        ring_st.ring_window()
+        e[2].record()
+        ring_choice, _ = ring_st.route_batch(arr_p, arr_d)
+        e[3].record()
+        ring_st.ring_fold(arr_p, arr_d, ring_choice)
+        e[4].record()
+        torch.cuda.synchronize()
+        ring_ms = [e[i].elapsed_time(e[i + 1]) for i in range(4)]
+    B.check(ring_st.status(), "ring tick")
+    ring_routed = int((ring_choice >= 0).sum())
+    ring_st.close()
+
     if rank != 0:
         D.finish(group)
         return 0
@@ -389,6 +415,15 @@ def main():
                                 events_last_tick={"early_finish": rf_counts[0], "extended": rf_counts[1]},
                                 note="separate call, not part of the step; bytes = five int32 columns of the "
                                      "table, the read-modify-write of the touched map cells is not counted"),
+        "full_width_maps": {
+            "width": wl.horizon, "window": ring_window, "routed": ring_routed,
+            "tick_ms": {"pre_ring_step": ring_ms[0], "pre_ring_window": ring_ms[1], "pre_route_batch": ring_ms[2],
+                        "pre_ring_fold": ring_ms[3]},
+            "routes_per_s": a / (sum(ring_ms) * 1e-3),
+            "dense_maps_same_tick_ms": {"pre_step": t_dstep, "pre_route_batch": t_route},
+            "note": "separate state, not part of the step: maps of the configuration's full width kept as a ring "
+                    "over absolute iterations, peaks taken over the next 100 iterations (the paper's l); one "
+                    "scheduler tick = decode step + window copy + routing of the batch + real update of the ring"},
         "e2e": {"value": world * a / (t_e2e * 1e-3), "unit": "routes/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e},
         "gpu_launches": 5 * args.steps,
