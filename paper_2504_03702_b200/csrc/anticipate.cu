@@ -482,6 +482,53 @@ __device__ __forceinline__ unsigned long long piece_sum(unsigned int v, unsigned
     return ((unsigned long long)hi << 16) + lo;
 }
 
+// The 32-bit scan of a tile whose every thread owns a run (rows of a whole number of 32-run
+// pieces, a full tile, no spare warps): thread t owns run t.  Straight-line code.
+__device__ __forceinline__ void tile_scan_whole(int cpw, unsigned char* cells, unsigned long long* cur,
+                                                uint2* piece_tot) {
+    const unsigned int tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const unsigned int row = warp / (unsigned int)cpw, piece = warp - row * (unsigned int)cpw;
+    const unsigned int j0 = (piece * 32u + lane) * RUN;
+    unsigned char* mine = cells + ((size_t)tid << 7);
+    const unsigned int sw = (tid & 7u) << 4;          // piece i of the run lies at byte (i*16) ^ sw
+
+    uint4 v[RUN / 2];     // {sum, count, sum, count} of two cells
+    #pragma unroll
+    for (int i = 0; i < RUN / 2; ++i) v[i] = *reinterpret_cast<const uint4*>(mine + ((i * 16) ^ sw));
+    unsigned int tn = 0, ts = 0;
+    #pragma unroll
+    for (int i = 0; i < RUN / 2; ++i) { ts += v[i].x + v[i].z; tn += v[i].y + v[i].w; }
+    unsigned int xn = tn, xs = ts;
+    #pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int yn = __shfl_down_sync(0xffffffffu, xn, off);
+        const unsigned int ys = __shfl_down_sync(0xffffffffu, xs, off);
+        if (lane + off < 32u) { xn += yn; xs += ys; }
+    }
+    unsigned int N = xn - tn, A = xs - ts;
+    if (cpw > 1) {
+        if (lane == 0) piece_tot[warp] = make_uint2(xn, xs);
+        __syncthreads();
+        for (unsigned int kk = piece + 1; kk < (unsigned int)cpw; ++kk) {
+            const uint2 t = piece_tot[warp - piece + kk];
+            N += t.x; A += t.y;
+        }
+    }
+    unsigned int sn = 0;
+    #pragma unroll
+    for (int i = RUN / 2 - 1; i >= 0; --i) {
+        uint4 o;
+        N += v[i].w; A += v[i].z; sn += N;
+        o.z = A + N * (j0 + 2 * i + 1); o.w = 0;
+        N += v[i].y; A += v[i].x; sn += N;
+        o.x = A + N * (j0 + 2 * i); o.y = 0;
+        *reinterpret_cast<uint4*>(mine + ((i * 16) ^ sw)) = o;
+    }
+    const unsigned int lo = __reduce_add_sync(0xffffffffu, sn & 0xFFFFu);
+    const unsigned int hi = __reduce_add_sync(0xffffffffu, sn >> 16);
+    if (lane == 0) atomicAdd(&cur[row], ((unsigned long long)hi << 16) + lo);
+}
+
 // The scan of one tile in 32 bits; results overwrite the cell words (int64 map values).
 __device__ __forceinline__ void tile_scan_narrow(const TileArgs& a, int rows, unsigned char* cells,
                                                  unsigned long long* cur, unsigned int* piece_n,
@@ -604,7 +651,7 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
     const TileGeom& g = a.g;
     const int H = a.sh.H, T = 1 << a.sh.tile_shift, hp = a.sh.hp, n_tiles = a.sh.n_tiles;
     const int nwarps = blockDim.x >> 5;
-    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
     // carve: cell buffers (1024-byte aligned: the swizzle pattern repeats every 1024 bytes), backlog
     // sums, piece sums, piece counts
     const unsigned int raw = (unsigned int)__cvta_generic_to_shared(smem_raw);
@@ -652,7 +699,7 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
 
         const unsigned long long beyond = tid < rows ? a.excess[row0 + tid] : 0ull;
 
-        // ---- the cell buffer is free once the store of the tile before the last has read it
+        // ---- the cell buffer is free once the store that last used it has read it
         if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(TILE_BUFFERS - 1) : "memory");
         __syncthreads();
         {
@@ -719,7 +766,10 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
             (unsigned long long)tile_records * ((largest > 32u ? largest : 32u) + (unsigned long long)H);
 
         if (bound < (1ull << 32)) {
-            tile_scan_narrow(a, rows, cells, cur, piece_n, reinterpret_cast<unsigned int*>(piece_s));
+            if (g.W == 32 && g.rpr == 32 * g.cpw && rows == T && nthr == 32 * T * g.cpw)
+                tile_scan_whole(g.cpw, cells, cur, reinterpret_cast<uint2*>(piece_s));
+            else
+                tile_scan_narrow(a, rows, cells, cur, piece_n, reinterpret_cast<unsigned int*>(piece_s));
             if (tma) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stores above, for the copy unit
                 __syncthreads();
