@@ -257,6 +257,14 @@ int pre_ring_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t
                   const int64_t* d_n_requests, int64_t* d_ring, int32_t width, int64_t* d_head, int64_t* d_queued_p,
                   int64_t* d_current_d, void* stream);
 
+/* pre_refine (Sec. 4.3.1, the correction of the maps against real response lengths) on ring
+ * maps: the same rule, with step j of a row at d_ring[i*width + (head + j) mod width] and the
+ * ramps cut at `width` instead of the window.  Call it once per tick after pre_ring_step and
+ * before pre_ring_window, so that the router sees the corrected window. */
+int pre_ring_refine(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated, int32_t* d_predicted,
+                    const int32_t* d_instance, const int32_t* d_actual, const int64_t* d_n_requests, int64_t* d_ring,
+                    int32_t width, const int64_t* d_head, int64_t* d_current_d, int64_t* d_counts, void* stream);
+
 /* Synchronises `stream`, then returns and clears the device status: the most severe of
  * PRE_ETIMEOUT, PRE_ECAPACITY, PRE_EBADREQ recorded since the last call, PRE_ECUDA if the
  * stream reports a CUDA error, else PRE_OK. */

@@ -16,7 +16,8 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
-           "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step")
+           "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step",
+           "pre_ring_refine")
 
 
 class pre_config(C.Structure):
@@ -43,6 +44,7 @@ def _load():
     lib.pre_ring_window.argtypes = [vp, vp, C.c_int32, vp, vp, vp]
     lib.pre_ring_fold.argtypes = [vp, vp, vp, vp, i64, vp, C.c_int32, vp, vp]
     lib.pre_ring_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
+    lib.pre_ring_refine.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
     lib.pre_last_cuda_error.argtypes = [vp]
     lib.pre_strerror.argtypes = [C.c_int]
@@ -160,6 +162,13 @@ def pre_ring_step(ctx, prompt, generated, predicted, instance, n_requests, ring,
     return lib.pre_ring_step(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(n_requests),
                              _ptr(ring), int(width), _ptr(head), _ptr(queued_p), _ptr(current_d),
                              _stream() if stream is None else stream)
+
+
+def pre_ring_refine(ctx, prompt, generated, predicted, instance, actual, n_requests, ring, width, head, current_d,
+                    counts, stream=None):
+    return lib.pre_ring_refine(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(actual),
+                               _ptr(n_requests), _ptr(ring), int(width), _ptr(head), _ptr(current_d), _ptr(counts),
+                               _stream() if stream is None else stream)
 
 
 def pre_status(ctx, stream=None):

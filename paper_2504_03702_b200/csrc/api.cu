@@ -199,7 +199,24 @@ int pre_refine(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated
         !aligned(d_actual, 4))
         return PRE_EINVAL;
     cudaError_t e = pre_launch_refine(ctx, d_prompt, d_generated, d_predicted, d_instance, d_actual, d_n_requests,
-                                      d_curves, d_current_d, d_counts, static_cast<cudaStream_t>(stream));
+                                      d_curves, ctx->cfg.horizon, nullptr, d_current_d, d_counts,
+                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_ring_refine(pre_ctx* ctx, const int32_t* d_prompt, const int32_t* d_generated, int32_t* d_predicted,
+                    const int32_t* d_instance, const int32_t* d_actual, const int64_t* d_n_requests, int64_t* d_ring,
+                    int32_t width, const int64_t* d_head, int64_t* d_current_d, int64_t* d_counts, void* stream) {
+    if (!ctx || !d_prompt || !d_generated || !d_predicted || !d_instance || !d_actual || !d_n_requests || !d_ring ||
+        !d_head || !d_current_d)
+        return PRE_EINVAL;
+    if (width < ctx->cfg.horizon || (long long)ctx->cfg.n_instances * width >= (1LL << 40)) return PRE_EINVAL;
+    if (!aligned(d_ring, 8) || !aligned(d_head, 8) || !aligned(d_current_d, 8) || !aligned(d_n_requests, 8) ||
+        !aligned(d_counts, 8) || !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) ||
+        !aligned(d_instance, 4) || !aligned(d_actual, 4))
+        return PRE_EINVAL;
+    cudaError_t e = pre_launch_refine(ctx, d_prompt, d_generated, d_predicted, d_instance, d_actual, d_n_requests,
+                                      d_ring, width, d_head, d_current_d, d_counts, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
 }
 

@@ -74,7 +74,8 @@ cudaError_t pre_launch_step(pre_ctx* ctx, int32_t* prompt, int32_t* generated, i
                             int64_t* queued_p, int64_t* current_d, cudaStream_t s);
 cudaError_t pre_launch_refine(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated, int32_t* predicted,
                               const int32_t* instance, const int32_t* actual, const int64_t* n_requests,
-                              int64_t* curves, int64_t* current_d, int64_t* counts, cudaStream_t s);
+                              int64_t* curves, int width, const int64_t* head, int64_t* current_d, int64_t* counts,
+                              cudaStream_t s);
 cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overload_level, double overload_share,
                               double idle_level, int32_t* over_count, int64_t* row_max, int64_t* summary,
                               cudaStream_t s);

@@ -20,12 +20,14 @@ __global__ void __launch_bounds__(REFINE_THREADS)
 pre_refine_requests(const int32_t* __restrict__ prompt, const int32_t* __restrict__ generated,
                     int32_t* __restrict__ predicted, const int32_t* __restrict__ instance,
                     const int32_t* __restrict__ actual, const int64_t* __restrict__ n_requests, int I, int H,
-                    int64_t* __restrict__ curves, int64_t* __restrict__ current_d,
+                    const int64_t* __restrict__ head_p, int64_t* __restrict__ curves, int64_t* __restrict__ current_d,
                     unsigned long long* __restrict__ counts, int* __restrict__ status) {
     __shared__ unsigned int sh_tally[3];
     if (threadIdx.x < 3) sh_tally[threadIdx.x] = 0;
     __syncthreads();
     const int64_t n = *n_requests;
+    // dense maps: step j of a row is cell j; maps kept as a ring: cell (head + j) mod H
+    const unsigned int head = head_p ? (unsigned int)(*head_p % H) : 0u;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t stride = (int64_t)gridDim.x * REFINE_WARPS * 32;
     unsigned int n_early = 0, n_ext = 0, n_bad = 0;
@@ -59,7 +61,9 @@ pre_refine_requests(const int32_t* __restrict__ prompt, const int32_t* __restric
             unsigned long long* c = reinterpret_cast<unsigned long long*>(curves + (size_t)row * H);
             for (int j = lane; j < len; j += 32) {
                 const long long v = f + j;
-                atomicAdd(c + j, (unsigned long long)(take_out ? -v : v));
+                unsigned int at = head + (unsigned int)j;
+                if (at >= (unsigned int)H) at -= (unsigned int)H;
+                atomicAdd(c + at, (unsigned long long)(take_out ? -v : v));
             }
         }
         if (kind != 0) {
@@ -86,9 +90,12 @@ pre_refine_requests(const int32_t* __restrict__ prompt, const int32_t* __restric
 
 }  // namespace
 
+// `width` and `head`: the maps are rows of `width` cells; with `head` (a device word) they are
+// rings and step j lies at cell (head + j) mod width, without it step j is cell j.
 cudaError_t pre_launch_refine(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated, int32_t* predicted,
                               const int32_t* instance, const int32_t* actual, const int64_t* n_requests,
-                              int64_t* curves, int64_t* current_d, int64_t* counts, cudaStream_t s) {
+                              int64_t* curves, int width, const int64_t* head, int64_t* current_d, int64_t* counts,
+                              cudaStream_t s) {
     if (counts) {
         cudaError_t e = cudaMemsetAsync(counts, 0, 3 * sizeof(int64_t), s);
         if (e != cudaSuccess) return e;
@@ -100,7 +107,7 @@ cudaError_t pre_launch_refine(pre_ctx* ctx, const int32_t* prompt, const int32_t
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     pre_refine_requests<<<(int)blocks, REFINE_THREADS, 0, s>>>(
-        prompt, generated, predicted, instance, actual, n_requests, ctx->cfg.n_instances, ctx->cfg.horizon, curves,
+        prompt, generated, predicted, instance, actual, n_requests, ctx->cfg.n_instances, width, head, curves,
         current_d, reinterpret_cast<unsigned long long*>(counts), ctx->d_status);
     return cudaGetLastError();
 }

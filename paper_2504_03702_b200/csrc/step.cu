@@ -118,7 +118,7 @@ cudaError_t pre_launch_step_requests(pre_ctx* ctx, int32_t* prompt, int32_t* gen
     const int I = ctx->cfg.n_instances;
     const size_t smem = I <= PRE_SMEM_BINS ? (size_t)I * sizeof(unsigned int) : 0;
     long long want = (ctx->cfg.max_requests + STEP_THREADS * 4 - 1) / (STEP_THREADS * 4);
-    int grid = (int)(want < 4LL * ctx->n_sm ? want : 4LL * ctx->n_sm);
+    int grid = (int)(want < 2LL * ctx->n_sm ? want : 2LL * ctx->n_sm);   // fewer blocks, fewer per-block flushes of the live counts
     if (grid < 1) grid = 1;
     pre_step_requests<<<grid, STEP_THREADS, smem, s>>>(prompt, generated, predicted, instance, n_requests,
                                                      ctx->cfg.max_requests, I, width, ctx->d_active, ctx->d_enter,

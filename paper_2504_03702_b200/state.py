@@ -138,6 +138,14 @@ class DeviceState:
                                 self.n_requests, self.ring, self.width, self.head, self.queued_p, self.current_d),
                 "pre_ring_step")
 
+    def ring_refine(self, actual, want_counts=True):
+        """pre_refine on the ring; returns the device tensor int64[3] of counts or None."""
+        counts = torch.empty(3, dtype=torch.int64, device=self.device) if want_counts else None
+        B.check(B.pre_ring_refine(self.ctx, self.prompt, self.generated, self.predicted, self.instance, actual,
+                                  self.n_requests, self.ring, self.width, self.head, self.current_d, counts),
+                "pre_ring_refine")
+        return counts
+
     def ring_logical(self):
         """The ring read out in logical order (column j = j iterations from now); synchronises."""
         h = int(self.head.item())

@@ -82,6 +82,41 @@ def test_ring_ticks_match_the_oracle(seed, n_inst, width, window, n, a, ticks):
     st.close()
 
 
+@pytest.mark.parametrize("seed,n_inst,width,window,n,a,ticks", [(77, 5, 24, 6, 120, 12, 60), (78, 40, 130, 100, 900, 40, 30)])
+def test_ring_ticks_with_refinement_match_the_oracle(seed, n_inst, width, window, n, a, ticks):
+    """A tick with the correction against real lengths: step, refine, window, route, fold."""
+    wl = W.make_random(seed, n_inst, width, n, 0, max_prompt=200, max_output=width)
+    st, ref = pair(wl, width, window, a * ticks)
+    rng = np.random.RandomState(seed)
+    cap = n + a * ticks
+    actual = np.ones(cap, np.int32)
+    actual[:n] = np.maximum(wl.generated + 1, wl.predicted + rng.randint(-15, 16, n)).astype(np.int32)
+    actual_dev = dev(actual)
+    early = extended = 0
+    for t in range(ticks):
+        ap = rng.randint(1, 200, a).astype(np.int32)
+        ad = rng.randint(1, width + 1, a).astype(np.int32)
+        n_before = int(ref.n[0])
+        actual[n_before:n_before + a] = np.maximum(1, ad + rng.randint(-15, 16, a))
+        actual_dev[n_before:n_before + a] = dev(actual[n_before:n_before + a])
+        st.ring_step()
+        ref.step()
+        got = st.ring_refine(actual_dev).cpu().numpy()
+        want = ref.refine(actual)
+        assert (got == want).all(), f"refinement counts differ at tick {t}"
+        early += int(want[0]); extended += int(want[1])
+        st.ring_window()
+        choice, score = st.route_batch(dev(ap), dev(ad))
+        st.ring_fold(dev(ap), dev(ad), choice)
+        want_c, want_s = ref.route_window(ap, ad, window)
+        assert (choice.cpu().numpy() == want_c).all()
+        assert_scores_close(score.cpu().numpy(), want_s, want_c)
+        same(st, ref, f"after tick {t}")
+    assert early > 0 and extended > 0
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
 def test_ring_streaming_config_first_ticks():
     """The streaming configuration on maps of its full width (1,024) with the paper's window of 100."""
     wl = W.make_config(4, n_ticks=3)
