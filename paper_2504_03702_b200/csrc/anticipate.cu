@@ -635,9 +635,11 @@ __device__ __forceinline__ void tile_scan_wide(const TileArgs& a, int row0, int 
     if (at.sub == 0 && at.row < rows && sum_n) atomicAdd(&cur[at.row], sum_n);
 }
 
-// One thread: bulk tensor stores of a finished tile (runs [run0, run0 + n_runs) of the map).
-__device__ __forceinline__ void store_tile_tma(const CUtensorMap* map, const unsigned char* cells, int run0, int n_runs) {
-    for (int r = 0; r < n_runs; r += TMA_BOX_RUNS) {
+// One thread: bulk tensor stores of the runs [run0 + first, run0 + first + n_runs) of the map
+// from the cell buffer, as one group.
+__device__ __forceinline__ void store_tile_tma(const CUtensorMap* map, const unsigned char* cells, int run0,
+                                               int first, int n_runs) {
+    for (int r = first; r < first + n_runs; r += TMA_BOX_RUNS) {
         const unsigned int src = (unsigned int)__cvta_generic_to_shared(cells + ((size_t)r << 7));
         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                      :: "l"(map), "r"(0), "r"(run0 + r), "r"(src) : "memory");
@@ -666,6 +668,10 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
 
     const bool fast = a.chunk_off != nullptr;
     const bool tma = a.use_tma != 0;
+    // A tile of exactly two store boxes built by 512 threads: threads 0 and 256 each store one
+    // box, and each half of the block clears its half of the buffer as soon as ITS box has been
+    // read, while the other box may still be on its way out.
+    const bool split = tma && nthr == 512 && T * g.rpr == 2 * TMA_BOX_RUNS;
     const int trip = nthr;                        // chunks the block covers in one trip: one per thread
 
     // ---- once: an upper bound of every B of the table (the largest of the chunks' maxima)
@@ -700,9 +706,17 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         const unsigned long long beyond = tid < rows ? a.excess[row0 + tid] : 0ull;
 
         // ---- the cell buffer is free once the store that last used it has read it
-        if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(TILE_BUFFERS - 1) : "memory");
-        __syncthreads();
-        {
+        if (split) {
+            const int half = tid >> 8, t = tid & 255;
+            if (t == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            asm volatile("bar.sync %0, 256;" :: "r"(1 + half) : "memory");      // the eight warps of this half
+            uint4* z = reinterpret_cast<uint4*>(cells) + (size_t)half * (TMA_BOX_RUNS << 3);
+            for (int i = t; i < (TMA_BOX_RUNS << 3); i += 256) z[i] = make_uint4(0, 0, 0, 0);
+            if (tid < T) cur[tid] = 0ull;
+            if (tid == 0) { tile_records = 0; tile_max_b = 0; }
+        } else {
+            if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(TILE_BUFFERS - 1) : "memory");
+            __syncthreads();
             uint4* z = reinterpret_cast<uint4*>(cells);
             const int nz = a.buffer_runs << 3;
             for (int i = tid; i < nz; i += nthr) z[i] = make_uint4(0, 0, 0, 0);
@@ -773,7 +787,11 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
             if (tma) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stores above, for the copy unit
                 __syncthreads();
-                if (tid == 0) store_tile_tma(&out_map, cells, tile * (T * g.rpr), T * g.rpr);
+                if (split) {
+                    if ((tid & 255) == 0) store_tile_tma(&out_map, cells, tile * (T * g.rpr), (tid >> 8) * TMA_BOX_RUNS, TMA_BOX_RUNS);
+                } else if (tid == 0) {
+                    store_tile_tma(&out_map, cells, tile * (T * g.rpr), 0, T * g.rpr);
+                }
             } else {
                 __syncthreads();
                 // consecutive lanes on consecutive 16 bytes: the pair p of cells of the tile lies
@@ -856,7 +874,7 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         if (!fast && tid == 0) { a.bin_cursor[tile] = 0; a.bin_count[tile] = 0; }   // for the next call
     }
     // shared memory must outlive the copy unit's reads of it
-    if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    if (tma && (tid == 0 || (split && tid == 256))) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
 }  // namespace
