@@ -99,6 +99,16 @@ def test_anticipate_table_ordered_by_instance():
     st.close()
 
 
+def test_anticipate_more_chunks_than_a_tile_block_has_threads():
+    """300,000 requests are cut into 293 chunks while a tile block of this shape has 256 threads:
+    a thread gathers from more than one chunk per tile (only its first is looked ahead)."""
+    wl = W.make_random(22, 600, 1024, 300000, 0, max_prompt=2000, max_output=1500)
+    st, ref = both(wl)
+    assert_state_equal(st, ref)
+    assert st.status() == B.PRE_OK
+    st.close()
+
+
 def test_anticipate_tombstones_and_malformed():
     wl = W.make_random(13, 5, 40, 600, 0)
     wl.generated[::7] = wl.predicted[::7]          # finished: silently ignored
