@@ -709,6 +709,7 @@ pre_tile_build(const TileArgs a, const __grid_constant__ CUtensorMap out_map) {
         if (split) {
             const int half = tid >> 8, t = tid & 255;
             if (t == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncwarp();    // the one-lane wait above must not leave the warp split in front of an aligned barrier
             asm volatile("bar.sync %0, 256;" :: "r"(1 + half) : "memory");      // the eight warps of this half
             uint4* z = reinterpret_cast<uint4*>(cells) + (size_t)half * (TMA_BOX_RUNS << 3);
             for (int i = t; i < (TMA_BOX_RUNS << 3); i += 256) z[i] = make_uint4(0, 0, 0, 0);

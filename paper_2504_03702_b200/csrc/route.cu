@@ -358,16 +358,19 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     // over[r] (ADMIT): steps of row r above the overload level; 64 bytes of fixed words per row then, else 48
     int* over = rstate + a.max_rows;
     unsigned char* res = reinterpret_cast<unsigned char*>(rstate + (ADMIT ? 5 : 1) * a.max_rows);  // 16-byte aligned
-    __shared__ int sh_winner;
-    __shared__ double sh_score;
+    // Words that one warp writes for exchange s while others may still read those of s-1 are kept
+    // twice, indexed by the parity of the exchange (or of the arrival being scored): the writer of
+    // s+1 never touches what the readers of s use, and s+2 is written only after a block barrier.
+    __shared__ int sh_winner[2];
+    __shared__ double sh_score[2];
     __shared__ int sh_dead;
     __shared__ long long sh_n0;
     __shared__ long long sh_part[ROUTE_WARPS];  // per-warp peaks of the row that was just folded and re-scored
-    __shared__ double sh_best_s[2];  // the block's best and second-best score for the arrival being scored
-    __shared__ int sh_best_i[2];     // ... and their rows
+    __shared__ double sh_best_s[2][2];  // [parity][best, second best]: the block's best scores for the arrival being scored
+    __shared__ int sh_best_i[2][2];     // ... and their rows
     __shared__ int sh_cnt[ROUTE_WARPS];   // ADMIT: per-warp change of the folded row's overload count
     __shared__ int sh_n_over;             // ADMIT: rows of this block that are overloaded
-    __shared__ int sh_all_over;           // ADMIT: every block reported all its rows overloaded
+    __shared__ int sh_all_over[2];        // ADMIT: every block reported all its rows overloaded (by exchange parity)
     constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
 
     const int G = gridDim.x, b = blockIdx.x;
@@ -481,7 +484,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             int n = 0;
             for (int r = 0; r < nrows; ++r) n += (double)over[r] > a.many;
             sh_n_over = n;
-            sh_all_over = 0;
+            sh_all_over[0] = sh_all_over[1] = 0;
         }
         __syncthreads();
     }
@@ -580,12 +583,12 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 atomicExch(a.abort_flag, 1);
                 sh_dead = 1;
             }
-            sh_winner = bi;
-            sh_score = bs;
+            sh_winner[s & 1] = bi;
+            sh_score[s & 1] = bs;
         }
         if (ADMIT) {
             all_over = __all_sync(0xffffffffu, all_over) && !lost;
-            if (lane == 0) sh_all_over = all_over;
+            if (lane == 0) sh_all_over[s & 1] = all_over;
         }
     };
 
@@ -650,7 +653,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             a.generated[slot] = 0;
             a.predicted[slot] = pD;
             a.instance[slot] = w;
-            put_result(pidx, w, sh_score);
+            put_result(pidx, w, sh_score[(seq - 1) & 1]);
         }
     };
 
@@ -723,6 +726,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         if (warp == 0) {
             if (pending) gather(seq - 1);
         } else {
+            // an aligned barrier wants the whole warp: the loop above ends in a one-lane branch
+            __syncwarp();
             asm volatile("bar.sync 1, %0;" ::"n"(ROUTE_THREADS - 32) : "memory");
             if (warp == 1) {
                 double b1s = CUDART_INF, b2s = CUDART_INF;
@@ -745,29 +750,29 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                         b1s = o1s; b1i = o1i;
                     } else if (better(o1s, o1i, b2s, b2i)) { b2s = o1s; b2i = o1i; }
                 }
-                if (lane == 0) { sh_best_s[0] = b1s; sh_best_s[1] = b2s; sh_best_i[0] = b1i; sh_best_i[1] = b2i; }
+                if (lane == 0) { sh_best_s[buf][0] = b1s; sh_best_s[buf][1] = b2s; sh_best_i[buf][0] = b1i; sh_best_i[buf][1] = b2i; }
             } else {
                 for (int r = tid - 64; r < nrows; r += ROUTE_THREADS - 64) pk[(buf ^ 1) * a.max_rows + r] = I64_MIN;
             }
         }
         __syncthreads();  // B: winner of the pending arrival known to the block
         if (sh_dead) break;
-        if (ADMIT && pending && sh_all_over) { blocked = true; break; }   // the pending request is not routed
+        if (ADMIT && pending && sh_all_over[(seq - 1) & 1]) { blocked = true; break; }   // the pending request is not routed
 
         // ---- 3. fold the pending arrival (owner only), publish the block's best row for arrival k
-        const int w = sh_winner;
+        const int w = sh_winner[(seq - 1) & 1];   // exchange seq-1 decided the pending arrival
         const bool owner = pending && w >= row0 && w < row1;
         if (pending) settle(w, true, P, Dc);   // for the owner: ends with the folded row's peak in sh_part
         if (warp == 0) {
-            double b1s = sh_best_s[0];
-            int b1i = sh_best_i[0];
+            double b1s = sh_best_s[buf][0];
+            int b1i = sh_best_i[buf][0];
             if (owner) {
                 // the folded row's score changed: best = better(best of the other rows, folded row)
                 __syncwarp();   // lane 0 updated sq/scd of that row inside settle
                 const int r = w - row0;
                 const long long fixed_peak = warp_max64(sh_part[lane]);
                 const double s = score_of(sq[r], scd[r], fixed_peak, P, D, a.theta, a.beta);
-                if (b1i == w) { b1s = sh_best_s[1]; b1i = sh_best_i[1]; }
+                if (b1i == w) { b1s = sh_best_s[buf][1]; b1i = sh_best_i[buf][1]; }
                 if (better(s, w, b1s, b1i)) { b1s = s; b1i = w; }
             }
             if (lane == 0) {
@@ -793,8 +798,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         __syncthreads();
         if (warp == 0) gather(seq - 1);
         __syncthreads();
-        if (ADMIT && !sh_dead && sh_all_over) blocked = true;
-        if (!sh_dead && !blocked) settle(sh_winner, false, 0, 0);
+        if (ADMIT && !sh_dead && sh_all_over[(seq - 1) & 1]) blocked = true;
+        if (!sh_dead && !blocked) settle(sh_winner[(seq - 1) & 1], false, 0, 0);
     }
 
     if (b == 0 && tid == 0) {
