@@ -32,6 +32,9 @@ void release(pre_ctx* c) {
     cudaFree(c->d_scaler_done);
     cudaFree(c->d_ring_done);
     cudaFree(c->d_queue_entry);
+    for (int k = 0; k < 2; ++k) { cudaFree(c->d_fused_totals[k]); cudaFree(c->d_fused_hint[k]); }
+    cudaFree(c->d_fused_base);
+    cudaFree(c->d_fused_sync);
     delete c;
 }
 
@@ -86,14 +89,26 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_count, (size_t)c->n_tiles);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_base, (size_t)c->n_tiles + 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_bin_cursor, (size_t)c->n_tiles);
-    if (e == cudaSuccess) e = alloc_zero(&c->d_records, (size_t)cfg->max_requests + 16);   // read in windows of four
+    // records: read in windows of four; the fused build pads every tile's list to 16 bytes
+    // (the fused build keeps an eighth and 32 records of spare room per list)
+    const size_t record_slots = (size_t)cfg->max_requests + (size_t)cfg->max_requests / 4 + 40 * (size_t)c->n_tiles + 64;
+    if (e == cudaSuccess) e = alloc_zero(&c->d_records, record_slots);
+    c->fused_record_words = (unsigned int)(2 * record_slots < 0xfffffff0ull ? 2 * record_slots : 0xfffffff0ull);
+    for (int k = 0; k < 2; ++k) {
+        if (e == cudaSuccess) e = alloc_zero(&c->d_fused_totals[k], (size_t)c->n_tiles);
+        if (e == cudaSuccess) e = alloc_zero(&c->d_fused_hint[k], (size_t)c->n_tiles + 1);
+    }
+    if (e == cudaSuccess) e = alloc_zero(&c->d_fused_base, (size_t)c->n_tiles + 1);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_fused_sync, 8);
     if (e == cudaSuccess) e = alloc_zero(&c->d_enter, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_done, 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_ring_done, 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_queue_entry, 2);
+    c->spin_limit = PRE_DEFAULT_SPIN_LIMIT;
     if (e == cudaSuccess) e = pre_anticipate_configure(c);
+    if (e == cudaSuccess) e = pre_fused_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
     if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)32 * c->route_blocks);
     if (e != cudaSuccess) {
@@ -279,7 +294,13 @@ int pre_status(pre_ctx* ctx, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(int), s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail_cuda(ctx, e);
-    if (word & PRE_ST_TIMEOUT) return PRE_ETIMEOUT;
+    if (word & PRE_ST_TIMEOUT) {
+        // a build that gave up leaves its counters half-way: start them afresh
+        e = pre_fused_reset(ctx, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return fail_cuda(ctx, e);
+        return PRE_ETIMEOUT;
+    }
     if (word & PRE_ST_CAPACITY) return PRE_ECAPACITY;
     if (word & PRE_ST_BADREQ) return PRE_EBADREQ;
     return PRE_OK;

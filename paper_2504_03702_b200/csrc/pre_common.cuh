@@ -52,6 +52,18 @@ struct pre_ctx {
     long long* d_scaler_partial;    // [8 * n_sm][3] block totals of the scaler-signal kernel
     unsigned int* d_scaler_done;    // blocks of that kernel that have finished (zero between calls)
     unsigned int* d_ring_done;      // the same for the kernel that advances a ring of maps
+    // fused (single-launch) build: 0 blocks when this shape does not use it
+    int fused_grid;
+    size_t fused_smem;
+    unsigned int fused_bar_base;    // value of the grid-barrier counter before the next launch
+    unsigned int fused_launch_id;
+    unsigned int spin_limit;        // polls before a bounded device-side wait gives up
+    int fused_flip;                 // which of the two totals / hint arrays the next launch uses
+    unsigned int fused_record_words;   // room in d_records, in 4-byte words
+    unsigned int* d_fused_totals[2];   // [n_tiles] records per tile: one in use, the other zero for the next call
+    unsigned int* d_fused_hint[2];     // [n_tiles + 1] where the lengths of one build put the next build's lists
+    unsigned int* d_fused_base;     // [n_tiles + 1] where each tile's list starts when laid out exactly
+    unsigned int* d_fused_sync;     // [8] barrier counter, largest B, id of an abandoned launch
 };
 
 // Launchers (defined next to their kernels).  Each returns a cudaError_t.
@@ -96,6 +108,13 @@ int pre_tile_threads(int tile_rows, int horizon);
 int pre_sort_max_chunks(int64_t max_requests, int n_sm);
 size_t pre_chunk_table_words(int n_tiles, int max_chunks);
 cudaError_t pre_anticipate_configure(pre_ctx* ctx);
+cudaError_t pre_fused_configure(pre_ctx* ctx);   // sets ctx->fused_grid (0: this shape keeps the two-kernel build)
+bool pre_fused_fits(const pre_ctx* ctx, int64_t n);
+cudaError_t pre_launch_anticipate_fused(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
+                                        const int32_t* predicted, const int32_t* instance, int64_t n,
+                                        int64_t* curves, int64_t* current_d, cudaStream_t s);
+cudaError_t pre_fused_reset(pre_ctx* ctx, cudaStream_t s);   // after a wait ran out
+constexpr unsigned int PRE_DEFAULT_SPIN_LIMIT = 1u << 22;
 
 __device__ __forceinline__ bool pre_request_ok(int32_t P, int32_t g, int32_t D, int32_t inst, int32_t I) {
     return P >= 0 && g >= 0 && D >= 1 && inst >= 0 && inst < I;
