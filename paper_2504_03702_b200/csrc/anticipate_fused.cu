@@ -40,7 +40,7 @@ constexpr unsigned int REC4_B_BITS = 19;
 constexpr unsigned int REC4_B_MASK = (1u << REC4_B_BITS) - 1u;
 constexpr unsigned int FUSED_SPIN_LIMIT = 1u << 22;
 // words of `sync`
-constexpr int SYNC_BARRIER = 0, SYNC_MAX_B = 1, SYNC_ABORT = 2, SYNC_REDO = 3;
+constexpr int SYNC_BARRIER = 0, SYNC_MAX_B = 1, SYNC_ABORT = 2, SYNC_REDO = 3, SYNC_TILE = 4;
 
 struct FusedArgs {
     const int32_t* prompt;
@@ -68,7 +68,7 @@ struct FusedArgs {
     int64_t* current_d;
     int* status;
     int buffer_runs;              // runs of 128 bytes in the tile buffer (a multiple of 8)
-    int use_tma;
+    int use_tma;                  // 1: the tensor map of whole tiles describes `curves`; 2: so does the one of 32-run boxes
 };
 
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
@@ -204,12 +204,14 @@ __device__ __forceinline__ Quad load_quad(const FusedArgs& a, long long r0, int 
 }
 
 __global__ void __launch_bounds__(FUSED_THREADS, 2)
-pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) {
+pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, const __grid_constant__ CUtensorMap warp_map) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned int warp_tot[FUSED_THREADS / 32];
     __shared__ unsigned int sh_max_b;
     __shared__ int sh_flag;
     __shared__ int sh_lost;      // a bulk copy did not arrive in time: every thread leaves after the next barrier
+    __shared__ unsigned int sh_word[2];
+    __shared__ unsigned int sh_tile[2][4];   // {tile, start of its list, records} of the tile being built, by parity of the step
     __shared__ __align__(8) unsigned long long mbar;
 
     const TileGeom& g = a.g;
@@ -235,6 +237,7 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
     const bool vec = ((reinterpret_cast<uintptr_t>(a.prompt) | reinterpret_cast<uintptr_t>(a.generated) |
                        reinterpret_cast<uintptr_t>(a.predicted) | reinterpret_cast<uintptr_t>(a.instance)) & 15) == 0;
 
+    if (b == 0 && tid == 0) a.sync[SYNC_TILE] = 2u * (unsigned int)G;   // tiles are handed out from here after the barrier
     // two quads of table rows are always on their way while one is being packed
     Quad qa = load_quad(a, r0, rows_here, 0, vec);
     Quad qb = load_quad(a, r0, rows_here, 1, vec);
@@ -342,9 +345,15 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
     // =====================================================================================
     // Phase B, only when some piece did not fit (the first build of a context, a table that
     // changed a lot, 8-byte records): lay the lists out exactly, from the totals, and copy again.
-    const unsigned int largest = __ldcg(a.sync + SYNC_MAX_B);
+    // (one thread reads the two words every block needs: thousands of warps asking the same L2 line would queue up)
+    if (tid == 0) {
+        sh_word[0] = __ldcg(a.sync + SYNC_MAX_B);
+        sh_word[1] = __ldcg(a.sync + SYNC_REDO);
+    }
+    __syncthreads();
+    const unsigned int largest = sh_word[0];
     const bool fmt8 = largest > REC4_B_MASK;
-    const bool exact = __ldcg(a.sync + SYNC_REDO) == a.launch_id;
+    const bool exact = sh_word[1] == a.launch_id;
     if (exact) {
         for (int t = tid; t < n_tiles; t += nthr) {
             const unsigned int c = __ldcg(a.totals + t);
@@ -407,36 +416,26 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
     __syncthreads();
 
     // =====================================================================================
-    // Phase C: tiles.
+    // Phase C: tiles.  A block builds one tile after another; which tile comes next is decided
+    // by a global counter (the first two of a block are fixed), so blocks that run ahead take
+    // more.  Thread 0 looks a tile's list up one step before its bulk copy starts, and starts the
+    // copy one step before the tile is built.
     const unsigned int raw = (unsigned int)__cvta_generic_to_shared(smem_raw);
     unsigned char* cells = smem_raw + ((1024u - (raw & 1023u)) & 1023u);       // the swizzle pattern repeats every 1024 bytes
     const size_t buffer_bytes = (size_t)a.buffer_runs << 7;
     unsigned int* compact = reinterpret_cast<unsigned int*>(cells + buffer_bytes);                  // [buffer_runs * 16]
     unsigned int* landing = compact + ((size_t)a.buffer_runs << 4);                                 // [FUSED_LANDING_WORDS]
-    unsigned long long* cur = reinterpret_cast<unsigned long long*>(landing + FUSED_LANDING_WORDS); // [T]
-    unsigned long long* piece_s = cur + T;                                                          // [32]
+    unsigned long long* cur = reinterpret_cast<unsigned long long*>(landing + FUSED_LANDING_WORDS); // [2][T] by parity of the step
+    unsigned long long* piece_s = cur + 2 * T;                                                      // [32]
     unsigned int* piece_n = reinterpret_cast<unsigned int*>(piece_s + 32);                          // [32]
     const bool tma = a.use_tma != 0;
     const unsigned int mb = (unsigned int)__cvta_generic_to_shared(&mbar);
     const unsigned int landing_cap = fmt8 ? FUSED_LANDING_WORDS / 2 : FUSED_LANDING_WORDS;   // in records
     const unsigned int rec_words = fmt8 ? 2u : 1u;
-
-    // the lists of the block's first two tiles are looked up while the compact cells are cleared
-    unsigned int nx_first = 0, nx_count = 0;      // list of the tile after the one being built
-    int tile = b;
-    unsigned int first = 0, count = 0;
-    if (tile < n_tiles) {
-        first = __ldcg(list_at + tile);
-        count = __ldcg(a.totals + tile);
-        if (tile + G < n_tiles) { nx_first = __ldcg(list_at + tile + G); nx_count = __ldcg(a.totals + tile + G); }
-    }
-    for (int i = tid; i < (a.buffer_runs << 2); i += nthr) reinterpret_cast<uint4*>(compact)[i] = make_uint4(0, 0, 0, 0);
-    if (tid == 0) {
-        sh_lost = 0;
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mb) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
+    const int warp = tid >> 5;
+    // Tiles of whole rows of whole 32-run pieces, one run per thread: every warp stores its own
+    // 32 runs as soon as it has written them and waits only for its own previous store.
+    const bool warp_stores = a.use_tma == 2 && g.W == 32 && g.rpr == 32 * g.cpw && nthr == 32 * T * g.cpw;
 
     // thread 0: one bulk copy of records [first, first + count) of a list into the landing area
     auto fetch = [&](unsigned int first, unsigned int count) {
@@ -458,20 +457,56 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
         phase ^= 1u;
         return done != 0;
     };
+    auto drain_own_stores = [&]() {      // every warp: the copy unit has read what this warp's lane 0 gave it
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+    };
 
-    // thread 0 keeps the list of the block's next tile one step ahead
-    if (tid == 0 && tile < n_tiles && count) fetch(first, count < landing_cap ? count : landing_cap);
-    for (; tile < n_tiles; tile += G) {
-        const int row0 = tile << a.sh.tile_shift;
+    // thread 0 only: the tile after the one being built (its list known), and the one after that
+    unsigned int t1 = 0, f1 = 0, c1 = 0, t2 = 0;
+    if (tid == 0) {
+        sh_lost = 0;
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(mb) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const unsigned int t0 = (unsigned int)b;
+        unsigned int f0 = 0, c0 = 0;
+        t1 = (unsigned int)(b + G);
+        if (t0 < (unsigned int)n_tiles) { f0 = __ldcg(list_at + t0); c0 = __ldcg(a.totals + t0); }
+        if (t1 < (unsigned int)n_tiles) { f1 = __ldcg(list_at + t1); c1 = __ldcg(a.totals + t1); }
+        t2 = t1 < (unsigned int)n_tiles ? atomicAdd(a.sync + SYNC_TILE, 1u) : (unsigned int)n_tiles;
+        sh_tile[0][0] = t0; sh_tile[0][1] = f0; sh_tile[0][2] = c0;
+    }
+    for (int i = tid; i < (a.buffer_runs << 2); i += nthr) reinterpret_cast<uint4*>(compact)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < 2 * T; i += nthr) cur[i] = 0ull;
+    __syncthreads();
+    if (tid == 0 && sh_tile[0][0] < (unsigned int)n_tiles && sh_tile[0][2])
+        fetch(sh_tile[0][1], sh_tile[0][2] < landing_cap ? sh_tile[0][2] : landing_cap);
+
+    // the tile finished one step ago: its backlog words are written one step late, after a barrier
+    int prev_row0 = 0, prev_rows = 0;
+    unsigned long long prev_beyond = 0;
+    auto finish_previous = [&](int par) {
+        if (tid < prev_rows) {
+            a.current_d[prev_row0 + tid] = (int64_t)(cur[par * T + tid] + prev_beyond);
+            cur[par * T + tid] = 0ull;
+            if (prev_beyond) a.excess[prev_row0 + tid] = 0ull;     // for the next call
+        }
+    };
+
+    int it = 0;
+    for (;; ++it) {
+        const int par = it & 1;
+        const unsigned int tile = sh_tile[par][0];
+        if (tile >= (unsigned int)n_tiles) break;
+        const unsigned int first = sh_tile[par][1], count = sh_tile[par][2];
+        const int row0 = (int)tile << a.sh.tile_shift;
         const int rows = (a.sh.I - row0) < T ? (a.sh.I - row0) : T;
+        // current_d = sum over j of N[j] + what lies beyond the window (left there by phase A)
         const unsigned long long beyond = tid < rows ? __ldcg(a.excess + row0 + tid) : 0ull;
         const unsigned long long bound = (unsigned long long)count * ((largest > 32u ? largest : 32u) + (unsigned long long)H);
         const bool wide = bound >= (1ull << 32);
         const bool try_compact = !wide && !fmt8;
-        const unsigned long long* list8 = reinterpret_cast<const unsigned long long*>(a.records) + first;
-        const unsigned int* list4 = a.records + first;
-
-        for (int i = tid; i < T; i += nthr) cur[i] = 0ull;
+        unsigned long long* my_cur = cur + par * T;
 
         // ---- accumulate the list into the compact cells as it arrives
         bool overflow = false;
@@ -502,122 +537,177 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
                 }
             }
         }
-        // The previous tile's stores must have read the tile buffer before anybody writes it again.
-        // The compact scan only writes it after the barrier it has inside (rows of several pieces):
-        // the wait moves there, so that the first half of the scan overlaps the store.
-        const bool late_drain = tma && try_compact && g.cpw > 1;
-        if (tma && !late_drain && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        const bool redo = __syncthreads_or(overflow) != 0;
+        const bool redo = __syncthreads_or(overflow) != 0;       // barrier 1: the tile's cells are complete, the landing area is free
         if (sh_lost) break;
-        // the landing area is free: the next tile's list starts its way in; the one after is looked up
-        const unsigned int my_first = first, my_count = count;
-        first = nx_first; count = nx_count;
-        if (tid == 0 && tile + G < n_tiles && count) fetch(first, count < landing_cap ? count : landing_cap);
-        if (tile + 2 * G < n_tiles) { nx_first = __ldcg(list_at + tile + 2 * G); nx_count = __ldcg(a.totals + tile + 2 * G); }
-
-        auto for_each_record = [&](auto f) {       // f(cell, B) over the tile's whole list, from global memory
-            if (fmt8) {
-                for (unsigned int i = tid; i < my_count; i += nthr) {
-                    const unsigned long long rec = __ldcg(list8 + i);
-                    f((unsigned int)(rec >> 32), (unsigned int)rec);
-                }
-            } else {
-                for (unsigned int i = tid; i < my_count; i += nthr) {
-                    const unsigned int rec = __ldcg(list4 + i);
-                    f(rec >> REC4_B_BITS, rec & REC4_B_MASK);
-                }
+        if (tid == 0) {
+            // the next tile's list starts its way in; the one after is looked up; one more is claimed
+            sh_tile[par ^ 1][0] = t1; sh_tile[par ^ 1][1] = f1; sh_tile[par ^ 1][2] = c1;
+            if (t1 < (unsigned int)n_tiles && c1) fetch(f1, c1 < landing_cap ? c1 : landing_cap);
+            t1 = t2; f1 = 0; c1 = 0;
+            if (t1 < (unsigned int)n_tiles) {
+                f1 = __ldcg(list_at + t1); c1 = __ldcg(a.totals + t1);
+                t2 = atomicAdd(a.sync + SYNC_TILE, 1u);
             }
-        };
-        const bool whole = g.W == 32 && g.rpr == 32 * g.cpw && rows == T && nthr == 32 * T * g.cpw;
-
-        if (try_compact && !redo) {
-            if (whole) tile_scan_whole<true>(g.cpw, cells, compact, cur, reinterpret_cast<uint2*>(piece_s), late_drain);
-            else tile_scan_narrow<true>(g, rows, cells, compact, cur, piece_n, reinterpret_cast<unsigned int*>(piece_s), late_drain);
-        } else if (!wide) {
-            // ---- 64-bit cells {sum of B : 32 | count : 32}, accumulated and scanned in the tile buffer
-            if (redo) {
-                for (int i = tid; i < (a.buffer_runs << 2); i += nthr) reinterpret_cast<uint4*>(compact)[i] = make_uint4(0, 0, 0, 0);
-                if (late_drain) {
-                    if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    __syncthreads();
-                }
-            }
-            for (int i = tid; i < (a.buffer_runs << 3); i += nthr) reinterpret_cast<uint4*>(cells)[i] = make_uint4(0, 0, 0, 0);
-            __syncthreads();
-            for_each_record([&](unsigned int c, unsigned int B) {
-                unsigned int* w = reinterpret_cast<unsigned int*>(cells + cell_bytes(c));
-                atomicAdd(w, B);
-                atomicAdd(w + 1, 1u);
-            });
-            __syncthreads();
-            if (whole) tile_scan_whole<false>(g.cpw, cells, nullptr, cur, reinterpret_cast<uint2*>(piece_s), false);
-            else tile_scan_narrow<false>(g, rows, cells, nullptr, cur, piece_n, reinterpret_cast<unsigned int*>(piece_s), false);
-        } else {
-            // ---- wide mode: counts in the tile buffer, sums of B in the tile's rows of `curves`
-            for (int i = tid; i < (a.buffer_runs << 3); i += nthr) reinterpret_cast<uint4*>(cells)[i] = make_uint4(0, 0, 0, 0);
-            unsigned long long* gsum = reinterpret_cast<unsigned long long*>(a.curves) + (size_t)row0 * H;
-            for (int i = tid; i < rows * H; i += nthr) gsum[i] = 0ull;
-            __threadfence();
-            __syncthreads();
-            for_each_record([&](unsigned int c, unsigned int B) {
-                atomicAdd(reinterpret_cast<unsigned int*>(cells + cell_bytes(c)) + 1, 1u);
-                const unsigned int local = c / (unsigned int)hp;
-                atomicAdd(gsum + (size_t)local * H + (c - local * hp), (unsigned long long)B);
-            });
-            __threadfence();
-            __syncthreads();
-            tile_scan_wide(g, H, a.curves, row0, rows, cells, cur, piece_n, piece_s);
+            a.totals_next[tile] = 0;     // the next call counts into the other array
         }
+        finish_previous(par ^ 1);
 
-        // ---- the finished rows leave
-        if (wide) {
-            __syncthreads();
-        } else if (tma) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the scan's stores, for the copy unit
-            __syncthreads();
-            if (tid == 0) store_tile_tma(&out_map, cells, tile * (T * g.rpr), 0, T * g.rpr);
+        if (warp_stores && rows == T && try_compact && !redo) {
+            // ---- the usual case.  First half of the scan: this thread's run (cleared as it is read),
+            // its totals, the suffix scan over the runs of the warp's piece.
+            const unsigned int row = (unsigned int)warp / (unsigned int)g.cpw, piece = (unsigned int)warp - row * (unsigned int)g.cpw;
+            const unsigned int j0 = (piece * 32u + (unsigned int)lane) * RUN;
+            unsigned char* mine = cells + ((size_t)tid << 7);
+            const unsigned int sw = ((unsigned int)tid & 7u) << 4;          // piece i of the run lies at byte (i*16) ^ sw
+            uint4 v[RUN / 2];     // {sum, count, sum, count} of two cells
+            load_run<true>(v, cells, compact, (unsigned int)tid, true);
+            unsigned int tn = 0, ts = 0;
+            #pragma unroll
+            for (int i = 0; i < RUN / 2; ++i) { ts += v[i].x + v[i].z; tn += v[i].y + v[i].w; }
+            unsigned int xn = tn, xs = ts;
+            #pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned int yn = __shfl_down_sync(0xffffffffu, xn, off);
+                const unsigned int ys = __shfl_down_sync(0xffffffffu, xs, off);
+                if ((unsigned int)lane + off < 32u) { xn += yn; xs += ys; }
+            }
+            unsigned int N = xn - tn, A = xs - ts;
+            uint2* piece_tot = reinterpret_cast<uint2*>(piece_s);
+            if (lane == 0) piece_tot[warp] = make_uint2(xn, xs);
+            __syncthreads();     // barrier 2: every compact cell has been read and cleared; the pieces' totals are in place
+            for (unsigned int kk = piece + 1; kk < (unsigned int)g.cpw; ++kk) {
+                const uint2 t = piece_tot[(unsigned int)warp - piece + kk];
+                N += t.x; A += t.y;
+            }
+            drain_own_stores();  // this warp's 32 runs of the previous tile have left the buffer
+            // second half: from the run's last cell down, N[j], A[j], c[j] = A[j] + j * N[j]
+            unsigned int sn = 0;
+            #pragma unroll
+            for (int i = RUN / 2 - 1; i >= 0; --i) {
+                uint4 o;
+                N += v[i].w; A += v[i].z; sn += N;
+                o.z = A + N * (j0 + 2 * i + 1); o.w = 0;
+                N += v[i].y; A += v[i].x; sn += N;
+                o.x = A + N * (j0 + 2 * i); o.y = 0;
+                *reinterpret_cast<uint4*>(mine + ((i * 16) ^ sw)) = o;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these stores, for the copy unit
+            // sum over j of N[j] = sum over the row's requests of R: each is counted on R steps
+            const unsigned int lo = __reduce_add_sync(0xffffffffu, sn & 0xFFFFu);
+            const unsigned int hi = __reduce_add_sync(0xffffffffu, sn >> 16);
+            __syncwarp();        // every lane's stores and fence come before the one lane's copy
+            if (lane == 0) {
+                const unsigned int src = (unsigned int)__cvta_generic_to_shared(cells + ((size_t)(warp * 32) << 7));
+                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                             :: "l"(&warp_map), "r"(0), "r"((int)tile * (T * g.rpr) + warp * 32), "r"(src) : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                atomicAdd(&my_cur[row], ((unsigned long long)hi << 16) + lo);
+            }
         } else {
+            // ---- every other tile (a last tile of fewer rows, shapes without whole pieces, sums that
+            // do not fit the compact cells or 32 bits, 8-byte records): built and stored by the
+            // whole block, without overlap.
+            drain_own_stores();
             __syncthreads();
-            // consecutive lanes on consecutive 16 bytes: the pair p of cells of the tile lies
-            // at 16-byte word p ^ ((p >> 3) & 7) of the buffer
-            const int half = hp >> 1;               // cell pairs per padded row
-            const int total = rows * half;
-            const uint4* src = reinterpret_cast<const uint4*>(cells);
-            if (hp == H) {
-                ulonglong2* dst = reinterpret_cast<ulonglong2*>(a.curves + (size_t)row0 * H);
-                for (int p = tid; p < total; p += nthr) {
-                    const uint4 v = src[p ^ ((p >> 3) & 7)];
-                    dst[p] = make_ulonglong2(v.x, v.z);
+            const unsigned long long* list8 = reinterpret_cast<const unsigned long long*>(a.records) + first;
+            const unsigned int* list4 = a.records + first;
+            auto for_each_record = [&](auto f) {       // f(cell, B) over the tile's whole list, from global memory
+                if (fmt8) {
+                    for (unsigned int i = tid; i < count; i += nthr) {
+                        const unsigned long long rec = __ldcg(list8 + i);
+                        f((unsigned int)(rec >> 32), (unsigned int)rec);
+                    }
+                } else {
+                    for (unsigned int i = tid; i < count; i += nthr) {
+                        const unsigned int rec = __ldcg(list4 + i);
+                        f(rec >> REC4_B_BITS, rec & REC4_B_MASK);
+                    }
                 }
+            };
+            const bool whole = g.W == 32 && g.rpr == 32 * g.cpw && rows == T && nthr == 32 * T * g.cpw;
+            if (try_compact && !redo) {
+                if (whole) tile_scan_whole<true>(g.cpw, cells, compact, my_cur, reinterpret_cast<uint2*>(piece_s), false);
+                else tile_scan_narrow<true>(g, rows, cells, compact, my_cur, piece_n, reinterpret_cast<unsigned int*>(piece_s), false);
+            } else if (!wide) {
+                // 64-bit cells {sum of B : 32 | count : 32}, accumulated and scanned in the tile buffer
+                if (redo)
+                    for (int i = tid; i < (a.buffer_runs << 2); i += nthr) reinterpret_cast<uint4*>(compact)[i] = make_uint4(0, 0, 0, 0);
+                for (int i = tid; i < (a.buffer_runs << 3); i += nthr) reinterpret_cast<uint4*>(cells)[i] = make_uint4(0, 0, 0, 0);
+                __syncthreads();
+                for_each_record([&](unsigned int c, unsigned int B) {
+                    unsigned int* w = reinterpret_cast<unsigned int*>(cells + cell_bytes(c));
+                    atomicAdd(w, B);
+                    atomicAdd(w + 1, 1u);
+                });
+                __syncthreads();
+                if (whole) tile_scan_whole<false>(g.cpw, cells, nullptr, my_cur, reinterpret_cast<uint2*>(piece_s), false);
+                else tile_scan_narrow<false>(g, rows, cells, nullptr, my_cur, piece_n, reinterpret_cast<unsigned int*>(piece_s), false);
             } else {
-                const bool vec_gl = (H & 1) == 0;
-                for (int p = tid; p < total; p += nthr) {
-                    const int row = p / half;
-                    const int j = (p - row * half) << 1;
-                    if (j < H) {
+                // wide mode: counts in the tile buffer, sums of B in the tile's rows of `curves`
+                for (int i = tid; i < (a.buffer_runs << 3); i += nthr) reinterpret_cast<uint4*>(cells)[i] = make_uint4(0, 0, 0, 0);
+                unsigned long long* gsum = reinterpret_cast<unsigned long long*>(a.curves) + (size_t)row0 * H;
+                for (int i = tid; i < rows * H; i += nthr) gsum[i] = 0ull;
+                __threadfence();
+                __syncthreads();
+                for_each_record([&](unsigned int c, unsigned int B) {
+                    atomicAdd(reinterpret_cast<unsigned int*>(cells + cell_bytes(c)) + 1, 1u);
+                    const unsigned int local = c / (unsigned int)hp;
+                    atomicAdd(gsum + (size_t)local * H + (c - local * hp), (unsigned long long)B);
+                });
+                __threadfence();
+                __syncthreads();
+                tile_scan_wide(g, H, a.curves, row0, rows, cells, my_cur, piece_n, piece_s);
+            }
+            // the finished rows leave
+            if (wide) {
+                __syncthreads();
+            } else if (tma) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the scan's stores, for the copy unit
+                __syncthreads();
+                if (tid == 0) {
+                    store_tile_tma(&out_map, cells, (int)tile * (T * g.rpr), 0, T * g.rpr);
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                }
+                __syncthreads();
+            } else {
+                __syncthreads();
+                // consecutive lanes on consecutive 16 bytes: the pair p of cells of the tile lies
+                // at 16-byte word p ^ ((p >> 3) & 7) of the buffer
+                const int half = hp >> 1;               // cell pairs per padded row
+                const int total = rows * half;
+                const uint4* src = reinterpret_cast<const uint4*>(cells);
+                if (hp == H) {
+                    ulonglong2* dst = reinterpret_cast<ulonglong2*>(a.curves + (size_t)row0 * H);
+                    for (int p = tid; p < total; p += nthr) {
                         const uint4 v = src[p ^ ((p >> 3) & 7)];
-                        int64_t* dst = a.curves + ((size_t)(row0 + row) * H + j);
-                        if (vec_gl) {
-                            *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(v.x, v.z);
-                        } else {
-                            dst[0] = (int64_t)v.x;
-                            if (j + 1 < H) dst[1] = (int64_t)v.z;
+                        dst[p] = make_ulonglong2(v.x, v.z);
+                    }
+                } else {
+                    const bool vec_gl = (H & 1) == 0;
+                    for (int p = tid; p < total; p += nthr) {
+                        const int row = p / half;
+                        const int j = (p - row * half) << 1;
+                        if (j < H) {
+                            const uint4 v = src[p ^ ((p >> 3) & 7)];
+                            int64_t* dst = a.curves + ((size_t)(row0 + row) * H + j);
+                            if (vec_gl) {
+                                *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(v.x, v.z);
+                            } else {
+                                dst[0] = (int64_t)v.x;
+                                if (j + 1 < H) dst[1] = (int64_t)v.z;
+                            }
                         }
                     }
                 }
+                __syncthreads();     // the tile buffer is read before the next scan writes it
             }
-            __syncthreads();     // the tile buffer is read before the next scan writes it
         }
-        // current_d = sum over j of N[j] + what lies beyond the window (left by phase A; cleared
-        // for the next call).  cur[] is complete: a barrier followed the scan.
-        if (tid < rows) {
-            a.current_d[row0 + tid] = (int64_t)(cur[tid] + beyond);
-            if (beyond) a.excess[row0 + tid] = 0ull;
-        }
-        if (tid == 0) a.totals_next[tile] = 0;     // the next call counts into the other array
-        __syncthreads();         // cur[] is read before the next tile clears it
+        prev_row0 = row0; prev_rows = rows; prev_beyond = beyond;
     }
-    if (sh_lost && tid == 0) {
+    __syncthreads();
+    if (!sh_lost) {
+        if (it > 0) finish_previous((it - 1) & 1);
+    } else if (tid == 0) {
         atomicOr(a.status, PRE_ST_TIMEOUT);
         // the copy that did not arrive in time may still be on its way: give it one more bounded wait
         unsigned int done = 0, polls = 0;
@@ -626,7 +716,7 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map) 
                          : "=r"(done) : "r"(mb), "r"(phase ^ 1u) : "memory");
     }
     // shared memory must outlive the copy unit's reads of it
-    if (tma && tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    drain_own_stores();
 }
 
 }  // namespace
@@ -640,7 +730,7 @@ static size_t fused_smem_bytes(int tile_rows, int horizon, int n_tiles) {
     const size_t ntp = ((size_t)n_tiles + 4) & ~(size_t)3;
     const size_t phase_a = 3 * ntp * 4 + (size_t)FUSED_CHUNK_MAX * 12;
     const size_t phase_c = 1024 + buffer_runs * 128 + buffer_runs * 64 + (size_t)FUSED_LANDING_WORDS * 4 +
-                           (size_t)tile_rows * 8 + 32 * 8 + 32 * 4;
+                           (size_t)tile_rows * 16 + 32 * 8 + 32 * 4;
     return phase_a > phase_c ? phase_a : phase_c;
 }
 
@@ -718,9 +808,11 @@ cudaError_t pre_launch_anticipate_fused(pre_ctx* ctx, const int32_t* prompt, con
     a.spin_limit = ctx->spin_limit;
     a.excess = ctx->d_excess; a.curves = curves; a.current_d = current_d; a.status = ctx->d_status;
     a.buffer_runs = (T * a.g.rpr + 7) & ~7;
-    CUtensorMap out_map;
+    CUtensorMap out_map, warp_map;
     a.use_tma = make_out_map(&out_map, curves, I, H, T) ? 1 : 0;
-    void* params[] = {(void*)&a, (void*)&out_map};
+    if (a.use_tma && (T * a.g.rpr) % 32 == 0 && make_out_map(&warp_map, curves, I, H, T, 32)) a.use_tma = 2;
+    else memset(&warp_map, 0, sizeof(warp_map));
+    void* params[] = {(void*)&a, (void*)&out_map, (void*)&warp_map};
     return cudaLaunchCooperativeKernel((const void*)pre_build_fused, dim3(G), dim3(FUSED_THREADS), params,
                                        ctx->fused_smem, s);
 }

@@ -343,16 +343,16 @@ static encode_tiled_fn tensor_map_encoder() {
     return fn;
 }
 
-static bool make_out_map(CUtensorMap* map, int64_t* curves, int I, int H, int T) {
+static bool make_out_map(CUtensorMap* map, int64_t* curves, int I, int H, int T, int box_runs = TMA_BOX_RUNS) {
     memset(map, 0, sizeof(*map));
     if (H % RUN != 0) return false;
     const int runs_per_tile = T * (H / RUN);
-    if (runs_per_tile > TMA_BOX_RUNS && runs_per_tile % TMA_BOX_RUNS != 0) return false;
+    if (runs_per_tile > box_runs && runs_per_tile % box_runs != 0) return false;
     encode_tiled_fn enc = tensor_map_encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)RUN, (cuuint64_t)I * (cuuint64_t)(H / RUN)};
     const cuuint64_t strides[1] = {(cuuint64_t)RUN * sizeof(int64_t)};
-    const cuuint32_t box[2] = {(cuuint32_t)RUN, (cuuint32_t)(runs_per_tile < TMA_BOX_RUNS ? runs_per_tile : TMA_BOX_RUNS)};
+    const cuuint32_t box[2] = {(cuuint32_t)RUN, (cuuint32_t)(runs_per_tile < box_runs ? runs_per_tile : box_runs)};
     const cuuint32_t elem[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_INT64, 2, curves, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
