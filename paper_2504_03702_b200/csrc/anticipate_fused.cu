@@ -313,12 +313,21 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, 
         }
     }
     __syncthreads();
-    for (int idx = tid; idx < ((rows_here + 3) & ~3); idx += nthr) {
-        const unsigned int t16 = arr_t[idx];
-        if (t16 != 0xffffu) {
-            const unsigned int pos = atomicAdd(&cursor[t16], 1u);
-            sorted_r[pos] = arr_r[idx];
-            sorted_t[pos] = (unsigned short)t16;
+    for (int idx = tid; idx < ((rows_here + 3) & ~3); idx += 4 * nthr) {     // four rows at a time: their atomics overlap
+        unsigned int t16[4], pos[4];
+        #pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int at = idx + k * nthr;
+            t16[k] = at < FUSED_CHUNK_MAX ? arr_t[at] : 0xffffu;
+            pos[k] = 0;
+            if (t16[k] != 0xffffu) pos[k] = atomicAdd(&cursor[t16[k]], 1u);
+        }
+        #pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (t16[k] != 0xffffu) {
+                sorted_r[pos[k]] = arr_r[idx + k * nthr];
+                sorted_t[pos[k]] = (unsigned short)t16[k];
+            }
         }
     }
     __syncthreads();
@@ -493,6 +502,14 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, 
         }
     };
 
+    // where this thread's run is when every thread owns one (the usual case below)
+    const unsigned int row = (unsigned int)warp / (unsigned int)g.cpw, piece = (unsigned int)warp - row * (unsigned int)g.cpw;
+    const unsigned int j0 = (piece * 32u + (unsigned int)lane) * RUN;
+    unsigned char* const mine = cells + ((size_t)tid << 7);
+    const unsigned int sw = ((unsigned int)tid & 7u) << 4;          // piece i of the run lies at byte (i*16) ^ sw
+    const int tile_runs = T * g.rpr;
+    const unsigned long long per_record = (unsigned long long)(largest > 32u ? largest : 32u) + (unsigned long long)H;
+
     int it = 0;
     for (;; ++it) {
         const int par = it & 1;
@@ -503,8 +520,7 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, 
         const int rows = (a.sh.I - row0) < T ? (a.sh.I - row0) : T;
         // current_d = sum over j of N[j] + what lies beyond the window (left there by phase A)
         const unsigned long long beyond = tid < rows ? __ldcg(a.excess + row0 + tid) : 0ull;
-        const unsigned long long bound = (unsigned long long)count * ((largest > 32u ? largest : 32u) + (unsigned long long)H);
-        const bool wide = bound >= (1ull << 32);
+        const bool wide = (unsigned long long)count * per_record >= (1ull << 32);
         const bool try_compact = !wide && !fmt8;
         unsigned long long* my_cur = cur + par * T;
 
@@ -555,10 +571,6 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, 
         if (warp_stores && rows == T && try_compact && !redo) {
             // ---- the usual case.  First half of the scan: this thread's run (cleared as it is read),
             // its totals, the suffix scan over the runs of the warp's piece.
-            const unsigned int row = (unsigned int)warp / (unsigned int)g.cpw, piece = (unsigned int)warp - row * (unsigned int)g.cpw;
-            const unsigned int j0 = (piece * 32u + (unsigned int)lane) * RUN;
-            unsigned char* mine = cells + ((size_t)tid << 7);
-            const unsigned int sw = ((unsigned int)tid & 7u) << 4;          // piece i of the run lies at byte (i*16) ^ sw
             uint4 v[RUN / 2];     // {sum, count, sum, count} of two cells
             load_run<true>(v, cells, compact, (unsigned int)tid, true);
             unsigned int tn = 0, ts = 0;
@@ -599,7 +611,7 @@ pre_build_fused(const FusedArgs a, const __grid_constant__ CUtensorMap out_map, 
             if (lane == 0) {
                 const unsigned int src = (unsigned int)__cvta_generic_to_shared(cells + ((size_t)(warp * 32) << 7));
                 asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                             :: "l"(&warp_map), "r"(0), "r"((int)tile * (T * g.rpr) + warp * 32), "r"(src) : "memory");
+                             :: "l"(&warp_map), "r"(0), "r"((int)tile * tile_runs + warp * 32), "r"(src) : "memory");
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 atomicAdd(&my_cur[row], ((unsigned long long)hi << 16) + lo);
             }
