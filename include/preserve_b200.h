@@ -47,7 +47,8 @@ typedef enum pre_error {
     PRE_EINVAL = -1,    /* null or misaligned pointer, size out of range, bad config        */
     PRE_ECAPACITY = -2, /* request table full: the arrivals that did not fit were not routed */
     PRE_EBADREQ = -3,   /* a malformed request or arrival was skipped                        */
-    PRE_ETIMEOUT = -4,  /* a bounded device-side wait ran out; the batch was abandoned       */
+    PRE_ETIMEOUT = -4,  /* a bounded device-side wait ran out; the call stopped early (see   */
+                        /* pre_route_batch and pre_anticipate for what is left behind)       */
     PRE_ECUDA = -5,     /* a CUDA runtime call failed (see pre_last_cuda_error)              */
     PRE_ENOMEM = -6,    /* scratch allocation failed in pre_create                           */
     PRE_ESIZE = -7      /* problem larger than the built-in scratch of pre_anticipate_static */
@@ -130,7 +131,16 @@ int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d
  *     (P, 0, D, i*) is appended to the request table at index *d_n_requests, which advances.
  * d_choice[k] (int32) receives i*, or -1 if arrival k was malformed (P < 0, D < 1, either
  * >= 2^28) or did not fit in the table; d_score[k] (binary64, may be NULL) the winning L.
- * *d_n_requests is a DEVICE int64, read at the start and written at the end of the batch. */
+ * *d_n_requests is a DEVICE int64, read at the start and written at the end of the batch.
+ *
+ * The blocks of the routing kernel exchange their best instances through device memory and wait
+ * for one another a bounded number of polls.  If such a wait runs out (PRE_ETIMEOUT from
+ * pre_status; it should never happen on a GPU that runs the kernel alone), the blocks agree on
+ * the last arrival that every one of them had scored: arrivals up to that one are routed exactly
+ * as above (maps, queued_p, current_d, table and *d_n_requests all include them and nothing
+ * else), every later arrival gets PRE_CHOICE_DROPPED and score 0, and the context stays usable.
+ * Only if the blocks cannot even meet to agree (a second, much longer bounded wait) may the maps
+ * hold one request more than the table; rebuild them with pre_anticipate then. */
 int pre_route_batch(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted,
                     int64_t n_arrivals, int64_t* d_curves, int64_t* d_queued_p, int64_t* d_current_d,
                     int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
@@ -172,7 +182,9 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
  * d_choice[k] for the arrivals receive the instance index or one of the PRE_CHOICE_* values;
  * d_score[k] (may be NULL) the winning L of a routed arrival, 0 otherwise.  Entries that leave
  * the queue are a prefix of it.  Other arguments, errors and the status word as for
- * pre_route_batch; n_arrivals and queue_capacity below 2^30. */
+ * pre_route_batch; n_arrivals and queue_capacity below 2^30.  After a wait that ran out
+ * (PRE_ETIMEOUT) the requests decided so far are as described for pre_route_batch, waiting
+ * requests that were not reached keep their place and arrivals that were not reached are dropped. */
 int pre_route_admit(pre_ctx* ctx, const int32_t* d_arr_prompt, const int32_t* d_arr_predicted, int64_t n_arrivals,
                     double overload_level, double overload_share, int32_t* d_queue_prompt,
                     int32_t* d_queue_predicted, int64_t* d_queue_state, int64_t queue_capacity,
@@ -272,6 +284,13 @@ int pre_status(pre_ctx* ctx, void* stream);
 
 /* The cudaError_t value of the last failed runtime call on this context (0 if none). */
 int pre_last_cuda_error(const pre_ctx* ctx);
+
+/* Test hook, not part of the method: sets how many polls a device-side wait of this context's
+ * kernels makes before it gives up (default 2^22; 0 gives up at the first unsuccessful poll).
+ * It exists so that a test can make a wait run out without disturbing the GPU: nothing faults or
+ * spins for long, the kernels leave through their ordinary give-up path and pre_status returns
+ * PRE_ETIMEOUT. */
+int pre_test_set_spin_limit(pre_ctx* ctx, uint32_t polls);
 
 /* Static, human-readable text for a pre_error value. */
 const char* pre_strerror(int code);

@@ -17,7 +17,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
            "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step",
-           "pre_ring_refine")
+           "pre_ring_refine", "pre_test_set_spin_limit")
 
 
 class pre_config(C.Structure):
@@ -46,6 +46,7 @@ def _load():
     lib.pre_ring_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
     lib.pre_ring_refine.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
+    lib.pre_test_set_spin_limit.argtypes = [vp, C.c_uint32]
     lib.pre_last_cuda_error.argtypes = [vp]
     lib.pre_strerror.argtypes = [C.c_int]
     lib.pre_strerror.restype = C.c_char_p
@@ -173,6 +174,10 @@ def pre_ring_refine(ctx, prompt, generated, predicted, instance, actual, n_reque
 
 def pre_status(ctx, stream=None):
     return lib.pre_status(ctx, _stream() if stream is None else stream)
+
+
+def pre_test_set_spin_limit(ctx, polls):
+    return lib.pre_test_set_spin_limit(ctx, int(polls))
 
 
 def pre_last_cuda_error(ctx):

@@ -75,9 +75,9 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     c->n_tiles = (I + t - 1) / t;
     if (pre_tile_smem_bytes(t, H) > (size_t)prop.sharedMemPerBlockOptin) { delete c; return PRE_EINVAL; }
 
-    e = alloc_zero(&c->d_status, 4);
+    e = alloc_zero(&c->d_status, 8);     // status | give-up flag, agreed exchange, blocks met | . | exchange counter
     c->d_abort = c->d_status ? c->d_status + 1 : nullptr;
-    c->d_epoch = c->d_status ? reinterpret_cast<unsigned int*>(c->d_status + 2) : nullptr;
+    c->d_epoch = c->d_status ? reinterpret_cast<unsigned int*>(c->d_status + 5) : nullptr;
     if (e == cudaSuccess) {   // the slots start as zeros: the first tags must not be zero
         const unsigned int first = 2;
         e = cudaMemcpy(c->d_epoch, &first, sizeof(first), cudaMemcpyHostToDevice);
@@ -308,13 +308,19 @@ int pre_status(pre_ctx* ctx, void* stream) {
 
 int pre_last_cuda_error(const pre_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
+int pre_test_set_spin_limit(pre_ctx* ctx, uint32_t polls) {
+    if (!ctx) return PRE_EINVAL;
+    ctx->spin_limit = polls;
+    return PRE_OK;
+}
+
 const char* pre_strerror(int code) {
     switch (code) {
         case PRE_OK: return "ok";
         case PRE_EINVAL: return "invalid argument (null or misaligned pointer, size out of range)";
         case PRE_ECAPACITY: return "request table full: some arrivals were not routed";
         case PRE_EBADREQ: return "malformed request or arrival skipped";
-        case PRE_ETIMEOUT: return "a bounded device-side wait ran out; the batch was abandoned";
+        case PRE_ETIMEOUT: return "a bounded device-side wait ran out; the call stopped early";
         case PRE_ECUDA: return "CUDA runtime error";
         case PRE_ENOMEM: return "out of memory";
         case PRE_ESIZE: return "problem larger than the built-in scratch of pre_anticipate_static";

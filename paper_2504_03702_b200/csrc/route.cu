@@ -38,7 +38,7 @@ constexpr int ROUTE_WARPS = ROUTE_THREADS / 32;
 constexpr int SCAN_WARPS = ROUTE_WARPS - 1;  // warp 0 coordinates
 constexpr long long I64_MIN = (-9223372036854775807LL - 1);
 constexpr long long I64_MAX = 9223372036854775807LL;
-constexpr unsigned int SPIN_LIMIT = 1u << 22;  // polls before a wait is declared lost
+constexpr unsigned int ABORT_SPIN_LIMIT = 1u << 24;  // polls (with pauses) for the other blocks once a wait has run out
 constexpr int GATHER_ILP = 5;                  // exchange slots a lane polls at once
 // A block's exchange slot has a 128-byte line to itself: with several slots per line the
 // polling of 148 blocks and the stores of the line's owners contend, and one exchange takes
@@ -53,6 +53,11 @@ __device__ __forceinline__ void st_relaxed_v2(unsigned long long* p, unsigned lo
 }
 __device__ __forceinline__ void ld_relaxed_v2(const unsigned long long* p, unsigned long long& x, unsigned long long& y) {
     asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(x), "=l"(y) : "l"(p) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 __device__ __forceinline__ int ld_relaxed_s32(const int* p) {
     int v;
@@ -130,6 +135,9 @@ struct RouteArgs {
     unsigned int* epoch_ptr;  // running exchange counter kept on the device: tags stay dense across launches
     int* status;
     int* abort_flag;
+    unsigned int* abort_key;    // 0xffffffff - (smallest exchange number at which a block's wait ran out); 0: none
+    unsigned int* abort_count;  // blocks that have given up
+    unsigned int spin_limit;    // polls before a wait is declared lost
     int max_rows;       // ceil(I / G)
     size_t resident_bytes;  // shared memory per block left for resident rows
     // admission queue (ADMIT kernels only): a ring of waiting requests, entry q at (head + q) mod capacity
@@ -364,6 +372,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     __shared__ int sh_winner[2];
     __shared__ double sh_score[2];
     __shared__ int sh_dead;
+    __shared__ unsigned int sh_cut;   // after a lost wait: the last exchange that every block had published
+    __shared__ int sh_agreed;         // ... and whether all blocks met to agree on it
     __shared__ long long sh_n0;
     __shared__ long long sh_part[ROUTE_WARPS];  // per-warp peaks of the row that was just folded and re-scored
     __shared__ double sh_best_s[2][2];  // [parity][best, second best]: the block's best scores for the arrival being scored
@@ -531,7 +541,8 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     // loads suffice: tags are dense across launches (the counter lives on the device), so a
     // slot's previous content is always exactly two exchanges old.  All of a lane's slots are
     // polled at once.
-    auto gather = [&](long long s) {
+    // `once`: every slot is known to be there already; a missing one is an error, not a reason to wait.
+    auto gather = [&](long long s, bool once) {
         const unsigned int tag = epoch + (unsigned int)s;
         const unsigned long long tag16 = (unsigned long long)(tag & 0xffffu);
         const unsigned long long* slot = a.slots + (size_t)(tag & 1u) * G * SLOT_WORDS;
@@ -554,7 +565,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 for (int i = 0; i < GATHER_ILP; ++i) all &= (w[i][0] >> 48) == tag16 && (w[i][1] >> 48) == tag16;
                 if (__all_sync(0xffffffffu, all)) break;
                 ++polls;
-                const bool give_up = polls > SPIN_LIMIT || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag));
+                const bool give_up = once || polls > a.spin_limit || ((polls & 63u) == 0 && ld_relaxed_s32(a.abort_flag));
                 if (__any_sync(0xffffffffu, give_up)) { lost = true; break; }
                 if (polls > 256) __nanosleep(64);
             }
@@ -582,6 +593,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 atomicOr(a.status, PRE_ST_TIMEOUT);
                 atomicExch(a.abort_flag, 1);
                 sh_dead = 1;
+                if (once) sh_agreed = 0;
             }
             sh_winner[s & 1] = bi;
             sh_score[s & 1] = bs;
@@ -608,6 +620,31 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             int64_t* sp64 = reinterpret_cast<int64_t*>(res) + (size_t)r * H;
             long long pkv = I64_MIN;
             int crossed = 0;   // ADMIT: cells the fold takes above the overload level
+            // The usual case in few instructions (all 1,024 threads pass here while every other block
+            // waits for this one): a resident row of 32-bit cells that stays below 2^32 with both ramps
+            // added; two cells per thread, 32-bit arithmetic, one 16-byte store to the map.
+            const bool quick = !ADMIT && in_smem && packed && !evict &&
+                               bound[r] + pP + pDc + (long long)P + Dc < 0xffffffffLL;
+            if (quick) {
+                unsigned int pk32 = 0;
+                const int upto = rescore ? H : pDc;       // H is even here (packed rows have whole 64-cell chunks)
+                for (int j = 2 * tid; j < upto; j += 2 * ROUTE_THREADS) {
+                    uint2 v = *reinterpret_cast<const uint2*>(sp32 + j);
+                    if (j < pDc) {
+                        v.x += (unsigned int)(pP + j);
+                        if (j + 1 < pDc) v.y += (unsigned int)(pP + j + 1);
+                        *reinterpret_cast<uint2*>(sp32 + j) = v;
+                        *reinterpret_cast<ulonglong2*>(gp + j) = make_ulonglong2(v.x, v.y);
+                    }
+                    const unsigned int x = v.x + (j < Dc ? (unsigned int)(P + j) : 0u);
+                    const unsigned int y = v.y + (j + 1 < Dc ? (unsigned int)(P + j + 1) : 0u);
+                    pk32 = max(pk32, max(x, y));
+                }
+                if (rescore) {
+                    pk32 = __reduce_max_sync(0xffffffffu, pk32);
+                    if (lane == 0) sh_part[warp] = (long long)pk32;
+                }
+            } else
             for (int j = tid; j < (rescore ? H : pDc); j += ROUTE_THREADS) {
                 long long c = !in_smem ? __ldcg(gp + j) : packed ? (long long)sp32[j] : sp64[j];
                 if (j < pDc) {
@@ -622,7 +659,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
                 }
                 pkv = max64(pkv, j < Dc ? c + ((long long)P + j) : c);
             }
-            if (rescore) {   // one partial per warp, reduced by warp 0 after the barrier (no contended atomics)
+            if (rescore && !quick) {   // one partial per warp, reduced by warp 0 after the barrier (no contended atomics)
                 pkv = warp_max64(pkv);
                 if (lane == 0) sh_part[warp] = pkv;
             }
@@ -724,7 +761,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         //         best rows for arrival k.  Only the row that receives the pending arrival can still
         //         change, so for every other block the best row found here is final.
         if (warp == 0) {
-            if (pending) gather(seq - 1);
+            if (pending) gather(seq - 1, false);
         } else {
             // an aligned barrier wants the whole warp: the loop above ends in a one-lane branch
             __syncwarp();
@@ -796,20 +833,71 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     // ---- the last arrival is still pending
     if (pending && !sh_dead && !blocked) {
         __syncthreads();
-        if (warp == 0) gather(seq - 1);
+        if (warp == 0) gather(seq - 1, false);
         __syncthreads();
         if (ADMIT && !sh_dead && sh_all_over[(seq - 1) & 1]) blocked = true;
         if (!sh_dead && !blocked) settle(sh_winner[(seq - 1) & 1], false, 0, 0);
     }
 
+    // ---- A wait ran out, here or in another block (every block ends up here then: the block that
+    // gave up publishes nothing more, so nobody gets past the next exchange).  The blocks meet and
+    // agree on m, the smallest exchange at which any of them gave up.  Every block had published m
+    // before it could wait for it, so a block that gave up at m reads the slots of m once more, now
+    // complete, and settles m like the blocks that got one exchange further.  Requests up to the one
+    // of exchange m are routed and folded everywhere, nothing after it is.
+    const bool dead = sh_dead != 0;
+    long long settled = (dead || blocked) && pending ? seq - 1 : seq;    // requests really added, as this block sees it
+    long long undone_from = dead ? pidx : n_items;                       // first item that gets no decision
+    unsigned int next_epoch = epoch + (unsigned int)seq;
+    if (dead) {
+        const unsigned int lost_s = (unsigned int)(seq - 1);     // the exchange whose slots did not all arrive here
+        if (tid == 0) {
+            atomicMax(a.abort_key, 0xffffffffu - lost_s);
+            __threadfence();
+            atomicAdd(a.abort_count, 1u);
+            bool met = true;
+            unsigned int polls = 0;
+            while (ld_relaxed_u32(a.abort_count) < (unsigned int)G) {
+                if (++polls > ABORT_SPIN_LIMIT) { met = false; break; }
+                __nanosleep(200);
+            }
+            __threadfence();
+            sh_cut = 0xffffffffu - ld_relaxed_u32(a.abort_key);
+            sh_agreed = met ? 1 : 0;
+        }
+        __syncthreads();
+        const unsigned int m = sh_cut;
+        if (sh_agreed) {
+            next_epoch = epoch + m + 2u;      // past every tag this launch may have left in a slot
+            if (lost_s == m) {
+                if (warp == 0) gather((long long)m, true);
+                __syncthreads();
+                if (sh_agreed) {
+                    if (ADMIT && sh_all_over[m & 1]) {
+                        blocked = true;
+                    } else {
+                        settle(sh_winner[m & 1], false, 0, 0);
+                        settled = seq;
+                        undone_from = pidx + 1;
+                    }
+                }
+            }
+        }
+        // (without agreement - a block that never came - the maps may hold one request more than the
+        // table: PRE_ETIMEOUT then means that the state has to be rebuilt)
+    }
+
     if (b == 0 && tid == 0) {
-        // after a lost wait, or when it found every instance overloaded, the pending request was never settled
-        *a.n_requests = n0 + ((sh_dead || blocked) && pending ? seq - 1 : seq);
-        *a.epoch_ptr = epoch + (unsigned int)seq;
+        *a.n_requests = n0 + settled;
+        *a.epoch_ptr = next_epoch;
         // what the loop noted beyond a blocked request is decided again below and does not count here
         const long long decided = (ADMIT && blocked) ? pidx : n_items;
         if (saw_bad && (!ADMIT || first_bad < decided)) atomicOr(a.status, PRE_ST_BADREQ);
         if (saw_full && (!ADMIT || first_full < decided)) atomicOr(a.status, PRE_ST_CAPACITY);
+    }
+
+    if (!ADMIT && b == 0 && dead) {
+        for (long long k = undone_from + tid; k < n_items; k += ROUTE_THREADS) put_result(k, CHOICE_DROPPED, 0.0);
     }
 
     if (ADMIT && b == 0) {
@@ -819,8 +907,9 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
         // the other blocks only look at items up to the one they are scanning, whose fields they
         // read before the exchange that stopped the batch.
         __syncthreads();
-        const bool lost = sh_dead != 0;
-        const long long stop = blocked ? pidx : n_items;
+        const bool lost = dead;
+        // after a lost wait nothing more is decided: waiting requests keep their place, arrivals are dropped
+        const long long stop = blocked ? pidx : (lost ? undone_from : n_items);
         const long long left = stop < q_len ? q_len - stop : 0;          // waiting entries that stay
         for (long long k = stop + tid; k < q_len; k += ROUTE_THREADS) a.queue_choice[k] = CHOICE_WAITS;
         __shared__ long long sh_joined;
@@ -861,8 +950,12 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
             if (tid == 0) sh_joined += total;
             __syncthreads();
         }
-        if (tid == 0 && !lost) {
-            long long joined = sh_joined;
+        for (long long i = a0 + tid; i < a.n_arrivals && lost; i += ROUTE_THREADS) {
+            a.choice[i] = CHOICE_DROPPED;
+            if (a.score) a.score[i] = 0.0;
+        }
+        if (tid == 0) {
+            long long joined = lost ? 0 : sh_joined;
             if (left + joined > a.queue_capacity) joined = a.queue_capacity - left;
             a.queue_state[0] = a.queue_capacity > 0 ? (q_head + (q_len - left)) % a.queue_capacity : 0;
             a.queue_state[1] = left + joined;
@@ -933,6 +1026,9 @@ static void fill_route_args(RouteArgs& a, pre_ctx* ctx, const int32_t* arr_promp
     a.theta = ctx->theta; a.beta = ctx->cfg.beta;
     a.slots = ctx->d_slots; a.epoch_ptr = ctx->d_epoch;
     a.status = ctx->d_status; a.abort_flag = ctx->d_abort;
+    a.abort_key = reinterpret_cast<unsigned int*>(ctx->d_abort + 1);
+    a.abort_count = reinterpret_cast<unsigned int*>(ctx->d_abort + 2);
+    a.spin_limit = ctx->spin_limit;
     a.max_rows = (a.I + ctx->route_blocks - 1) / ctx->route_blocks;
     a.resident_bytes = ctx->route_resident_bytes;
     a.queue_prompt = nullptr; a.queue_predicted = nullptr; a.queue_state = nullptr; a.queue_entry = nullptr;
@@ -944,7 +1040,7 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
                              int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
                              int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
     if (n_arrivals == 0) return cudaSuccess;
-    cudaError_t e = cudaMemsetAsync(ctx->d_abort, 0, sizeof(int), s);
+    cudaError_t e = cudaMemsetAsync(ctx->d_abort, 0, 3 * sizeof(int), s);   // flag, agreed exchange, blocks met
     if (e != cudaSuccess) return e;
     RouteArgs a;
     fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
@@ -965,7 +1061,7 @@ cudaError_t pre_launch_route_admit(pre_ctx* ctx, const int32_t* arr_prompt, cons
     // new ones: they read a copy taken here, in stream order.
     cudaError_t e = cudaMemcpyAsync(ctx->d_queue_entry, queue_state, 2 * sizeof(int64_t), cudaMemcpyDeviceToDevice, s);
     if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(ctx->d_abort, 0, sizeof(int), s);
+    e = cudaMemsetAsync(ctx->d_abort, 0, 3 * sizeof(int), s);
     if (e != cudaSuccess) return e;
     RouteArgs a;
     fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
