@@ -299,6 +299,12 @@ const char* pre_strerror(int code);
  * persistent routing kernel and instance rows per build tile.  Either pointer may be NULL. */
 int pre_query(const pre_ctx* ctx, int32_t* route_blocks, int32_t* tile_rows);
 
+/* More of the same, for reports: out[0] = bytes of shared memory each block of the routing kernel
+ * has for resident map rows, out[1] = threads of a routing block, out[2] = blocks of the
+ * single-launch anticipator build (0 when this shape uses the two-kernel build), out[3] = the
+ * largest table (rows) that build takes. */
+int pre_query_layout(const pre_ctx* ctx, int64_t out[4]);
+
 #ifdef __cplusplus
 }
 #endif

@@ -17,7 +17,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
            "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step",
-           "pre_ring_refine", "pre_test_set_spin_limit")
+           "pre_ring_refine", "pre_test_set_spin_limit", "pre_query_layout")
 
 
 class pre_config(C.Structure):
@@ -51,6 +51,7 @@ def _load():
     lib.pre_strerror.argtypes = [C.c_int]
     lib.pre_strerror.restype = C.c_char_p
     lib.pre_query.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.pre_query_layout.argtypes = [vp, C.POINTER(C.c_int64)]
     for name in EXPORTS:
         if name != "pre_strerror":
             getattr(lib, name).restype = C.c_int
@@ -188,6 +189,12 @@ def pre_query(ctx):
     g, t = C.c_int32(), C.c_int32()
     code = lib.pre_query(ctx, C.byref(g), C.byref(t))
     return code, g.value, t.value
+
+
+def pre_query_layout(ctx):
+    out = (C.c_int64 * 4)()
+    code = lib.pre_query_layout(ctx, out)
+    return code, [int(v) for v in out]
 
 
 def check(code: int, where: str = "preserve_b200"):

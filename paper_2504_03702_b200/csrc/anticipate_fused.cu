@@ -783,9 +783,9 @@ cudaError_t pre_fused_configure(pre_ctx* ctx) {
 }
 
 // Whether the fused build can take a table of n rows on this context.
-bool pre_fused_fits(const pre_ctx* ctx, int64_t n) {
-    return ctx->fused_grid > 0 && n <= (int64_t)ctx->fused_grid * FUSED_CHUNK_MAX;
-}
+int64_t pre_fused_max_rows(const pre_ctx* ctx) { return (int64_t)ctx->fused_grid * FUSED_CHUNK_MAX; }
+
+bool pre_fused_fits(const pre_ctx* ctx, int64_t n) { return ctx->fused_grid > 0 && n <= pre_fused_max_rows(ctx); }
 
 cudaError_t pre_launch_anticipate_fused(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
                                         const int32_t* predicted, const int32_t* instance, int64_t n,

@@ -308,6 +308,15 @@ int pre_status(pre_ctx* ctx, void* stream) {
 
 int pre_last_cuda_error(const pre_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
+int pre_query_layout(const pre_ctx* ctx, int64_t out[4]) {
+    if (!ctx || !out) return PRE_EINVAL;
+    out[0] = (int64_t)ctx->route_resident_bytes;
+    out[1] = ctx->route_threads;
+    out[2] = ctx->fused_grid;
+    out[3] = pre_fused_max_rows(ctx);
+    return PRE_OK;
+}
+
 int pre_test_set_spin_limit(pre_ctx* ctx, uint32_t polls) {
     if (!ctx) return PRE_EINVAL;
     ctx->spin_limit = polls;

@@ -110,6 +110,7 @@ size_t pre_chunk_table_words(int n_tiles, int max_chunks);
 cudaError_t pre_anticipate_configure(pre_ctx* ctx);
 cudaError_t pre_fused_configure(pre_ctx* ctx);   // sets ctx->fused_grid (0: this shape keeps the two-kernel build)
 bool pre_fused_fits(const pre_ctx* ctx, int64_t n);
+int64_t pre_fused_max_rows(const pre_ctx* ctx);
 cudaError_t pre_launch_anticipate_fused(pre_ctx* ctx, const int32_t* prompt, const int32_t* generated,
                                         const int32_t* predicted, const int32_t* instance, int64_t n,
                                         int64_t* curves, int64_t* current_d, cudaStream_t s);
