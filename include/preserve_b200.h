@@ -230,6 +230,18 @@ int pre_scaler_signals(pre_ctx* ctx, const int64_t* d_curves, double overload_le
                        double idle_level, int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary,
                        void* stream);
 
+/* One scheduler tick in one call: pre_step, then (when d_actual is given) pre_refine against the
+ * real response lengths, then (when the three signal outputs are given) pre_scaler_signals on the
+ * maps as the first two leave them (Sec. 2, Sec. 4.3.1, Sec. 4.3.2).  Results are those of the three
+ * calls made one after the other, bit for bit; the table is read once and the maps are read and
+ * written once instead of twice and three times.  d_actual may be NULL (no refinement; d_counts is
+ * then zeroed if given).  d_over_count, d_row_max and d_summary are given together or all NULL.
+ * Every other argument as for the three calls. */
+int pre_tick(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+             const int32_t* d_actual, const int64_t* d_n_requests, int64_t* d_curves, int64_t* d_queued_p,
+             int64_t* d_current_d, double overload_level, double overload_share, double idle_level,
+             int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary, int64_t* d_counts, void* stream);
+
 /* Full-width maps (Sec. 4.3.1: the load-look-ahead map covers the next L iterations, L the
  * largest response the model can produce, e.g. 4,096; the load is projected over the next l
  * iterations, e.g. l = 100, for the router of Sec. 4.3.3).  A row is kept as a ring over

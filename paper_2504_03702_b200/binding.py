@@ -17,7 +17,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
            "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step",
-           "pre_ring_refine", "pre_test_set_spin_limit", "pre_query_layout")
+           "pre_ring_refine", "pre_test_set_spin_limit", "pre_query_layout", "pre_tick")
 
 
 class pre_config(C.Structure):
@@ -39,6 +39,7 @@ def _load():
     lib.pre_route_batch.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.pre_refine.argtypes = [vp] * 11
+    lib.pre_tick.argtypes = [vp] * 10 + [C.c_double] * 3 + [vp] * 5
     lib.pre_route_admit.argtypes = [vp, vp, vp, i64, C.c_double, C.c_double, vp, vp, vp, i64] + [vp] * 12
     lib.pre_scaler_signals.argtypes = [vp, vp, C.c_double, C.c_double, C.c_double, vp, vp, vp, vp]
     lib.pre_ring_window.argtypes = [vp, vp, C.c_int32, vp, vp, vp]
@@ -140,6 +141,14 @@ def pre_refine(ctx, prompt, generated, predicted, instance, actual, n_requests, 
     return lib.pre_refine(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(actual),
                           _ptr(n_requests), _ptr(curves), _ptr(current_d), _ptr(counts),
                           _stream() if stream is None else stream)
+
+
+def pre_tick(ctx, prompt, generated, predicted, instance, actual, n_requests, curves, queued_p, current_d,
+             overload_level, overload_share, idle_level, over_count, row_max, summary, counts, stream=None):
+    return lib.pre_tick(ctx, _ptr(prompt), _ptr(generated), _ptr(predicted), _ptr(instance), _ptr(actual),
+                        _ptr(n_requests), _ptr(curves), _ptr(queued_p), _ptr(current_d), float(overload_level),
+                        float(overload_share), float(idle_level), _ptr(over_count), _ptr(row_max), _ptr(summary),
+                        _ptr(counts), _stream() if stream is None else stream)
 
 
 def pre_scaler_signals(ctx, curves, overload_level, overload_share, idle_level, over_count, row_max, summary,

@@ -102,7 +102,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = alloc_zero(&c->d_fused_sync, 8);
     if (e == cudaSuccess) e = alloc_zero(&c->d_enter, (size_t)I);
     if (e == cudaSuccess) e = alloc_zero(&c->d_active, (size_t)I);
-    if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)8 * c->n_sm * 3);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_partial, (size_t)16 * c->n_sm * 3);
     if (e == cudaSuccess) e = alloc_zero(&c->d_scaler_done, 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_ring_done, 1);
     if (e == cudaSuccess) e = alloc_zero(&c->d_queue_entry, 2);
@@ -200,6 +200,29 @@ int pre_step(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
         return PRE_EINVAL;
     cudaError_t e = pre_launch_step(ctx, d_prompt, d_generated, d_predicted, d_instance, d_n_requests, d_curves,
                                     d_queued_p, d_current_d, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
+}
+
+int pre_tick(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_predicted, int32_t* d_instance,
+             const int32_t* d_actual, const int64_t* d_n_requests, int64_t* d_curves, int64_t* d_queued_p,
+             int64_t* d_current_d, double overload_level, double overload_share, double idle_level,
+             int32_t* d_over_count, int64_t* d_row_max, int64_t* d_summary, int64_t* d_counts, void* stream) {
+    if (!ctx || !d_prompt || !d_generated || !d_predicted || !d_instance || !d_n_requests || !d_curves ||
+        !d_queued_p || !d_current_d)
+        return PRE_EINVAL;
+    const int given = (d_over_count != nullptr) + (d_row_max != nullptr) + (d_summary != nullptr);
+    if (given != 0 && given != 3) return PRE_EINVAL;
+    if (given == 3 && (!std::isfinite(overload_level) || !std::isfinite(overload_share) || !std::isfinite(idle_level)))
+        return PRE_EINVAL;
+    if (!aligned(d_curves, 16) || !aligned(d_queued_p, 8) || !aligned(d_current_d, 8) || !aligned(d_n_requests, 8) ||
+        !aligned(d_prompt, 4) || !aligned(d_generated, 4) || !aligned(d_predicted, 4) || !aligned(d_instance, 4) ||
+        !aligned(d_actual, 4) || !aligned(d_over_count, 4) || !aligned(d_row_max, 8) || !aligned(d_summary, 8) ||
+        !aligned(d_counts, 8))
+        return PRE_EINVAL;
+    if (given == 0) { overload_level = 0.0; overload_share = 0.0; idle_level = 0.0; }
+    cudaError_t e = pre_launch_tick(ctx, d_prompt, d_generated, d_predicted, d_instance, d_actual, d_n_requests, d_curves,
+                                    d_queued_p, d_current_d, overload_level, overload_share, idle_level, d_over_count,
+                                    d_row_max, d_summary, d_counts, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? PRE_OK : fail_cuda(ctx, e);
 }
 

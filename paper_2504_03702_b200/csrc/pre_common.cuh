@@ -49,7 +49,7 @@ struct pre_ctx {
     unsigned long long* d_slots;    // [2][G][16] routing exchange, one 128-byte line per block and parity
     unsigned long long* d_enter;    // [I] tokens entering the window at step H-1 (zero between calls)
     unsigned int* d_active;         // [I] live requests per instance (zero between calls)
-    long long* d_scaler_partial;    // [8 * n_sm][3] block totals of the scaler-signal kernel
+    long long* d_scaler_partial;    // [16 * n_sm][3] block totals of the kernels that sum the scaler's signals
     unsigned int* d_scaler_done;    // blocks of that kernel that have finished (zero between calls)
     unsigned int* d_ring_done;      // the same for the kernel that advances a ring of maps
     // fused (single-launch) build: 0 blocks when this shape does not use it
@@ -91,6 +91,10 @@ cudaError_t pre_launch_refine(pre_ctx* ctx, const int32_t* prompt, const int32_t
 cudaError_t pre_launch_scaler(pre_ctx* ctx, const int64_t* curves, double overload_level, double overload_share,
                               double idle_level, int32_t* over_count, int64_t* row_max, int64_t* summary,
                               cudaStream_t s);
+cudaError_t pre_launch_tick(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                            const int32_t* actual, const int64_t* n_requests, int64_t* curves, int64_t* queued_p,
+                            int64_t* current_d, double overload_level, double overload_share, double idle_level,
+                            int32_t* over_count, int64_t* row_max, int64_t* summary, int64_t* counts, cudaStream_t s);
 cudaError_t pre_launch_step_requests(pre_ctx* ctx, int32_t* prompt, int32_t* generated, int32_t* predicted,
                                      int32_t* instance, const int64_t* n_requests, int width, cudaStream_t s);
 cudaError_t pre_launch_ring_window(pre_ctx* ctx, const int64_t* ring, int width, const int64_t* head,

@@ -106,6 +106,20 @@ class DeviceState:
                                      row_max, summary), "pre_scaler_signals")
         return over, row_max, summary
 
+    def tick(self, actual=None, signals=True, overload_level=0.95, overload_share=0.10, idle_level=0.30):
+        """pre_tick: decode step, refinement against `actual` (if given) and scaler signals (if wanted) in one call.
+        Returns (counts int64[3] or None, over_count, row_max, summary) as device tensors (None where not asked)."""
+        counts = torch.empty(3, dtype=torch.int64, device=self.device) if actual is not None else None
+        over = row_max = summary = None
+        if signals:
+            over = torch.empty(self.I, dtype=torch.int32, device=self.device)
+            row_max = torch.empty(self.I, dtype=torch.int64, device=self.device)
+            summary = torch.empty(3, dtype=torch.int64, device=self.device)
+        B.check(B.pre_tick(self.ctx, self.prompt, self.generated, self.predicted, self.instance, actual,
+                           self.n_requests, self.curves, self.queued_p, self.current_d, overload_level,
+                           overload_share, idle_level, over, row_max, summary, counts), "pre_tick")
+        return counts, over, row_max, summary
+
     # ---- full-width maps kept as a ring (the state's own maps are then the window of width H = l)
 
     def make_ring(self, width, builder=None):
