@@ -18,7 +18,7 @@
 
 namespace {
 
-constexpr int TICK_THREADS = 256;
+constexpr int TICK_THREADS = 512;
 constexpr int TICK_WARPS = TICK_THREADS / 32;
 constexpr int SHIFT_THREADS = 256;
 constexpr int SHIFT_WARPS = SHIFT_THREADS / 32;
@@ -39,7 +39,7 @@ pre_tick_requests(const int32_t* __restrict__ prompt, int32_t* __restrict__ gene
                   const int64_t* __restrict__ n_requests, long long max_requests, int I, int H,
                   int64_t* __restrict__ curves, int64_t* __restrict__ current_d, unsigned int* __restrict__ active,
                   unsigned long long* __restrict__ enter, unsigned long long* __restrict__ counts,
-                  int* __restrict__ status) {
+                  long long* __restrict__ summary, int* __restrict__ status) {
     extern __shared__ unsigned int sh_active[];
     __shared__ unsigned int sh_tally[3];
     const bool use_sh = I <= PRE_SMEM_BINS;
@@ -48,6 +48,7 @@ pre_tick_requests(const int32_t* __restrict__ prompt, int32_t* __restrict__ gene
     if (use_sh)
         for (int i = threadIdx.x; i < I; i += blockDim.x) sh_active[i] = 0;
     if (threadIdx.x < 3) sh_tally[threadIdx.x] = 0;
+    if (summary && blockIdx.x == 0 && threadIdx.x < 3) summary[threadIdx.x] = 0;   // the map pass adds its block totals
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool vec = ((reinterpret_cast<uintptr_t>(prompt) | reinterpret_cast<uintptr_t>(generated) |
@@ -179,15 +180,24 @@ __global__ void __launch_bounds__(SHIFT_THREADS)
 pre_tick_shift(int64_t* __restrict__ curves, int64_t* __restrict__ queued_p, int64_t* __restrict__ current_d,
                unsigned int* __restrict__ active, unsigned long long* __restrict__ enter, int I, int H,
                long long hot, double many, double idle, int32_t* __restrict__ over_count,
-               int64_t* __restrict__ row_max, long long* __restrict__ summary, long long* __restrict__ partial,
-               unsigned int* __restrict__ done) {
-    __shared__ int sh_cnt[SHIFT_WARPS];
-    __shared__ long long sh_max[SHIFT_WARPS];
-    __shared__ bool sh_last;
+               int64_t* __restrict__ row_max, long long* __restrict__ summary) {
+    __shared__ int sh_cnt[2][SHIFT_WARPS];          // per-warp partials of a row, by parity of the block's row count:
+    __shared__ long long sh_max[2][SHIFT_WARPS];    // thread 0 adds them up one row later, after the barrier that ends the row
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool signals = summary != nullptr;
     long long n_over = 0, n_busy = 0, sum = 0;     // thread 0 only
-    for (int row = blockIdx.x; row < I; row += gridDim.x) {
+    auto close_row = [&](int row, int par) {       // thread 0: the signals of a row whose partials are complete
+        int c = 0;
+        long long m = I64_MIN;
+        for (int w = 0; w < SHIFT_WARPS; ++w) { c += sh_cnt[par][w]; m = sh_max[par][w] > m ? sh_max[par][w] : m; }
+        over_count[row] = c;
+        row_max[row] = m;
+        n_over += (double)c > many;
+        n_busy += !((double)m < idle);
+        sum += m;
+    };
+    int it = 0;
+    for (int row = blockIdx.x; row < I; row += gridDim.x, ++it) {
         int64_t* rp = curves + (size_t)row * H;
         const long long last = (long long)enter[row];
         int cnt = 0;
@@ -214,49 +224,23 @@ pre_tick_shift(int64_t* __restrict__ curves, int64_t* __restrict__ queued_p, int
         if (signals) {
             cnt = __reduce_add_sync(0xffffffffu, cnt);
             mx = warp_max64(mx);
-            if (lane == 0) { sh_cnt[warp] = cnt; sh_max[warp] = mx; }
-            __syncthreads();
+            if (lane == 0) { sh_cnt[it & 1][warp] = cnt; sh_max[it & 1][warp] = mx; }
         }
         if (threadIdx.x == 0) {
             current_d[row] -= (long long)active[row];
             queued_p[row] = 0;
             active[row] = 0;
             enter[row] = 0;
-            if (signals) {
-                int c = 0;
-                long long m = I64_MIN;
-                for (int w = 0; w < SHIFT_WARPS; ++w) { c += sh_cnt[w]; m = sh_max[w] > m ? sh_max[w] : m; }
-                over_count[row] = c;
-                row_max[row] = m;
-                n_over += (double)c > many;
-                n_busy += !((double)m < idle);
-                sum += m;
-            }
+            if (signals && it > 0) close_row(row - (int)gridDim.x, (it - 1) & 1);
         }
         __syncthreads();
     }
-    if (!signals) return;
-    if (threadIdx.x == 0) {
-        partial[blockIdx.x * 3 + 0] = n_over;
-        partial[blockIdx.x * 3 + 1] = n_busy;
-        partial[blockIdx.x * 3 + 2] = sum;
-        __threadfence();
-        sh_last = atomicAdd(done, 1u) == gridDim.x - 1;
-    }
-    __syncthreads();
-    if (sh_last && threadIdx.x < 32) {   // every other block's totals are visible (fence before its count)
-        __threadfence();
-        long long o = 0, b = 0, s = 0;
-        for (int g = lane; g < (int)gridDim.x; g += 32) {
-            o += __ldcg(&partial[g * 3 + 0]); b += __ldcg(&partial[g * 3 + 1]); s += __ldcg(&partial[g * 3 + 2]);
-        }
-        #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            o += __shfl_xor_sync(0xffffffffu, o, off);
-            b += __shfl_xor_sync(0xffffffffu, b, off);
-            s += __shfl_xor_sync(0xffffffffu, s, off);
-        }
-        if (lane == 0) { summary[0] = o; summary[1] = b; summary[2] = s; *done = 0; }   // ready for the next call
+    if (signals && threadIdx.x == 0) {
+        if (it > 0) close_row(blockIdx.x + (it - 1) * (int)gridDim.x, (it - 1) & 1);
+        // integer sums into words that the table pass cleared: no fence, no waiting for the block's stores
+        if (n_over) atomicAdd(reinterpret_cast<unsigned long long*>(summary), (unsigned long long)n_over);
+        if (n_busy) atomicAdd(reinterpret_cast<unsigned long long*>(summary) + 1, (unsigned long long)n_busy);
+        if (sum) atomicAdd(reinterpret_cast<unsigned long long*>(summary) + 2, (unsigned long long)sum);
     }
 }
 
@@ -273,12 +257,13 @@ cudaError_t pre_launch_tick(pre_ctx* ctx, int32_t* prompt, int32_t* generated, i
     }
     const size_t smem = I <= PRE_SMEM_BINS ? (size_t)I * sizeof(unsigned int) : 0;
     long long want = (ctx->cfg.max_requests + TICK_THREADS * 4 - 1) / (TICK_THREADS * 4);
-    int grid = (int)(want < 4LL * ctx->n_sm ? want : 4LL * ctx->n_sm);
+    // two blocks per SM: every block flushes its live counts with one global atomic per instance
+    int grid = (int)(want < 2LL * ctx->n_sm ? want : 2LL * ctx->n_sm);
     if (grid < 1) grid = 1;
     pre_tick_requests<<<grid, TICK_THREADS, smem, s>>>(prompt, generated, predicted, instance, actual, n_requests,
                                                       ctx->cfg.max_requests, I, H, curves, current_d, ctx->d_active,
                                                       ctx->d_enter, reinterpret_cast<unsigned long long*>(counts),
-                                                      ctx->d_status);
+                                                      reinterpret_cast<long long*>(summary), ctx->d_status);
     // For a whole number c, c > x holds exactly when c > floor(x): the per-cell test is done on integers.
     double hot_d = floor(overload_level * (double)ctx->cfg.capacity_tokens);
     if (hot_d > 9.2e18) hot_d = 9.2e18;
@@ -288,7 +273,6 @@ cudaError_t pre_launch_tick(pre_ctx* ctx, int32_t* prompt, int32_t* generated, i
     int sgrid = I < 16 * ctx->n_sm ? I : 16 * ctx->n_sm;
     pre_tick_shift<<<sgrid, SHIFT_THREADS, 0, s>>>(curves, queued_p, current_d, ctx->d_active, ctx->d_enter, I, H,
                                                   (long long)hot_d, many, idle, over_count, row_max,
-                                                  reinterpret_cast<long long*>(summary), ctx->d_scaler_partial,
-                                                  ctx->d_scaler_done);
+                                                  reinterpret_cast<long long*>(summary));
     return cudaGetLastError();
 }
