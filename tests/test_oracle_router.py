@@ -195,3 +195,50 @@ def test_step_after_route_on_tiny_config():
     n = int(s.n[0])
     ref = brute_curves(s.prompt[:n], s.generated[:n], s.predicted[:n], s.instance[:n], 8, 64)
     assert (s.curves == ref).all()
+
+
+# ---------------------------------------------------------------- admission of the running-maxima mode on the large configurations
+
+def _clone(s):
+    import copy
+    return copy.deepcopy(s)
+
+
+@pytest.mark.slow
+def test_identity_mode_on_a_prefix_of_the_large_configuration():
+    """The expected values of the largest configuration come from the running-maxima mode (the literal mode
+    needs hours there): on its first 512 arrivals the two modes must agree bit for bit."""
+    wl = W.make_config(3)
+    a = fresh(wl)
+    b = _clone(a)
+    ap, ad = wl.ticks[0][0][:512], wl.ticks[0][1][:512]
+    ca, sa = a.route_batch(ap, ad)
+    cb, sb = b.route_batch(ap, ad, fast=True)
+    assert (ca == cb).all() and (sa == sb).all()
+    assert (a.curves == b.curves).all() and (a.queued_p == b.queued_p).all() and (a.current_d == b.current_d).all()
+    assert (a.instance[:int(a.n[0])] == b.instance[:int(b.n[0])]).all()
+    # and with the admission queue (levels at which some arrivals of the prefix find every instance overloaded
+    # are not reached here: the rule must then route exactly like the plain router, in both modes)
+    c, d = _clone(b), _clone(b)
+    ap2, ad2 = wl.ticks[0][0][512:768], wl.ticks[0][1][512:768]
+    c.make_queue(64)
+    d.make_queue(64)
+    rc = c.route_admit(ap2, ad2, overload_level=0.95, overload_share=0.10)
+    rd = d.route_admit(ap2, ad2, overload_level=0.95, overload_share=0.10, fast=True)
+    for x, y in zip(rc, rd):
+        assert (np.asarray(x) == np.asarray(y)).all()
+    assert (c.curves == d.curves).all() and (c.queue_state == d.queue_state).all()
+
+
+@pytest.mark.slow
+def test_identity_mode_on_the_first_streaming_ticks():
+    wl = W.make_config(4, n_ticks=2)
+    a = fresh(wl)
+    b = _clone(a)
+    for ap, ad in wl.ticks:
+        a.step()
+        b.step()
+        ca, sa = a.route_batch(ap, ad)
+        cb, sb = b.route_batch(ap, ad, fast=True)
+        assert (ca == cb).all() and (sa == sb).all()
+    assert (a.curves == b.curves).all() and (a.queued_p == b.queued_p).all() and (a.current_d == b.current_d).all()

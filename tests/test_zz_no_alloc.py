@@ -5,8 +5,10 @@ pool allocator owns the whole GPU, under the allocator's lock, or in a control l
 not risk the device-wide synchronisation an allocation can bring.  For them the library
 carries its scratch inside its own image and exposes one entry point that needs no context.
 This file checks, through the C-ABI, that it computes exactly what pre_anticipate computes
-(int64 maps and backlogs, bit for bit), on two calls in a row that share the built-in
-scratch, and that it refuses problems larger than that scratch.
+(int64 maps and backlogs, bit for bit) and what the CPU oracle computes, on calls in a row that
+share the built-in scratch, and that it refuses problems larger than that scratch.  (The allocation
+check sees torch's allocator only; that the entry point itself requests no memory is a property of
+its source, which calls no allocating routine.)
 
 It is collected last on purpose (see conftest.py): if it fails, every other test has run.
 """
@@ -16,6 +18,7 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
+import oracle  # noqa: E402
 from paper_2504_03702_b200 import binding as B  # noqa: E402
 from paper_2504_03702_b200 import workloads as W  # noqa: E402
 from paper_2504_03702_b200.state import DeviceState  # noqa: E402
@@ -52,6 +55,11 @@ def test_two_calls_in_a_row_match_the_context_path():
         assert torch.equal(curves, want_curves)
         assert torch.equal(current_d, want_d)
         assert int(flags.item()) == 0
+        # and both against the definition written out on the CPU, not only against each other
+        ref = oracle.State.from_workload(wl)
+        ref.anticipate()
+        assert (curves.cpu().numpy() == ref.curves).all()
+        assert (current_d.cpu().numpy() == ref.current_d).all()
         st.close()
 
 
