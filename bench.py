@@ -34,17 +34,20 @@ import numpy as np  # noqa: E402
 METRIC = "routes/sec over the whole step (anticipate + route batch + decode step)"
 METRIC_STREAM = "routes/sec over the whole stream (decode step + routing of the tick's arrivals, per tick)"
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configuration 3;
-# other configurations report null).  The routing kernel reads the maps once per launch (whatever the
-# batch length) and writes 655 B per arrival (folded cells, appended requests): the written part is scaled
-# to the batch.  The fused build reads the table and writes the tiles' lists; most of the 64 MiB of maps is
-# still in L2 when the launch ends, which is why its figure is below the algorithmic bytes.
-ROUTE_DRAM_READ = {3: 67312384}
-ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 655}
-ANTICIPATE_DRAM_TRAFFIC = {3: 33697280 + 17827840}
-STEP_DRAM_TRAFFIC = {3: 76922880 + 10365952}
-SCALER_DRAM_TRAFFIC = {3: 67150848}
-REFINE_DRAM_TRAFFIC = {3: None}
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configuration 3; other
+# configurations report null).  profiles/ncu_full_step_kernels_config3_256_arrivals.txt: the routing kernel
+# reads the maps once per launch, whatever the batch length (67.31 MB), and wrote 420,864 B for 256 arrivals
+# (folded cells, appended requests): the written part is scaled to the batch.  The single-launch build reads the
+# table and moves the tiles' lists; most of the 64 MiB of maps is still in L2 when the launch ends, which is why
+# its figure is below the algorithmic bytes.  pre_step: its two kernels added.
+# profiles/ncu_full_tick_scaler_refine_config3.txt: refinement and the fused tick (two kernels added).
+ROUTE_DRAM_READ = {3: 67314944}
+ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 420864 / 256}
+ANTICIPATE_DRAM_TRAFFIC = {3: 33807872 + 20073216}
+STEP_DRAM_TRAFFIC = {3: 33640192 + 67196160 + 8895232}
+SCALER_DRAM_TRAFFIC = {3: None}
+REFINE_DRAM_TRAFFIC = {3: 44149248 + 40192}
+TICK_DRAM_TRAFFIC = {3: 44138240 + 50944 + 67200000 + 8971776}
 
 
 def measured_peak_gbs():
@@ -480,7 +483,7 @@ def extras_leg(res, wl, index, device):
             tk_ev.append((e0, e1))
         torch.cuda.synchronize()
         t_tick = float(np.median([x.elapsed_time(y) for x, y in tk_ev[1:]]))
-        out["tick_fused"] = {"tick_fused_ms": t_tick, "pre_step_alone_ms": t_step_here,
+        out["tick_fused"] = {"tick_fused_ms": t_tick, "pre_step_alone_ms": t_step_here, "traffic": TICK_DRAM_TRAFFIC.get(index),
                              "separate_calls_ms": {"pre_step": t_step_here, "pre_refine": t_refine, "pre_scaler_signals": t_scaler},
                              "ratio_to_pre_step": t_tick / t_step_here,
                              "note": "pre_tick: decode step, refinement against real lengths and scaler signals in one pass "
@@ -599,7 +602,7 @@ def route_roofline(wl, index, t_route_ms, n_arrivals, map_max, layout, route_blo
     literal = n_arrivals * (8 * i * h + 16 * h + 16 * i)
     traffic = None
     if index in ROUTE_DRAM_READ:
-        traffic = ROUTE_DRAM_READ[index] + ROUTE_DRAM_WRITE_PER_ARRIVAL[index] * n_arrivals
+        traffic = int(ROUTE_DRAM_READ[index] + ROUTE_DRAM_WRITE_PER_ARRIVAL[index] * n_arrivals)
     hbm_peak, kind = measured_peak_gbs()
     return {
         "bound": "smem", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

@@ -183,10 +183,10 @@ __device__ __forceinline__ Quad load_quad(const FusedArgs& a, long long r0, int 
     q.p = q.g = q.d = q.i = make_int4(0, 0, 0, 0);
     if (vec && li0 + 4 <= cnt) {           // r0 is a multiple of 4
         const long long at = (r0 + li0) >> 2;
-        q.p = __ldg(reinterpret_cast<const int4*>(a.prompt) + at);
-        q.g = __ldg(reinterpret_cast<const int4*>(a.generated) + at);
-        q.d = __ldg(reinterpret_cast<const int4*>(a.predicted) + at);
-        q.i = __ldg(reinterpret_cast<const int4*>(a.instance) + at);
+        q.p = __ldcs(reinterpret_cast<const int4*>(a.prompt) + at);
+        q.g = __ldcs(reinterpret_cast<const int4*>(a.generated) + at);
+        q.d = __ldcs(reinterpret_cast<const int4*>(a.predicted) + at);
+        q.i = __ldcs(reinterpret_cast<const int4*>(a.instance) + at);
         q.present = 15u;
     } else if (li0 < cnt) {
         int32_t* pp = &q.p.x; int32_t* gg = &q.g.x; int32_t* dd = &q.d.x; int32_t* ii = &q.i.x;
