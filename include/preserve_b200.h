@@ -133,7 +133,13 @@ int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d
  * >= 2^28) or did not fit in the table; d_score[k] (binary64, may be NULL) the winning L.
  * *d_n_requests is a DEVICE int64, read at the start and written at the end of the batch.
  *
- * The blocks of the routing kernel exchange their best instances through device memory and wait
+ * Two kernels implement the call with identical results (pre_route_select picks one).  The summary
+ * kernel keeps four numbers per row (largest cell, largest cell + step and where it sits, cell 0)
+ * that give the peak of almost every row for any arrival without reading the row, scans the few
+ * rows they leave undecided, routes with a single block and waits for nobody; it takes the batch
+ * when the context's instances fit its shared memory and every value stays below 2^32 during the
+ * batch, which it checks on the device.  Otherwise the scanning kernel routes: it reads every cell
+ * for every arrival, its blocks exchange their best instances through device memory and wait
  * for one another a bounded number of polls.  If such a wait runs out (PRE_ETIMEOUT from
  * pre_status; it should never happen on a GPU that runs the kernel alone), the blocks agree on
  * the last arrival that every one of them had scored: arrivals up to that one are routed exactly
@@ -296,6 +302,16 @@ int pre_status(pre_ctx* ctx, void* stream);
 
 /* The cudaError_t value of the last failed runtime call on this context (0 if none). */
 int pre_last_cuda_error(const pre_ctx* ctx);
+
+/* Which kernel routes the batches of pre_route_batch on this context: PRE_ROUTE_AUTO (default:
+ * the summary kernel when the shape fits it, the scanning kernel otherwise or when the summary
+ * kernel declines a batch), PRE_ROUTE_SCAN (always the scanning kernel), PRE_ROUTE_SUMMARY (as
+ * AUTO, but PRE_ESIZE here when the shape does not fit the summary kernel).  Results do not
+ * depend on it. */
+#define PRE_ROUTE_AUTO    0
+#define PRE_ROUTE_SCAN    1
+#define PRE_ROUTE_SUMMARY 2
+int pre_route_select(pre_ctx* ctx, int32_t path);
 
 /* Test hook, not part of the method: sets how many polls a device-side wait of this context's
  * kernels makes before it gives up (default 2^22; 0 gives up at the first unsuccessful poll).

@@ -17,7 +17,7 @@ PRE_OK, PRE_EINVAL, PRE_ECAPACITY, PRE_EBADREQ, PRE_ETIMEOUT, PRE_ECUDA, PRE_ENO
 EXPORTS = ("pre_create", "pre_destroy", "pre_anticipate", "pre_route_batch", "pre_step", "pre_status",
            "pre_last_cuda_error", "pre_strerror", "pre_query", "pre_anticipate_static", "pre_scaler_signals",
            "pre_refine", "pre_route_admit", "pre_ring_window", "pre_ring_fold", "pre_ring_step",
-           "pre_ring_refine", "pre_test_set_spin_limit", "pre_query_layout", "pre_tick")
+           "pre_ring_refine", "pre_test_set_spin_limit", "pre_query_layout", "pre_tick", "pre_route_select")
 
 
 class pre_config(C.Structure):
@@ -48,6 +48,7 @@ def _load():
     lib.pre_ring_refine.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, C.c_int32, vp, vp, vp, vp]
     lib.pre_status.argtypes = [vp, vp]
     lib.pre_test_set_spin_limit.argtypes = [vp, C.c_uint32]
+    lib.pre_route_select.argtypes = [vp, C.c_int32]
     lib.pre_last_cuda_error.argtypes = [vp]
     lib.pre_strerror.argtypes = [C.c_int]
     lib.pre_strerror.restype = C.c_char_p
@@ -184,6 +185,13 @@ def pre_ring_refine(ctx, prompt, generated, predicted, instance, actual, n_reque
 
 def pre_status(ctx, stream=None):
     return lib.pre_status(ctx, _stream() if stream is None else stream)
+
+
+ROUTE_AUTO, ROUTE_SCAN, ROUTE_SUMMARY = 0, 1, 2
+
+
+def pre_route_select(ctx, path):
+    return lib.pre_route_select(ctx, int(path))
 
 
 def pre_test_set_spin_limit(ctx, polls):

@@ -35,6 +35,10 @@ void release(pre_ctx* c) {
     for (int k = 0; k < 2; ++k) { cudaFree(c->d_fused_totals[k]); cudaFree(c->d_fused_hint[k]); }
     cudaFree(c->d_fused_base);
     cudaFree(c->d_fused_sync);
+    cudaFree(c->d_rs_summary);
+    cudaFree(c->d_rs_jtop);
+    cudaFree(c->d_rs_guard);
+    cudaFree(c->d_rs_handled);
     delete c;
 }
 
@@ -111,6 +115,13 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess) e = pre_fused_configure(c);
     if (e == cudaSuccess) e = pre_route_configure(c);
     if (e == cudaSuccess) e = alloc_zero(&c->d_slots, (size_t)32 * c->route_blocks);
+    if (e == cudaSuccess) e = pre_route_summary_configure(c);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_rs_guard, 8);
+    if (e == cudaSuccess) e = alloc_zero(&c->d_rs_handled, 1);
+    if (e == cudaSuccess && c->route_summary_smem) {
+        e = alloc_zero(&c->d_rs_summary, (size_t)2 * I);
+        if (e == cudaSuccess) e = alloc_zero(&c->d_rs_jtop, (size_t)I);
+    }
     if (e != cudaSuccess) {
         const bool oom = (e == cudaErrorMemoryAllocation);
         cudaGetLastError();
@@ -337,6 +348,13 @@ int pre_query_layout(const pre_ctx* ctx, int64_t out[4]) {
     out[1] = ctx->route_threads;
     out[2] = ctx->fused_grid;
     out[3] = pre_fused_max_rows(ctx);
+    return PRE_OK;
+}
+
+int pre_route_select(pre_ctx* ctx, int32_t path) {
+    if (!ctx || path < PRE_ROUTE_AUTO || path > PRE_ROUTE_SUMMARY) return PRE_EINVAL;
+    if (path == PRE_ROUTE_SUMMARY && !pre_route_summary_fits(ctx)) return PRE_ESIZE;
+    ctx->route_path = path;
     return PRE_OK;
 }
 

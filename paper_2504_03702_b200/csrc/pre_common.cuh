@@ -64,6 +64,13 @@ struct pre_ctx {
     unsigned int* d_fused_hint[2];     // [n_tiles + 1] where the lengths of one build put the next build's lists
     unsigned int* d_fused_base;     // [n_tiles + 1] where each tile's list starts when laid out exactly
     unsigned int* d_fused_sync;     // [8] barrier counter, largest B, id of an abandoned launch
+    // routing on per-row summaries: 0 bytes of shared memory when this shape does not use it
+    int route_path;                 // PRE_ROUTE_AUTO / _SCAN / _SUMMARY
+    size_t route_summary_smem;
+    unsigned long long* d_rs_summary;   // [I] {token count, largest cell, largest cell + step, cell 0} per row (16 bytes)
+    uint32_t* d_rs_jtop;            // [I] the first step of a row's largest cell + step
+    unsigned long long* d_rs_guard; // [8] what the summarising kernel found (largest cell, totals of the batch, ...)
+    int* d_rs_handled;              // 1 when the summary kernel routed the last batch, 0 when it left it to the scanning kernel
 };
 
 // Launchers (defined next to their kernels).  Each returns a cudaError_t.
@@ -106,6 +113,12 @@ cudaError_t pre_launch_ring_step(pre_ctx* ctx, int32_t* prompt, int32_t* generat
                                  int32_t* instance, const int64_t* n_requests, int64_t* ring, int width,
                                  int64_t* head, int64_t* queued_p, int64_t* current_d, cudaStream_t s);
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
+cudaError_t pre_route_summary_configure(pre_ctx* ctx);   // sets ctx->route_summary_smem (0: this shape keeps the scanning kernel)
+bool pre_route_summary_fits(const pre_ctx* ctx);
+cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                     int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                                     int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                                     int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s);
 size_t pre_tile_smem_bytes(int tile_rows, int horizon);
 int pre_tile_rows_for(int n_instances, int horizon, int n_sm);
 int pre_tile_threads(int tile_rows, int horizon);

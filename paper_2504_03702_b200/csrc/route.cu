@@ -138,6 +138,7 @@ struct RouteArgs {
     unsigned int* abort_key;    // 0xffffffff - (smallest exchange number at which a block's wait ran out); 0: none
     unsigned int* abort_count;  // blocks that have given up
     unsigned int spin_limit;    // polls before a wait is declared lost
+    const int* done_elsewhere;  // when set and non-zero: the batch has been routed by the summary kernel, nothing to do
     int max_rows;       // ceil(I / G)
     size_t resident_bytes;  // shared memory per block left for resident rows
     // admission queue (ADMIT kernels only): a ring of waiting requests, entry q at (head + q) mod capacity
@@ -383,6 +384,7 @@ __global__ void __launch_bounds__(ROUTE_THREADS, 1) pre_route_persistent(const R
     __shared__ int sh_all_over[2];        // ADMIT: every block reported all its rows overloaded (by exchange parity)
     constexpr int RS_RESIDENT = 1, RS_WIDE = 2;
 
+    if (a.done_elsewhere && *a.done_elsewhere) return;   // the same word for every block; nobody writes it meanwhile
     const int G = gridDim.x, b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int I = a.I, H = a.H;
@@ -1029,6 +1031,7 @@ static void fill_route_args(RouteArgs& a, pre_ctx* ctx, const int32_t* arr_promp
     a.abort_key = reinterpret_cast<unsigned int*>(ctx->d_abort + 1);
     a.abort_count = reinterpret_cast<unsigned int*>(ctx->d_abort + 2);
     a.spin_limit = ctx->spin_limit;
+    a.done_elsewhere = nullptr;
     a.max_rows = (a.I + ctx->route_blocks - 1) / ctx->route_blocks;
     a.resident_bytes = ctx->route_resident_bytes;
     a.queue_prompt = nullptr; a.queue_predicted = nullptr; a.queue_state = nullptr; a.queue_entry = nullptr;
@@ -1040,11 +1043,22 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
                              int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
                              int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
     if (n_arrivals == 0) return cudaSuccess;
-    cudaError_t e = cudaMemsetAsync(ctx->d_abort, 0, 3 * sizeof(int), s);   // flag, agreed exchange, blocks met
+    // The summary kernel takes the batch when the shape fits it; it declines (on the device) when 32-bit
+    // arithmetic could overflow during the batch, and the scanning kernel launched behind it then does
+    // the work.  When the summary kernel has routed the batch the scanning kernel returns at once.
+    const bool summaries = ctx->route_path != PRE_ROUTE_SCAN && pre_route_summary_fits(ctx);
+    cudaError_t e = cudaSuccess;
+    if (summaries) {
+        e = pre_launch_route_summary(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt,
+                                     generated, predicted, instance, n_requests, choice, score, s);
+        if (e != cudaSuccess) return e;
+    }
+    e = cudaMemsetAsync(ctx->d_abort, 0, 3 * sizeof(int), s);   // flag, agreed exchange, blocks met
     if (e != cudaSuccess) return e;
     RouteArgs a;
     fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
                     predicted, instance, n_requests, choice, score);
+    if (summaries) a.done_elsewhere = ctx->d_rs_handled;
     void* params[] = {(void*)&a};
     return cudaLaunchCooperativeKernel((const void*)pre_route_persistent<false>, dim3(ctx->route_blocks),
                                        dim3(ROUTE_THREADS), params, ctx->route_smem, s);

@@ -1,0 +1,753 @@
+// Load-aware request router (paper Sec. 4.3.3) on per-row summaries of the maps.
+//
+// The score of an arrival (P, D) against a row c[0..H) needs one number of the row, the peak
+// of the map with the arrival's ramp added (Sec. 4.3.1 update), Dc = min(D, H):
+//     peak = max( max_{j<Dc}(c[j] + P + j),  max_{j>=Dc} c[j] ).
+// Four numbers per row decide it without reading the row in almost every case:
+//     top  = max_j (c[j] + j)          jtop = the first step where that maximum is taken
+//     rmax = max_j c[j]                c0   = c[0]
+//   * Dc > jtop:  the ramp covers the step of the maximum, so max_{j<Dc}(c[j]+j) = top; and
+//                 P + top >= c[j] for every j, so   peak = P + top   exactly;
+//   * otherwise:  max(rmax, P + c0) <= peak <= P + top   (the ramp covers step 0; top bounds every step).
+// In maps of requests that are being decoded the occupancy falls as requests finish, the maximum
+// of c[j] + j sits at the first steps, and the first case is the rule.  The kernel never relies on
+// that: a row that is only bounded and could hold the smallest score is scanned cell by cell.
+//
+// Two kernels per batch:
+//   pre_summarise_rows   one pass over the maps: the four numbers of every row, the rows' token
+//                        counts (queued_p + current_d) and the guards that tell whether 32-bit
+//                        arithmetic stays exact for the whole batch;
+//   pre_route_summaries  routes the batch with ONE block: summaries in shared memory, no exchange
+//                        between blocks, hence no device-side wait on another block anywhere.
+//
+// pre_route_summaries works in rounds, one block barrier per round, two groups of warps:
+//   score warps: decide one arrival per round.  Every row's score comes from its summary; the
+//                last warp to finish takes the block's best row, writes the decision and hands
+//                the row to the fold warps.
+//   fold warps:  add an arrival to its row in the map (Sec. 4.3.1 update) and take the row's new
+//                summary in the same pass - RS_LAG rounds after the decision, so that the row's
+//                cells can be fetched a round ahead and no decision waits for a fold.
+// Between its decision and its fold a row is "pending": it is left out of the scoring pass and
+// represented by a lower bound of its score (its token count is exact at once; the cell that
+// held `top` only grows).  A pending row whose lower bound could win makes the round a stall:
+// nothing is decided, the folds go on, and the arrival is decided once the row is exact again.
+// The decisions are therefore the same as with every fold done at once.
+#include "pre_common.cuh"
+
+#include <math_constants.h>
+
+#include <cmath>
+#include <cstdlib>
+
+namespace {
+
+constexpr int RS_FOLD_WARPS = 8;
+constexpr int RS_FOLD_THREADS = 32 * RS_FOLD_WARPS;
+constexpr int RS_CONTROL_WARP = RS_FOLD_WARPS;     // the warp after the fold warps decides; the score warps follow it
+constexpr int RS_MAX_SCORE_WARPS = 23;
+constexpr int RS_MAX_THREADS = RS_FOLD_THREADS + 32 + 32 * RS_MAX_SCORE_WARPS;
+#ifndef PRE_RS_LAG
+#define PRE_RS_LAG 3
+#endif
+constexpr int RS_LAG = PRE_RS_LAG;         // rounds between a decision and the fold of its row
+constexpr int RS_PENDING = RS_LAG + 1;     // rows that can be pending at once (and row slots in shared memory)
+// Distance between the binary32 estimate of a score and the binary64 score, relative to
+// estimate + 2 * beta * theta: eight roundings of 2^-24 each on terms that add up to at most that
+// (2^-21), taken four times as large.
+constexpr float RS_EPS = 1.9073486328125e-06f;   // 2^-19
+constexpr int SUM_THREADS = 256;
+// whole-number scores: token count of a row that is left out of the pass (pending, or padding)
+constexpr unsigned int RS_OUT = 0xc0000000u;
+
+// named barriers (0 is __syncthreads)
+constexpr int BAR_SCORE = 1;    // among the score warps
+
+// guard words written by the summarising kernel
+constexpr int GUARD_MAX_CELL = 0, GUARD_MAX_BASE = 1, GUARD_BAD = 2, GUARD_SUM_RAMP = 3, GUARD_SUM_TOKENS = 4,
+              GUARD_MAX_PD = 5, GUARD_MAX_JTOP = 6;
+
+struct __align__(16) Item {
+    int P, D, Dc;
+    int k;   // index in the batch; -1: the batch has ended
+};
+
+// {token count, rmax, top, c0} of a row; jtop is kept beside it
+typedef uint4 RowSummary;
+
+// A row between its decision and its fold.
+struct __align__(16) Pending {
+    int row;                 // -1: free
+    int P, D, Dc;            // the arrival that goes into it
+    unsigned int tokens;     // token count with the arrival (exact)
+    unsigned int top_lb;     // cell jw + jw with the arrival added: a lower bound of the new top
+    unsigned int jw;         // the step of that cell (the old jtop)
+    unsigned int rmax;       // old largest cell: a lower bound of the new one
+    unsigned int c0;         // cell 0 with the arrival added (exact)
+    unsigned int unused[3];  // (three 16-byte stores write an entry)
+};
+
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+    const unsigned int d = (unsigned int)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bar_sync(int id, int count) {
+    __syncwarp();
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Score of one instance, binary64, every operation rounded on its own (the sums of whole
+// numbers below 2^53 are exact, so adding the two token counts first changes nothing).
+__device__ __forceinline__ double summary_score(unsigned int tokens, unsigned int peak, int P, int D, double theta,
+                                                double beta) {
+    double over = __dsub_rn((double)peak, theta);
+    if (over < 0.0) over = 0.0;
+    const double l = (double)((unsigned long long)tokens + (unsigned long long)P + (unsigned long long)D);
+    return __dadd_rn(l, __dmul_rn(beta, over));
+}
+
+__device__ __forceinline__ bool better_row(double s, int i, double bs, int bi) {
+    return s < bs || (s == bs && i < bi);
+}
+
+struct SumArgs {
+    const int64_t* curves;
+    const int64_t* queued_p;
+    const int64_t* current_d;
+    const int32_t* arr_prompt;
+    const int32_t* arr_predicted;
+    long long n_arrivals;
+    int I, H;
+    RowSummary* summary;
+    uint32_t* jtop;
+    unsigned long long* guard;
+};
+
+// One warp per row.
+__global__ void __launch_bounds__(SUM_THREADS) pre_summarise_rows(const SumArgs a) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int row = blockIdx.x * (SUM_THREADS / 32) + (tid >> 5);
+    const int H = a.H;
+    bool bad = false;
+    if (row < a.I) {
+        const int64_t* src = a.curves + (size_t)row * H;
+        unsigned int rmax = 0, top = 0, jtop = 0;
+        auto take = [&](long long v, int j) {
+            bad |= (v < 0) || (v > 0xffffffffLL);
+            const unsigned int c = (unsigned int)v;
+            rmax = max(rmax, c);
+            const unsigned long long t = (unsigned long long)c + (unsigned long long)j;
+            if (t > 0xffffffffull) bad = true;
+            if ((unsigned int)t > top) { top = (unsigned int)t; jtop = (unsigned int)j; }   // a lane's steps ascend
+        };
+        if ((H & 1) == 0) {
+            for (int j = 2 * lane; j < H; j += 64) {
+                const longlong2 v = __ldcs(reinterpret_cast<const longlong2*>(src + j));
+                take(v.x, j);
+                take(v.y, j + 1);
+            }
+        } else {
+            for (int j = lane; j < H; j += 32) take(__ldcs(src + j), j);
+        }
+        rmax = __reduce_max_sync(0xffffffffu, rmax);
+        const unsigned int t = __reduce_max_sync(0xffffffffu, top);
+        const unsigned int jt = __reduce_min_sync(0xffffffffu, top == t ? jtop : 0xffffffffu);
+        if (lane == 0) {
+            const long long q = a.queued_p[row], d = a.current_d[row];
+            const long long tok = q + d;
+            const bool ok = q >= 0 && d >= 0 && q <= 0xffffffffLL && d <= 0xffffffffLL && tok <= 0xffffffffLL;
+            if (!ok) bad = true;
+            a.summary[row] = make_uint4(ok ? (unsigned int)tok : 0u, rmax, t, (unsigned int)src[0]);
+            a.jtop[row] = jt;
+            if (ok) atomicMax(a.guard + GUARD_MAX_BASE, (unsigned long long)tok);
+            if (rmax) atomicMax(a.guard + GUARD_MAX_CELL, (unsigned long long)rmax);
+            if (jt) atomicMax(a.guard + GUARD_MAX_JTOP, (unsigned long long)jt);
+        }
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(a.guard + GUARD_BAD, 1ull);
+    // the arrivals' own totals: what the batch can add to a cell (ramps) and to a row's token count
+    unsigned long long ramp = 0, tokens = 0;
+    unsigned int max_pd = 0;
+    for (long long k = (long long)blockIdx.x * SUM_THREADS + tid; k < a.n_arrivals; k += (long long)gridDim.x * SUM_THREADS) {
+        const int P = a.arr_prompt[k], D = a.arr_predicted[k];
+        if (P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX) continue;
+        ramp += (unsigned long long)P + (unsigned long long)(D < H ? D : H);
+        tokens += (unsigned long long)P + (unsigned long long)D;
+        max_pd = max(max_pd, (unsigned int)P + (unsigned int)D);
+    }
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        ramp += __shfl_xor_sync(0xffffffffu, ramp, off);
+        tokens += __shfl_xor_sync(0xffffffffu, tokens, off);
+    }
+    max_pd = __reduce_max_sync(0xffffffffu, max_pd);
+    if (lane == 0 && (ramp | tokens)) {
+        atomicAdd(a.guard + GUARD_SUM_RAMP, ramp);
+        atomicAdd(a.guard + GUARD_SUM_TOKENS, tokens);
+        atomicMax(a.guard + GUARD_MAX_PD, (unsigned long long)max_pd);
+    }
+}
+
+struct RouteSumArgs {
+    const int32_t* arr_prompt;
+    const int32_t* arr_predicted;
+    long long n_arrivals;
+    int64_t* curves;
+    int64_t* queued_p;
+    int64_t* current_d;
+    int32_t* prompt;
+    int32_t* generated;
+    int32_t* predicted;
+    int32_t* instance;
+    int64_t* n_requests;
+    long long max_requests;
+    int32_t* choice;
+    double* score;
+    int I, H;
+    double theta, beta;
+    const RowSummary* summary0;
+    const uint32_t* jtop0;
+    const unsigned long long* guard;
+    int* status;
+    int* handled;   // 1: this kernel routed the batch; 0: the scanning kernel has to
+    int score_warps;
+};
+
+
+// CPT: cells of the folded row per fold thread (H <= CPT * RS_FOLD_THREADS).
+// VEC: H is even, so 16-byte accesses to the rows are legal.
+// The block has RS_FOLD_WARPS fold warps and a.score_warps score warps.
+template <int CPT, bool VEC>
+__global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const RouteSumArgs a) {
+    extern __shared__ __align__(16) unsigned char rs_smem[];
+    const int I = a.I, H = a.H;
+    const int Ip = (I + 31) & ~31;
+    uint2* tt = reinterpret_cast<uint2*>(rs_smem);          // [Ip] {token count (RS_OUT: left out of the pass), top}
+    uint2* aux = tt + Ip;                                   // [Ip] {rmax, c0}
+    uint32_t* jst = reinterpret_cast<uint32_t*>(aux + Ip);  // [Ip] jtop
+    int* list = reinterpret_cast<int*>(jst + Ip);           // [Ip] binary64 path: rows that have to be scanned
+    __shared__ Item sh_item[2];             // the arrival to decide, by round parity
+    __shared__ int sh_decided[2];           // whether the round decided its arrival
+    __shared__ Pending pend[RS_PENDING];
+    __shared__ unsigned long long sh_wkey[2][RS_MAX_SCORE_WARPS];   // the warps' best rows: score bits (binary64) or score << 32 | row
+    __shared__ int sh_wrow[2][RS_MAX_SCORE_WARPS];
+    __shared__ unsigned int sh_emin[2];     // bits of the block's smallest binary32 upper estimate, by round parity
+    __shared__ int sh_nlist[2];
+    __shared__ uint4 sh_fold[RS_FOLD_WARPS];   // per fold warp {rmax, top, jtop, -}
+    __shared__ unsigned int sh_jmax;        // no row's jtop is larger
+    __shared__ int sh_mode;                 // 0: decline the batch; 1: binary64 scores; 2: whole-number scores
+    __shared__ long long sh_n0;
+    __shared__ int sh_arr_p[64], sh_arr_d[64];   // the arrivals around the walker's position
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nsw = a.score_warps, nst = 32 * nsw, nthreads = RS_FOLD_THREADS + 32 + nst;
+    const double theta = a.theta, beta = a.beta;
+    if (tid == 0) {
+        const unsigned long long mc = a.guard[GUARD_MAX_CELL], mb = a.guard[GUARD_MAX_BASE];
+        // every cell, every cell + step with a prompt added, and every token count stay below 2^32 all batch long
+        const unsigned long long peak_bound = mc + a.guard[GUARD_SUM_RAMP] + (unsigned long long)H + (unsigned long long)PRE_FIELD_MAX;
+        const unsigned long long token_bound = mb + a.guard[GUARD_SUM_TOKENS];
+        const bool ok = a.guard[GUARD_BAD] == 0 && peak_bound <= 0xffffffffull && token_bound < (unsigned long long)RS_OUT;
+        // Whole-number scores: with beta and theta whole numbers every term of the score is a whole number
+        // below 2^53, each binary64 operation is exact, and the score is the same number in integer
+        // arithmetic; it is taken in 32 bits when even the largest possible score stays below 2^30.
+        bool whole = ok && beta == floor(beta) && theta == floor(theta) && beta <= 1048576.0 && theta < 1073741824.0;
+        if (whole) whole = token_bound + a.guard[GUARD_MAX_PD] + (unsigned long long)beta * peak_bound < (1ull << 30);
+        sh_mode = ok ? (whole ? 2 : 1) : 0;
+        sh_n0 = *a.n_requests;
+        sh_emin[0] = sh_emin[1] = 0x7f7fffffu;
+        sh_nlist[0] = sh_nlist[1] = 0;
+        sh_jmax = (unsigned int)a.guard[GUARD_MAX_JTOP];
+        for (int x = 0; x < RS_PENDING; ++x) pend[x].row = -1;
+    }
+    __syncthreads();
+    if (sh_mode == 0) {
+        if (tid == 0) *a.handled = 0;
+        return;
+    }
+    const bool whole = sh_mode == 2;
+    const unsigned int beta_i = whole ? (unsigned int)beta : 0u;
+    const int theta_i = whole ? (int)theta : 0;
+    for (int i = tid; i < Ip; i += nthreads) {
+        const RowSummary q = i < I ? a.summary0[i] : make_uint4(RS_OUT, 0, 0, 0);
+        tt[i] = make_uint2(q.x, q.z);
+        aux[i] = make_uint2(q.y, q.w);
+        jst[i] = i < I ? a.jtop0[i] : 0u;
+    }
+    const long long n0 = sh_n0;
+    long long room = a.max_requests - n0;
+    if (room < 0) room = 0;
+    const float thetaf = (float)theta, betaf = (float)beta;
+    const float c0f = 2.0f * betaf * thetaf;
+
+    // ---- the walker turns the batch into the sequence of requests that are really routed;
+    // malformed arrivals and those beyond the table's room are answered on the spot.  The deciding
+    // warp runs it, all lanes alike; the arrivals come through a ring of two 32-entry chunks in shared
+    // memory, each chunk copied while the one before it is being used.
+    auto copy_chunk = [&](long long first) {
+        const long long k = first + lane;
+        if (k < a.n_arrivals) {
+            cp_async4(&sh_arr_p[k & 63], a.arr_prompt + k);
+            cp_async4(&sh_arr_d[k & 63], a.arr_predicted + k);
+        }
+        cp_async_commit();
+    };
+    long long cursor = 0, entered = 0;   // (control warp, all lanes alike)
+    int walk_flags = 0;
+    auto walk_next = [&]() {
+        Item it;
+        it.P = it.D = it.Dc = 0;
+        it.k = -1;
+        while (cursor < a.n_arrivals) {
+            if ((cursor & 31) == 0) {   // a new chunk: its copy was started a chunk ago; start the next one
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                __syncwarp();
+                copy_chunk(cursor + 32);
+            }
+            const int P = sh_arr_p[cursor & 63], D = sh_arr_d[cursor & 63];
+            const bool bad = P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX;
+            if (bad || entered >= room) {
+                walk_flags |= bad ? PRE_ST_BADREQ : PRE_ST_CAPACITY;
+                if (lane == 0) {
+                    a.choice[cursor] = -1;
+                    if (a.score) a.score[cursor] = 0.0;
+                }
+                ++cursor;
+                continue;
+            }
+            it.P = P; it.D = D; it.Dc = D < H ? D : H; it.k = (int)cursor;
+            ++cursor; ++entered;
+            break;
+        }
+        return it;
+    };
+    // (control warp) the last decision, not yet written out
+    int out_w = -1, out_k = 0, out_P = 0, out_D = 0;
+    long long out_slot = 0;
+    double out_score = 0.0;
+    auto flush_outputs = [&]() {
+        if (out_w < 0) return;
+        if (lane == 0) { a.prompt[out_slot] = out_P; a.generated[out_slot] = 0; }
+        if (lane == 1) { a.predicted[out_slot] = out_D; a.instance[out_slot] = out_w; }
+        if (lane == 2) { a.choice[out_k] = out_w; if (a.score) a.score[out_k] = out_score; }
+        if (lane == 3) atomicAdd(reinterpret_cast<unsigned long long*>(a.queued_p + out_w), (unsigned long long)out_P);
+        if (lane == 4) atomicAdd(reinterpret_cast<unsigned long long*>(a.current_d + out_w), (unsigned long long)out_D);
+        out_w = -1;
+    };
+    Item nxt;               // (control warp) the arrival after the one being decided, walked to ahead of time
+    bool have_nxt = false;
+    nxt.P = nxt.D = nxt.Dc = 0; nxt.k = -1;
+    if (warp == RS_CONTROL_WARP) {
+        copy_chunk(0);
+        const Item first = walk_next();
+        if (lane == 0) sh_item[0] = first;
+    }
+    __syncthreads();
+
+    const int st = tid - RS_FOLD_THREADS - 32;      // score warps
+    const int sw_id = warp - RS_FOLD_WARPS - 1;
+    // fold warps: thread t holds cells 2t, 2t+1, then the same 2 * RS_FOLD_THREADS further on (16-byte accesses, a warp
+    // reads 512 contiguous bytes); without 16-byte accesses cells t, t + RS_FOLD_THREADS, ...
+    auto cell = [&](int u) { return VEC ? 2 * tid + (u >> 1) * (2 * RS_FOLD_THREADS) + (u & 1) : tid + u * RS_FOLD_THREADS; };
+    unsigned int c[CPT], cn[CPT];              // fold warps: the row being folded, the row fetched for the next fold
+    int fetched = -1;                          // the row in cn[]
+    // literal scan of one row by a warp: the peak with the arrival (P, Dc) added
+    auto scan_row = [&](int i, int P, int Dc) {
+        const int64_t* src = a.curves + (size_t)i * H;
+        unsigned int pk = 0;
+        if (VEC) {
+            for (int j = 2 * lane; j < H; j += 64) {
+                const longlong2 v = __ldcg(reinterpret_cast<const longlong2*>(src + j));
+                pk = max(pk, (unsigned int)v.x + (j < Dc ? (unsigned int)(P + j) : 0u));
+                pk = max(pk, (unsigned int)v.y + (j + 1 < Dc ? (unsigned int)(P + j + 1) : 0u));
+            }
+        } else {
+            for (int j = lane; j < H; j += 32)
+                pk = max(pk, (unsigned int)__ldcg(src + j) + (j < Dc ? (unsigned int)(P + j) : 0u));
+        }
+        return __reduce_max_sync(0xffffffffu, pk);
+    };
+    auto fetch = [&](int row, unsigned int* dst) {
+        const int64_t* src = a.curves + (size_t)row * H;
+        if (VEC) {
+            #pragma unroll
+            for (int u = 0; u < CPT; u += 2) {
+                longlong2 v = make_longlong2(0, 0);
+                if (cell(u) < H) v = __ldcg(reinterpret_cast<const longlong2*>(src + cell(u)));
+                dst[u] = (unsigned int)v.x; dst[u + 1] = (unsigned int)v.y;
+            }
+        } else {
+            #pragma unroll
+            for (int u = 0; u < CPT; ++u) dst[u] = cell(u) < H ? (unsigned int)__ldcg(src + cell(u)) : 0u;
+        }
+    };
+    auto whole_over = [&](unsigned int peak) { return (int)peak > theta_i ? peak - (unsigned int)theta_i : 0u; };
+
+    long long ndec = 0, nfold = 0;   // decisions made, folds done: every thread keeps them
+    bool stalled = false;
+    // Every arrival is decided after at most RS_PENDING stalled rounds and folded RS_LAG rounds later:
+    // the loop below ends by itself.  The limit only keeps a mistake in that reasoning from spinning.
+    const long long round_limit = (a.n_arrivals + 2) * (RS_PENDING + 2) + 64;
+    bool overrun = false;
+    for (long long round = 0;; ++round) {
+        if (round > round_limit) { overrun = true; break; }
+        const int par = (int)(round & 1);
+        const Item it = sh_item[par];
+        const bool have = it.k >= 0;
+        if (!have && nfold == ndec) break;
+        const bool do_fold = nfold < ndec && (ndec - nfold >= RS_LAG || !have || stalled);
+        unsigned int pend_lb_i = 0xffffffffu;   // (control warp) lower bound of pending entry nfold + lane for this arrival
+        double pend_lb_d = CUDART_INF;
+        int pend_row = -1;
+        if (warp == RS_CONTROL_WARP) {
+            // =============================== control warp, while the pass runs ===============================
+            // what does not depend on the pass: the last decision's outputs, the pending rows' lower
+            // bounds, the arrival after this one
+            flush_outputs();
+            if (have) {
+                const long long d = nfold + lane;
+                if (lane < RS_PENDING && d < ndec) {
+                    const Pending p = pend[d % RS_PENDING];
+                    const unsigned int peak_lb = (unsigned int)it.Dc > p.jw ? (unsigned int)it.P + p.top_lb
+                                                                             : max(p.rmax, (unsigned int)it.P + p.c0);
+                    pend_row = p.row;
+                    if (whole) pend_lb_i = p.tokens + beta_i * whole_over(peak_lb);   // (without the arrival's own P + D, like the pass)
+                    else pend_lb_d = summary_score(p.tokens, peak_lb, it.P, it.D, theta, beta);
+                }
+                if (!have_nxt) { nxt = walk_next(); have_nxt = true; }
+            }
+        } else if (warp > RS_CONTROL_WARP) {
+            // =============================== score warps: every row's score for arrival `it` ===============================
+            if (have) {
+                const int P = it.P, D = it.D, Dc = it.Dc;
+                const unsigned int PD = (unsigned int)P + (unsigned int)D;
+                if (whole) {
+                    unsigned int best = 0xffffffffu;   // scores without the arrival's own P + D
+                    int brow = 0x7fffffff;
+                    const int K = P - theta_i;
+                    if ((unsigned int)Dc > sh_jmax) {
+                        // every row's summary gives its peak: two words per row
+                        #pragma unroll 4
+                        for (int i = sw_id * 32 + lane; i < Ip; i += nst) {
+                            const uint2 q = tt[i];
+                            const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
+                            if (t < best) { best = t; brow = i; }
+                        }
+                    } else {
+                        // Some rows are only bounded.  First the smallest upper bound among the warp's rows
+                        // (every row's score is at most the score with peak P + top): no row whose lower
+                        // bound exceeds it can hold the smallest score.  Then the rows: exact ones compete,
+                        // bounded ones that pass that test are scanned by the warp.
+                        unsigned int reach = 0xffffffffu;
+                        for (int i = sw_id * 32 + lane; i < Ip; i += nst) {
+                            const uint2 q = tt[i];
+                            reach = min(reach, q.x + beta_i * (unsigned int)max((int)q.y + K, 0));
+                        }
+                        reach = __reduce_min_sync(0xffffffffu, reach);
+                        for (int base = sw_id * 32; base < Ip; base += nst) {
+                            const int i = base + lane;
+                            const uint2 q = tt[i];
+                            bool undecided = false;
+                            if (q.x != RS_OUT) {
+                                if ((unsigned int)Dc > jst[i]) {
+                                    const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
+                                    if (t < best) { best = t; brow = i; }
+                                } else {
+                                    const uint2 x = aux[i];
+                                    undecided = q.x + beta_i * whole_over(max(x.x, (unsigned int)P + x.y)) <= min(best, reach);
+                                }
+                            }
+                            unsigned int todo = __ballot_sync(0xffffffffu, undecided);
+                            while (todo) {
+                                const int src = __ffs(todo) - 1;
+                                todo &= todo - 1;
+                                const int row = base + src;
+                                const unsigned int t = tt[row].x + beta_i * whole_over(scan_row(row, P, Dc));
+                                if (lane == src && t < best) { best = t; brow = row; }   // a lane's rows ascend
+                            }
+                        }
+                    }
+                    const unsigned int m = __reduce_min_sync(0xffffffffu, best);
+                    const unsigned int r = __reduce_min_sync(0xffffffffu, best == m ? (unsigned int)brow : 0x7fffffffu);
+                    if (lane == 0) sh_wkey[par][sw_id] = m < RS_OUT ? ((unsigned long long)m << 32) | r : 0xffffffffffffffffull;
+                } else {
+                    // Pass 1, binary32: a lower and an upper estimate of every row's score (the same number when
+                    // the summary gives the peak exactly).  The block's smallest upper estimate bounds which rows
+                    // can hold the smallest score; pass 2 takes the binary64 score of those rows only.
+                    auto estimate = [&](unsigned int tokens, unsigned int peak) {
+                        return fmaf(betaf, fmaxf((float)peak - thetaf, 0.0f), (float)(tokens + PD));
+                    };
+                    float umin = 3.402823466e38f;
+                    auto pass1 = [&](int i) {
+                        const uint2 q = tt[i];
+                        if (q.x == RS_OUT) return CUDART_INF_F;
+                        const unsigned int up = (unsigned int)P + q.y;
+                        const uint2 x = aux[i];
+                        const unsigned int lo = (unsigned int)Dc > jst[i] ? up : max(x.x, (unsigned int)P + x.y);
+                        umin = fminf(umin, estimate(q.x, up));
+                        return estimate(q.x, lo);
+                    };
+                    for (int i = st; i < I; i += nst) pass1(i);
+                    // estimates are >= 0 and never NaN here (fminf drops a NaN): their bit patterns order like the values
+                    const unsigned int wmin = __reduce_min_sync(0xffffffffu, __float_as_uint(umin));
+                    if (lane == 0) atomicMin(&sh_emin[par], wmin);
+                    bar_sync(BAR_SCORE, nst);
+                    const float E = __uint_as_float(sh_emin[par]);
+                    // lower_m * (1 - eps) <= E * (1 + eps) + 2 * eps * c0 for the row m of the smallest score
+                    const float T = fmaf(E, 1.0f + RS_EPS, 2.0f * RS_EPS * c0f) * (1.0f + 3.0f * RS_EPS);
+                    double dbs = CUDART_INF;
+                    int dbi = 0x7fffffff;
+                    for (int i = st; i < I; i += nst) {
+                        if (pass1(i) > T) continue;
+                        const uint2 q = tt[i];
+                        if (q.x == RS_OUT) continue;
+                        if ((unsigned int)Dc > jst[i]) {
+                            const double sc = summary_score(q.x, (unsigned int)P + q.y, P, D, theta, beta);
+                            if (better_row(sc, i, dbs, dbi)) { dbs = sc; dbi = i; }
+                        } else {
+                            list[atomicAdd(&sh_nlist[par], 1)] = i;   // only bounded: the row itself decides
+                        }
+                    }
+                    bar_sync(BAR_SCORE, nst);
+                    const int n_list = sh_nlist[par];
+                    for (int x = sw_id; x < n_list; x += nsw) {
+                        const int i = list[x];
+                        const unsigned int pk = scan_row(i, P, Dc);
+                        const double sc = summary_score(tt[i].x, pk, P, D, theta, beta);
+                        if (lane == 0 && better_row(sc, i, dbs, dbi)) { dbs = sc; dbi = i; }
+                    }
+                    // scores are >= 0: their bit patterns order like the values
+                    unsigned long long key = (unsigned long long)__double_as_longlong(dbs);
+                    unsigned int hi = (unsigned int)(key >> 32), lo = (unsigned int)key;
+                    unsigned int mh = __reduce_min_sync(0xffffffffu, hi);
+                    unsigned int ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+                    int wrow = (int)__reduce_min_sync(0xffffffffu, (hi == mh && lo == ml) ? (unsigned int)dbi : 0x7fffffffu);
+                    if (lane == 0) {
+                        sh_wkey[par][sw_id] = ((unsigned long long)mh << 32) | ml;
+                        sh_wrow[par][sw_id] = wrow;
+                    }
+                }
+            }
+        } else if (do_fold) {
+            // =============================== fold warps: entry nfold goes into its row ===============================
+            const Pending p = pend[nfold % RS_PENDING];
+            const int w = p.row, P = p.P, Dc = p.Dc;
+            int64_t* grow = a.curves + (size_t)w * H;
+            if (fetched == w) {
+                #pragma unroll
+                for (int u = 0; u < CPT; ++u) c[u] = cn[u];
+            } else {
+                fetch(w, c);
+            }
+            // the row of the next entry, when it is known already, is fetched while this fold runs
+            fetched = -1;
+            if (CPT <= 8 && nfold + 1 < ndec) {   // (registers allowing)
+                fetched = pend[(nfold + 1) % RS_PENDING].row;
+                fetch(fetched, cn);
+            }
+            #pragma unroll
+            for (int u = 0; u < CPT; ++u)
+                if (cell(u) < Dc) c[u] += (unsigned int)(P + cell(u));
+            if (VEC) {
+                #pragma unroll
+                for (int u = 0; u < CPT; u += 2)   // (a pair whose second cell lies past the ramp writes that cell back unchanged)
+                    if (cell(u) < Dc) *reinterpret_cast<longlong2*>(grow + cell(u)) = make_longlong2((long long)c[u], (long long)c[u + 1]);
+            } else {
+                #pragma unroll
+                for (int u = 0; u < CPT; ++u)
+                    if (cell(u) < Dc) grow[cell(u)] = (long long)c[u];
+            }
+            unsigned int rmax = 0, top = 0, jtop = 0xffffffffu;
+            #pragma unroll
+            for (int u = 0; u < CPT; ++u) {   // a thread's steps ascend with u
+                const int j = cell(u);
+                if (j < H) {
+                    rmax = max(rmax, c[u]);
+                    const unsigned int t = c[u] + (unsigned int)j;
+                    if (jtop == 0xffffffffu || t > top) { top = t; jtop = (unsigned int)j; }
+                }
+            }
+            rmax = __reduce_max_sync(0xffffffffu, rmax);
+            const unsigned int wt = __reduce_max_sync(0xffffffffu, jtop != 0xffffffffu ? top : 0u);
+            const unsigned int wj = __reduce_min_sync(0xffffffffu, (jtop != 0xffffffffu && top == wt) ? jtop : 0xffffffffu);
+            if (lane == 0) sh_fold[warp] = make_uint4(rmax, wt, wj, 0u);
+        }
+        __syncthreads();   // the pass and the fold's per-warp maxima are complete
+        if (warp == RS_CONTROL_WARP) {
+            if (have) {
+                // ---- the decision.  The pass's best row wins unless a pending row could do better.
+                const int P = it.P, D = it.D, Dc = it.Dc;
+                const unsigned int PD = (unsigned int)P + (unsigned int)D;
+                double b1s = CUDART_INF;   // binary64 path: the pass's best score
+                unsigned int b1i = 0xffffffffu;   // whole-number path: the same without the arrival's own P + D
+                int b1r = -1;
+                {   // the best of the warps' rows: (key, row) pairs, smallest first (shuffles: a warp reduction
+                    // instruction costs a lone warp a few hundred cycles here)
+                    unsigned long long key = lane < nsw ? sh_wkey[par][lane] : 0xffffffffffffffffull;
+                    int row = (!whole && lane < nsw) ? sh_wrow[par][lane] : 0x7fffffff;
+                    for (int off = 1; off < nsw; off <<= 1) {
+                        const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, key, off);
+                        const int r2 = __shfl_xor_sync(0xffffffffu, row, off);
+                        if (k2 < key || (k2 == key && r2 < row)) { key = k2; row = r2; }
+                    }
+                    key = __shfl_sync(0xffffffffu, key, 0);   // lanes beyond the warps' count hold no result of their own
+                    row = __shfl_sync(0xffffffffu, row, 0);
+                    if (whole) {
+                        if (key != 0xffffffffffffffffull) { b1i = (unsigned int)(key >> 32); b1r = (int)(unsigned int)key; }
+                    } else if (row != 0x7fffffff) {
+                        b1s = __longlong_as_double((long long)key);
+                        b1r = row;
+                    }
+                }
+                bool stall = b1r < 0;
+                if (pend_row >= 0) {
+                    const bool could_win = whole ? (pend_lb_i < b1i || (pend_lb_i == b1i && pend_row < b1r))
+                                                 : better_row(pend_lb_d, pend_row, b1s, b1r);
+                    if (pend_row == b1r || could_win) stall = true;
+                }
+                stall = __any_sync(0xffffffffu, stall);
+                if (!stall) {
+                    // the row is pending from now on: exact token count, bounds for the rest
+                    const int w = b1r;
+                    if (lane == 0) {
+                        const uint2 q = tt[w], x = aux[w];
+                        const unsigned int jw = jst[w];
+                        uint4* dst = reinterpret_cast<uint4*>(&pend[ndec % RS_PENDING]);
+                        dst[0] = make_uint4((unsigned int)w, (unsigned int)P, (unsigned int)D, (unsigned int)Dc);
+                        dst[1] = make_uint4(q.x + PD, q.y + ((int)jw < Dc ? (unsigned int)P + jw : 0u), jw, x.x);
+                        dst[2] = make_uint4(x.y + (unsigned int)P, 0u, 0u, 0u);
+                        tt[w] = make_uint2(RS_OUT, 0u);
+                        *reinterpret_cast<uint4*>(&sh_item[par ^ 1]) = make_uint4((unsigned int)nxt.P, (unsigned int)nxt.D, (unsigned int)nxt.Dc, (unsigned int)nxt.k);
+                    }
+                    // what the outside sees of the decision is written while the next pass runs
+                    out_w = w; out_k = it.k; out_P = P; out_D = D; out_slot = n0 + ndec;
+                    out_score = whole ? (double)(b1i + PD) : b1s;
+                    have_nxt = false;
+                } else if (lane == 0) {
+                    sh_item[par ^ 1] = it;
+                }
+                if (lane == 0) {
+                    sh_decided[par] = stall ? 0 : 1;
+                    sh_emin[par] = 0x7f7fffffu;
+                    sh_nlist[par] = 0;
+                }
+            } else if (lane == 0) {
+                sh_item[par ^ 1] = it;   // the batch has ended; the remaining folds go on
+            }
+        } else if (tid == 0 && do_fold) {
+            // ---- the folded row's new summary; the row takes part in the next pass again
+            const Pending p = pend[nfold % RS_PENDING];
+            unsigned int rmax = 0, top = 0, jtop = 0xffffffffu;
+            #pragma unroll
+            for (int x = 0; x < RS_FOLD_WARPS; ++x) {   // the first step at which the largest cell + step is taken
+                const uint4 q = sh_fold[x];
+                rmax = max(rmax, q.x);
+                if (q.z != 0xffffffffu && (jtop == 0xffffffffu || q.y > top || (q.y == top && q.z < jtop))) { top = q.y; jtop = q.z; }
+            }
+            if (jtop == 0xffffffffu) jtop = 0u;
+            aux[p.row] = make_uint2(rmax, c[0]);
+            jst[p.row] = jtop;
+            if (jtop > sh_jmax) sh_jmax = jtop;
+            tt[p.row] = make_uint2(p.tokens, top);
+        }
+        __syncthreads();
+        if (have) {
+            stalled = sh_decided[par] == 0;
+            if (!stalled) ++ndec;
+        } else {
+            stalled = false;
+        }
+        if (do_fold) ++nfold;
+    }
+    if (warp == RS_CONTROL_WARP) flush_outputs();
+    if (overrun && tid == 0) atomicOr(a.status, PRE_ST_TIMEOUT);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (tid == RS_FOLD_THREADS) {   // the control warp kept the walker's counts
+        *a.n_requests = n0 + entered;
+        if (walk_flags) atomicOr(a.status, walk_flags);
+        *a.handled = 1;
+    }
+}
+
+}  // namespace
+
+// ---- host side
+
+static size_t summaries_smem_bytes(int I) {
+    const size_t Ip = (size_t)((I + 31) & ~31);
+    return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + sizeof(int));
+}
+
+// Score warps: about eight rows per score thread.
+static int summaries_score_warps(int I) {
+    int w = (I + 8 * 32 - 1) / (8 * 32);
+    if (const char* e = getenv("PRE_RS_SCORE_WARPS")) w = atoi(e);
+    return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
+}
+
+template <int CPT>
+static const void* summaries_kernel(bool vec) {
+    return vec ? (const void*)pre_route_summaries<CPT, true> : (const void*)pre_route_summaries<CPT, false>;
+}
+static const void* summaries_kernel_for(int H) {
+    const bool vec = (H & 1) == 0;
+    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4>(vec);
+    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8>(vec);
+    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16>(vec);
+    return summaries_kernel<32>(vec);
+}
+
+cudaError_t pre_route_summary_configure(pre_ctx* ctx) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    ctx->route_summary_smem = 0;
+    if (H > 32 * RS_FOLD_THREADS) return cudaSuccess;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
+    if (e != cudaSuccess) return e;
+    const void* fn = summaries_kernel_for(H);
+    cudaFuncAttributes attr;
+    e = cudaFuncGetAttributes(&attr, fn);
+    if (e != cudaSuccess) return e;
+    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
+    const size_t smem = summaries_smem_bytes(I);
+    if (smem + attr.sharedSizeBytes + 256 > limit) return cudaSuccess;   // too many instances
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    ctx->route_summary_smem = smem;
+    return cudaSuccess;
+}
+
+bool pre_route_summary_fits(const pre_ctx* ctx) { return ctx->route_summary_smem != 0 && ctx->d_rs_summary != nullptr; }
+
+cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                     int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                                     int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                                     int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    cudaError_t e = cudaMemsetAsync(ctx->d_rs_guard, 0, 8 * sizeof(unsigned long long), s);
+    if (e != cudaSuccess) return e;
+    SumArgs p;
+    p.curves = curves; p.queued_p = queued_p; p.current_d = current_d;
+    p.arr_prompt = arr_prompt; p.arr_predicted = arr_predicted; p.n_arrivals = n_arrivals;
+    p.I = I; p.H = H;
+    p.summary = reinterpret_cast<RowSummary*>(ctx->d_rs_summary);
+    p.jtop = ctx->d_rs_jtop; p.guard = ctx->d_rs_guard;
+    const int rows_per_block = SUM_THREADS / 32;
+    pre_summarise_rows<<<(I + rows_per_block - 1) / rows_per_block, SUM_THREADS, 0, s>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    RouteSumArgs a;
+    a.arr_prompt = arr_prompt; a.arr_predicted = arr_predicted; a.n_arrivals = n_arrivals;
+    a.curves = curves; a.queued_p = queued_p; a.current_d = current_d;
+    a.prompt = prompt; a.generated = generated; a.predicted = predicted; a.instance = instance;
+    a.n_requests = n_requests; a.max_requests = ctx->cfg.max_requests;
+    a.choice = choice; a.score = score;
+    a.I = I; a.H = H;
+    a.theta = ctx->theta; a.beta = ctx->cfg.beta;
+    a.summary0 = p.summary; a.jtop0 = p.jtop; a.guard = p.guard;
+    a.status = ctx->d_status; a.handled = ctx->d_rs_handled;
+    a.score_warps = summaries_score_warps(I);
+    void* params[] = {(void*)&a};
+    return cudaLaunchKernel(summaries_kernel_for(H), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
+                            ctx->route_summary_smem, s);
+}

@@ -169,6 +169,10 @@ class DeviceState:
     def status(self):
         return B.pre_status(self.ctx)
 
+    def select_router(self, path):
+        """B.ROUTE_AUTO, B.ROUTE_SCAN or B.ROUTE_SUMMARY: which kernel routes the batches (same results)."""
+        B.check(B.pre_route_select(self.ctx, path), "pre_route_select")
+
     def sync_count(self):
         """Reads the device-side request count back (synchronises)."""
         self.n_host = int(self.n_requests.item())

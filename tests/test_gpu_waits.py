@@ -30,6 +30,7 @@ def test_router_wait_that_runs_out_keeps_a_routed_prefix(idx):
     ap, ad = wl.ticks[0]
     ap, ad = ap[:256], ad[:256]
 
+    st.select_router(B.ROUTE_SCAN)      # the kernel whose blocks wait for one another
     assert B.pre_test_set_spin_limit(st.ctx, 0) == B.PRE_OK
     choice, score = st.route_batch(dev(ap), dev(ad))
     assert st.status() == B.PRE_ETIMEOUT
