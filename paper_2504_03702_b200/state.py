@@ -12,6 +12,9 @@ from . import binding as B
 
 
 class DeviceState:
+    # which routing kernel new states select (B.ROUTE_AUTO leaves the library's choice)
+    default_router = B.ROUTE_AUTO
+
     def __init__(self, n_instances, horizon, capacity_tokens, max_requests, t_mem=0.8, beta=1.0,
                  device="cuda:0"):
         self.I, self.H = int(n_instances), int(horizon)
@@ -21,6 +24,8 @@ class DeviceState:
         with torch.cuda.device(self.device):
             code, self.ctx = B.pre_create(n_instances, horizon, capacity_tokens, t_mem, beta, max_requests)
         B.check(code, "pre_create")
+        if DeviceState.default_router != B.ROUTE_AUTO:
+            B.check(B.pre_route_select(self.ctx, DeviceState.default_router), "pre_route_select")
         i32 = dict(dtype=torch.int32, device=self.device)
         i64 = dict(dtype=torch.int64, device=self.device)
         self.prompt = torch.zeros(self.max_requests, **i32)

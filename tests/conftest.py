@@ -22,3 +22,14 @@ def pytest_collection_modifyitems(config, items):
 def has_gpu():
     import torch
     return torch.cuda.is_available()
+
+
+@pytest.fixture(params=["auto", "scan"])
+def router(request):
+    """Runs a routing test once with the library's choice of kernel and once with the scanning kernel."""
+    from paper_2504_03702_b200 import binding as B
+    from paper_2504_03702_b200.state import DeviceState
+    old = DeviceState.default_router
+    DeviceState.default_router = {"auto": B.ROUTE_AUTO, "scan": B.ROUTE_SCAN}[request.param]
+    yield request.param
+    DeviceState.default_router = old

@@ -184,7 +184,7 @@ def test_argument_errors_launch_nothing():
 # ------------------------------------------------------------------ router
 
 @pytest.mark.parametrize("idx", [0, 1, 2])
-def test_route_configs_against_literal_oracle(idx):
+def test_route_configs_against_literal_oracle(idx, router):
     wl = W.make_config(idx)
     st, ref = both(wl)
     ap, ad = wl.ticks[0]
@@ -200,11 +200,12 @@ def test_route_configs_against_literal_oracle(idx):
 
 ROUTE_SHAPES = [(21, 1, 5, 10, 6), (22, 3, 9, 30, 25), (23, 7, 16, 60, 40), (24, 4, 1, 20, 10),
                 (25, 6, 40, 0, 30), (26, 200, 7, 500, 300), (27, 150, 64, 2000, 200), (28, 5, 1001, 300, 100),
-                (29, 333, 130, 3000, 257)]
+                (29, 333, 130, 3000, 257), (30, 6, 4100, 200, 60), (34, 3, 8190, 100, 40), (36, 9000, 6, 20000, 300),
+                (37, 12000, 4, 20000, 200)]
 
 
 @pytest.mark.parametrize("seed,n_inst,h,n,a", ROUTE_SHAPES)
-def test_route_shapes(seed, n_inst, h, n, a):
+def test_route_shapes(seed, n_inst, h, n, a, router):
     wl = W.make_random(seed, n_inst, h, n, a, max_prompt=300, max_output=2 * h + 3)
     st, ref = both(wl)
     ap, ad = wl.ticks[0]
@@ -217,7 +218,7 @@ def test_route_shapes(seed, n_inst, h, n, a):
 
 
 @pytest.mark.parametrize("max_prompt,n", [(2 ** 27, 6000), (2 ** 24, 18000), (2 ** 24, 20000), (2 ** 20, 40000)])
-def test_route_values_around_and_above_32_bits(max_prompt, n):
+def test_route_values_around_and_above_32_bits(max_prompt, n, router):
     """Rows whose cells cross 2^32 during the batch, start above it, or stay below it."""
     wl = W.make_random(35, 40, 128, n, 400, max_prompt=max_prompt, max_output=300, capacity=10 ** 9)
     st, ref = both(wl)
@@ -231,7 +232,7 @@ def test_route_values_around_and_above_32_bits(max_prompt, n):
     st.close()
 
 
-def test_route_fractional_threshold_and_beta_without_score_output():
+def test_route_fractional_threshold_and_beta_without_score_output(router):
     wl = W.make_random(31, 50, 24, 800, 300, capacity=33337, beta=0.75)
     wl.t_mem = 0.8
     st, ref = both(wl)
@@ -243,7 +244,7 @@ def test_route_fractional_threshold_and_beta_without_score_output():
     st.close()
 
 
-def test_route_consecutive_batches_and_empty_batch():
+def test_route_consecutive_batches_and_empty_batch(router):
     wl = W.make_random(32, 40, 32, 500, 400)
     wl.max_requests = 500 + 400
     st, ref = both(wl)
@@ -258,7 +259,7 @@ def test_route_consecutive_batches_and_empty_batch():
     st.close()
 
 
-def test_route_table_full_and_malformed_arrivals():
+def test_route_table_full_and_malformed_arrivals(router):
     wl = W.make_random(33, 6, 16, 100, 20)
     wl.max_requests = 100 + 12
     st, ref = both(wl)
@@ -279,7 +280,7 @@ def test_route_table_full_and_malformed_arrivals():
     st.close()
 
 
-def test_route_large_prefix_against_literal_oracle():
+def test_route_large_prefix_against_literal_oracle(router):
     """Largest configuration, launch shape of the benchmark; the literal oracle on the first arrivals."""
     wl = W.make_config(3)
     st, ref = both(wl)
@@ -293,7 +294,7 @@ def test_route_large_prefix_against_literal_oracle():
 
 
 @pytest.mark.slow
-def test_route_large_full_batch():
+def test_route_large_full_batch(router):
     """All 65,536 decisions of the largest configuration.
 
     Expected values come from the oracle's identity mode, which the CPU tests admit only
@@ -342,7 +343,7 @@ def test_step_shapes(seed, n_inst, h, n):
 
 
 @pytest.mark.parametrize("idx", [0, 1, 2])
-def test_route_then_step_configs(idx):
+def test_route_then_step_configs(idx, router):
     wl = W.make_config(idx)
     st, ref = both(wl)
     ap, ad = wl.ticks[0]
