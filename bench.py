@@ -35,19 +35,22 @@ METRIC = "routes/sec over the whole step (anticipate + route batch + decode step
 METRIC_STREAM = "routes/sec over the whole stream (decode step + routing of the tick's arrivals, per tick)"
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configuration 3; other
-# configurations report null).  profiles/ncu_full_step_kernels_config3_256_arrivals.txt: the routing kernel
-# reads the maps once per launch, whatever the batch length (67.31 MB), and wrote 420,864 B for 256 arrivals
+# configurations report null).  profiles/ncu_full_route_scan_kernel_config3_256_arrivals.txt: the scanning routing kernel
+# reads the maps once per launch, whatever the batch length (67.32 MB), and wrote 639,488 B for 256 arrivals
 # (folded cells, appended requests): the written part is scaled to the batch.  The single-launch build reads the
 # table and moves the tiles' lists; most of the 64 MiB of maps is still in L2 when the launch ends, which is why
 # its figure is below the algorithmic bytes.  pre_step: its two kernels added.
 # profiles/ncu_full_tick_scaler_refine_config3.txt: refinement and the fused tick (two kernels added).
-ROUTE_DRAM_READ = {3: 67314944}
-ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 420864 / 256}
-ANTICIPATE_DRAM_TRAFFIC = {3: 33807872 + 20073216}
-STEP_DRAM_TRAFFIC = {3: 33640192 + 67196160 + 8895232}
+ROUTE_DRAM_READ = {3: 67317760}
+# profiles/ncu_dram_route_summary_kernels_config3_full_batch.txt: both kernels of the summary router on the full
+# batch (the traffic does not grow in proportion to the batch, so the figure is used for the full batch only)
+ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67720000 + 124160 + 55920000 + 5480000}
+ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 639488 / 256}
+ANTICIPATE_DRAM_TRAFFIC = {3: 33807616 + 20817152}
+STEP_DRAM_TRAFFIC = {3: 33669120 + 67196160 + 9473792}
 SCALER_DRAM_TRAFFIC = {3: None}
-REFINE_DRAM_TRAFFIC = {3: 44149248 + 40192}
-TICK_DRAM_TRAFFIC = {3: 44138240 + 50944 + 67200000 + 8971776}
+REFINE_DRAM_TRAFFIC = {3: 44150272 + 29952}
+TICK_DRAM_TRAFFIC = {3: 44136960 + 50176 + 67199488 + 10226944}
 
 
 def measured_peak_gbs():
@@ -282,6 +285,8 @@ def bench_oneshot(args, wl, index, device, group, world, steps, warmup, headline
     n0, a = wl.n_requests, wl.n_arrivals
     arr_p_host, arr_d_host = wl.ticks[0]
     st = DeviceState.from_workload(wl, device=device)
+    if args.router == "scan":
+        st.select_router(B.ROUTE_SCAN)
     pristine_generated = st.generated[:n0].clone()
     arr_p = torch.as_tensor(arr_p_host).to(device)
     arr_d = torch.as_tensor(arr_d_host).to(device)
@@ -339,6 +344,8 @@ def bench_oneshot(args, wl, index, device, group, world, steps, warmup, headline
     res["t_dstep"] = float(np.mean([e[2].elapsed_time(e[3]) for e in events]))
     res["t_step"] = D.max_over_ranks(res["t_build"] + res["t_route"] + res["t_dstep"], group, device)
     res["map_max"] = int(st.curves.max().item())
+    res["route_kernel"] = "summary" if B.pre_route_select(st.ctx, B.ROUTE_SUMMARY) == B.PRE_OK and args.router != "scan" else "scan"
+    B.check(B.pre_route_select(st.ctx, B.ROUTE_SCAN if args.router == "scan" else B.ROUTE_AUTO), "pre_route_select")
     # what the timed steps left behind, for the parity check (taken before anything else touches the state)
     res["snapshot"] = (choice.clone(), score.clone())
     res["reset"], res["flush"], res["arr"] = reset, flush, (arr_p, arr_d)
@@ -429,6 +436,29 @@ def extras_leg(res, wl, index, device):
                               st.generated, st.predicted, st.instance, st.n_requests, choice, score),
             "pre_route_batch")
     st.step()
+
+    # the scanning kernel on the first arrivals of the same batch (it routes what the summary kernel declines,
+    # and every call of the admission router)
+    if res["route_kernel"] == "summary":
+        n_scan = min(a, 8192)
+        st.select_router(B.ROUTE_SCAN)
+        rebuild_and_route()
+        flush.zero_()
+        e0, e1 = ev(), ev()
+        e0.record()
+        B.check(B.pre_route_batch(st.ctx, arr_p, arr_d, n_scan, st.curves, st.queued_p, st.current_d, st.prompt,
+                                  st.generated, st.predicted, st.instance, st.n_requests, choice, score),
+                "pre_route_batch (scanning kernel)")
+        e1.record()
+        torch.cuda.synchronize()
+        B.check(st.status(), "scanning kernel")
+        out["route_scan_sample"] = (e0.elapsed_time(e1), n_scan, int(st.curves.max().item()))
+        st.select_router(B.ROUTE_AUTO)
+        rebuild_and_route()
+        B.check(B.pre_route_batch(st.ctx, arr_p, arr_d, a, st.curves, st.queued_p, st.current_d, st.prompt,
+                                  st.generated, st.predicted, st.instance, st.n_requests, choice, score),
+                "pre_route_batch")
+        st.step()
 
     # scaler signals over the maps (Sec. 4.3.2)
     sc_ev = []
@@ -531,6 +561,8 @@ def bench_stream(args, wl, index, device, group, n_check_ticks):
     from paper_2504_03702_b200 import dist as D
     from paper_2504_03702_b200.state import DeviceState
     st = DeviceState.from_workload(wl, device=device)
+    if args.router == "scan":
+        st.select_router(B.ROUTE_SCAN)
     arrs = [(torch.as_tensor(ap).to(device), torch.as_tensor(ad).to(device)) for ap, ad in wl.ticks]
     e_b0, e_b1 = ev(), ev()
     torch.cuda.synchronize()
@@ -582,8 +614,8 @@ def bench_stream(args, wl, index, device, group, n_check_ticks):
     return res
 
 
-def route_roofline(wl, index, t_route_ms, n_arrivals, map_max, layout, route_blocks, clocks, n_sm):
-    """The routing kernel against the roof it runs under.  Every arrival scans every cell of every map, but the
+def route_scan_roofline(wl, index, t_route_ms, n_arrivals, map_max, layout, route_blocks, clocks, n_sm):
+    """The scanning routing kernel against the roof it runs under.  Every arrival scans every cell of every map, but the
     maps are copied into shared memory once per batch (32-bit cells when every value is below 2^32), so the roof
     is the shared-memory bandwidth of the SMs: 128 bytes per clock and SM at the sampled clock."""
     i, h = wl.n_instances, wl.horizon
@@ -620,6 +652,37 @@ def route_roofline(wl, index, t_route_ms, n_arrivals, map_max, layout, route_blo
                 f"capture scaled to this batch ({kind} HBM peak {hbm_peak:.0f} GB/s for hbm_frac_of_captured_traffic)"}
 
 
+def route_summary_roofline(wl, index, t_route_ms, n_arrivals, clocks):
+    """The summary routing kernel.  One block on one SM: per arrival it reads the rows' summaries from shared
+    memory (8 bytes per instance), reads and rewrites the receiving row in the map (16 bytes per step), and is
+    bound by the latency of its rounds (two block barriers and the dependent steps of a decision), not by any
+    bandwidth.  The roof quoted is the shared-memory bandwidth of the ONE SM the block runs on."""
+    i, h = wl.n_instances, wl.horizon
+    ip = (i + 31) // 32 * 32
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+    peak = 128 * mhz * 1e6 / 1e9
+    sec = t_route_ms * 1e-3
+    smem_bytes = 8 * ip * n_arrivals
+    achieved = smem_bytes / sec / 1e9
+    literal = n_arrivals * (8 * i * h + 16 * h + 16 * i)
+    traffic = ROUTE_SUMMARY_DRAM_TRAFFIC.get((index, n_arrivals))
+    hbm_peak, kind = measured_peak_gbs()
+    return {
+        "bound": "smem", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "peak_kind": f"derived: 1 SM x 128 B/clk x {mhz:.0f} MHz (the kernel is one block; SM clock sampled during the timed region)",
+        "traffic": traffic, "kernel": "pre_summarise_rows + pre_route_summaries", "us_per_arrival": sec * 1e6 / n_arrivals,
+        "bytes_of_shared_memory_read_per_arrival": 8 * ip, "bytes_of_map_read_and_written_per_arrival": 16 * h,
+        "scan_equivalent_gbs": literal / sec / 1e9,
+        "hbm_frac_of_captured_traffic": None if traffic is None else traffic / sec / 1e9 / hbm_peak,
+        "limiter": "latency: every arrival is one round of the block (two block barriers, the scoring pass, the "
+                   "dependent steps of the decision); the pass itself needs 8 bytes per instance",
+        "note": "the kernel decides from four numbers per row instead of scanning the maps (identical decisions); "
+                "achieved = bytes of row summaries read from shared memory over time; scan_equivalent_gbs is the "
+                "literal formulation's 8 bytes per cell and arrival over time, a convenience number that is not "
+                f"memory traffic; traffic = DRAM bytes of both kernels from the ncu capture of this batch "
+                f"({kind} HBM peak {hbm_peak:.0f} GB/s for hbm_frac_of_captured_traffic)"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -632,6 +695,8 @@ def main():
     ap.add_argument("--cpu-arrivals", type=int, default=600, help="arrivals routed literally by the cpu_baseline leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (no parity check either)")
     ap.add_argument("--no-extras", action="store_true", help="skip the separate calls and the per-configuration entries")
+    ap.add_argument("--router", default="auto", choices=["auto", "scan"],
+                    help="auto: the summary routing kernel where the shape fits it; scan: always the scanning kernel")
     ap.add_argument("--stream-ticks", type=int, default=0, help="shorten the stream to this many ticks (0: all 1,000)")
     ap.add_argument("--arrivals", type=int, default=0,
                     help="route only the first ARRIVALS of the batch (short kernels for profiler captures; "
@@ -742,18 +807,25 @@ def main():
         "anticipated_request_steps_per_s": world * wl.n_requests * wl.horizon / (t_build * 1e-3),
         "routes_per_s_route_call_only": world * a / (t_route * 1e-3),
         "parity_checked": parity,
-        "roofline": route_roofline(wl, args.config, t_route, a, res["map_max"], layout, route_blocks, res["clocks"], n_sm),
+        "roofline": (route_summary_roofline(wl, args.config, t_route, a, res["clocks"]) if res["route_kernel"] == "summary"
+                     else route_scan_roofline(wl, args.config, t_route, a, res["map_max"], layout, route_blocks, res["clocks"], n_sm)),
+        "route_kernel": res["route_kernel"],
         "roofline_anticipate": anticipate_roof,
         "roofline_step": roof_hbm(b_step, t_dstep, 2, STEP_DRAM_TRAFFIC.get(args.config),
                                   "pre_step_requests + pre_step_shift",
                                   note="runs right after the routing kernel: part of the maps is served from L2, see traffic"),
         "e2e": {"value": world * a / (t_e2e * 1e-3), "unit": "routes/s", "h2d_bytes_per_step": res["h2d"],
                 "d2h_bytes_per_step": res["d2h"], "ms_per_step": t_e2e},
-        "gpu_launches": (4 if fused else 5) * args.steps,
+        "gpu_launches": ((4 if fused else 5) + (2 if res["route_kernel"] == "summary" else 0)) * args.steps,
         "clocks": res["clocks"],
         "wall_s_timed_region": res["wall_s"],
         "routed": routed_ok,
     }
+    if "route_scan_sample" in extras:
+        t_scan, n_scan, scan_max = extras.pop("route_scan_sample")
+        out["roofline_route_scan"] = route_scan_roofline(wl, args.config, t_scan, n_scan, scan_max, layout, route_blocks,
+                                                         res["clocks"], n_sm)
+        out["roofline_route_scan"]["sample"] = f"the first {n_scan} arrivals of the batch through the scanning kernel, one call"
     out.update(extras)
     if args.arrivals > 0:
         out["truncated_batch"] = "profiling run, not a benchmark result"

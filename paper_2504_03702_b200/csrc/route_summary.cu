@@ -91,6 +91,30 @@ __device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// Warp-wide minimum / maximum of a 64-bit key with shuffles.  (Measured in this kernel: a redux.sync costs a warp
+// 250 to 300 cycles, five shuffle steps about half of that.)
+__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v) {
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = o < v ? o : v;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = o > v ? o : v;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned int warp_max_u32(unsigned int v) {
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, off));
+    return v;
+}
+
 __device__ __forceinline__ void bar_sync(int id, int count) {
     __syncwarp();
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -467,9 +491,9 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                             }
                         }
                     }
-                    const unsigned int m = __reduce_min_sync(0xffffffffu, best);
-                    const unsigned int r = __reduce_min_sync(0xffffffffu, best == m ? (unsigned int)brow : 0x7fffffffu);
-                    if (lane == 0) sh_wkey[par][sw_id] = m < RS_OUT ? ((unsigned long long)m << 32) | r : 0xffffffffffffffffull;
+                    // smallest (score, row) of the warp: one 64-bit key
+                    const unsigned long long wk = warp_min_u64(((unsigned long long)best << 32) | (unsigned int)brow);
+                    if (lane == 0) sh_wkey[par][sw_id] = (unsigned int)(wk >> 32) < RS_OUT ? wk : 0xffffffffffffffffull;
                 } else {
                     // Pass 1, binary32: a lower and an upper estimate of every row's score (the same number when
                     // the summary gives the peak exactly).  The block's smallest upper estimate bounds which rows
@@ -567,9 +591,11 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                     if (jtop == 0xffffffffu || t > top) { top = t; jtop = (unsigned int)j; }
                 }
             }
-            rmax = __reduce_max_sync(0xffffffffu, rmax);
-            const unsigned int wt = __reduce_max_sync(0xffffffffu, jtop != 0xffffffffu ? top : 0u);
-            const unsigned int wj = __reduce_min_sync(0xffffffffu, (jtop != 0xffffffffu && top == wt) ? jtop : 0xffffffffu);
+            rmax = warp_max_u32(rmax);
+            // largest cell + step and the first step that has it: (top, ~step) as one 64-bit key
+            const unsigned long long tk = warp_max_u64(jtop != 0xffffffffu ? ((unsigned long long)top << 32) | (0xffffffffu - jtop) : 0ull);
+            const unsigned int wt = (unsigned int)(tk >> 32);
+            const unsigned int wj = tk ? 0xffffffffu - (unsigned int)tk : 0xffffffffu;
             if (lane == 0) sh_fold[warp] = make_uint4(rmax, wt, wj, 0u);
         }
         __syncthreads();   // the pass and the fold's per-warp maxima are complete
@@ -678,9 +704,10 @@ static size_t summaries_smem_bytes(int I) {
     return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + sizeof(int));
 }
 
-// Score warps: about eight rows per score thread.
+// Score warps: about sixteen rows per score thread (measured: 4,096 instances are fastest with 8 score warps,
+// 1,024 with 2 to 4; more warps lengthen the block barriers more than they shorten the pass).
 static int summaries_score_warps(int I) {
-    int w = (I + 8 * 32 - 1) / (8 * 32);
+    int w = (I + 16 * 32 - 1) / (16 * 32);
     if (const char* e = getenv("PRE_RS_SCORE_WARPS")) w = atoi(e);
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
