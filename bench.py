@@ -45,6 +45,9 @@ ROUTE_DRAM_READ = {3: 67317760}
 # profiles/ncu_dram_route_summary_kernels_config3_full_batch.txt: both kernels of the summary router on the full
 # batch (the traffic does not grow in proportion to the batch, so the figure is used for the full batch only)
 ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67720000 + 124160 + 55920000 + 5480000}
+# warp instructions per arrival of pre_route_summaries (smsp__inst_executed.sum of the 2,048-arrival capture in
+# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 12,760,381 / 2,048)
+ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 12760381 / 2048}
 ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 639488 / 256}
 ANTICIPATE_DRAM_TRAFFIC = {3: 33807616 + 20817152}
 STEP_DRAM_TRAFFIC = {3: 33669120 + 67196160 + 9473792}
@@ -656,7 +659,8 @@ def route_summary_roofline(wl, index, t_route_ms, n_arrivals, clocks):
     """The summary routing kernel.  One block on one SM: per arrival it reads the rows' summaries from shared
     memory (8 bytes per instance), reads and rewrites the receiving row in the map (16 bytes per step), and is
     bound by the latency of its rounds (two block barriers and the dependent steps of a decision), not by any
-    bandwidth.  The roof quoted is the shared-memory bandwidth of the ONE SM the block runs on."""
+    bandwidth.  Where the instructions per arrival are known from an ncu capture the roof quoted is the instruction
+    issue of the ONE SM the block runs on, else that SM's shared-memory bandwidth."""
     i, h = wl.n_instances, wl.horizon
     ip = (i + 31) // 32 * 32
     mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
@@ -667,20 +671,35 @@ def route_summary_roofline(wl, index, t_route_ms, n_arrivals, clocks):
     literal = n_arrivals * (8 * i * h + 16 * h + 16 * i)
     traffic = ROUTE_SUMMARY_DRAM_TRAFFIC.get((index, n_arrivals))
     hbm_peak, kind = measured_peak_gbs()
-    return {
-        "bound": "smem", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_kind": f"derived: 1 SM x 128 B/clk x {mhz:.0f} MHz (the kernel is one block; SM clock sampled during the timed region)",
+    out = {
         "traffic": traffic, "kernel": "pre_summarise_rows + pre_route_summaries", "us_per_arrival": sec * 1e6 / n_arrivals,
         "bytes_of_shared_memory_read_per_arrival": 8 * ip, "bytes_of_map_read_and_written_per_arrival": 16 * h,
+        "smem_gbs": achieved, "smem_peak_gbs_of_the_one_sm": peak, "smem_frac": achieved / peak,
         "scan_equivalent_gbs": literal / sec / 1e9,
         "hbm_frac_of_captured_traffic": None if traffic is None else traffic / sec / 1e9 / hbm_peak,
         "limiter": "latency: every arrival is one round of the block (two block barriers, the scoring pass, the "
-                   "dependent steps of the decision); the pass itself needs 8 bytes per instance",
-        "note": "the kernel decides from four numbers per row instead of scanning the maps (identical decisions); "
-                "achieved = bytes of row summaries read from shared memory over time; scan_equivalent_gbs is the "
-                "literal formulation's 8 bytes per cell and arrival over time, a convenience number that is not "
-                f"memory traffic; traffic = DRAM bytes of both kernels from the ncu capture of this batch "
-                f"({kind} HBM peak {hbm_peak:.0f} GB/s for hbm_frac_of_captured_traffic)"}
+                   "dependent steps of the decision); neither a memory nor the instruction issue is saturated",
+        "note": "the kernel decides from four numbers per row instead of scanning the maps (identical decisions) and "
+                "runs as ONE block; smem_* = bytes of row summaries read from shared memory over time against 128 "
+                f"B/clk x {mhz:.0f} MHz of the one SM it occupies; scan_equivalent_gbs is the literal formulation's 8 "
+                "bytes per cell and arrival over time, a convenience number that is not memory traffic; traffic = DRAM "
+                f"bytes of both kernels from the ncu capture of this batch ({kind} HBM peak {hbm_peak:.0f} GB/s for "
+                "hbm_frac_of_captured_traffic)"}
+    inst = ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL.get(index)
+    if inst is not None:
+        # not memory-bound: the roof is the instruction issue of the SM the block runs on, 4 warp instructions per clock
+        issue_peak = 4 * mhz * 1e6 / 1e9
+        issued = inst * n_arrivals / sec / 1e9
+        out.update({"bound": "alu", "achieved": issued, "peak": issue_peak, "unit": "G warp-instructions/s",
+                    "frac": issued / issue_peak,
+                    "peak_kind": f"derived: 1 SM x 4 schedulers x 1 warp instruction per clock x {mhz:.0f} MHz (SM clock "
+                                 "sampled during the timed region)",
+                    "warp_instructions_per_arrival": inst})
+    else:
+        out.update({"bound": "smem", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "peak_kind": f"derived: 1 SM x 128 B/clk x {mhz:.0f} MHz (the kernel is one block; SM clock sampled "
+                                 "during the timed region)"})
+    return out
 
 
 def main():
