@@ -262,7 +262,12 @@ int pre_tick(pre_ctx* ctx, int32_t* d_prompt, int32_t* d_generated, int32_t* d_p
  *     pre_ring_fold with the choices the router returned,
  * and gives the decisions of a router that takes its peaks over the first l steps of the
  * full-width maps and really adds each routed request's whole ramp: no score of a batch
- * depends on a step beyond the window, and the additions beyond it commute. */
+ * depends on a step beyond the window, and the additions beyond it commute.
+ * With pre_route_admit the routed requests are not only arrivals (waiting requests come first,
+ * and the queue's slots may be rewritten during the call): fold from the rows the call appended to
+ * the request table instead - pre_ring_fold(d_prompt + n0, d_predicted + n0, d_instance + n0,
+ * n1 - n0, ...) with n0, n1 the request count before and after the call; those rows are exactly
+ * the routed requests, each with its instance. */
 
 /* d_window[i*l + j] = d_ring[i*width + (head + j) mod width], j < l: the dense maps of width
  * l (16-byte aligned) that pre_route_batch, pre_route_admit and pre_scaler_signals take. */

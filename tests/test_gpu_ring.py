@@ -117,6 +117,65 @@ def test_ring_ticks_with_refinement_match_the_oracle(seed, n_inst, width, window
     st.close()
 
 
+@pytest.mark.parametrize("level", [0.7, 0.8])
+def test_ring_ticks_with_the_admission_queue(level):
+    """Full-width maps with pre_route_admit: waiting requests are routed out of the queue while arrivals
+    join it, and the ring is brought up to date from the rows the call appended to the request table.
+    The oracle routes on the first `window` steps of its full-width maps (its admission router on a state
+    of that width) and rebuilds the full-width maps from the table by the definition."""
+    seed, n_inst, width, window, n, a, ticks, qcap = 79, 6, 48, 10, 300, 24, 14, 40
+    wl = W.make_random(seed, n_inst, width, n, 0, max_prompt=300, max_output=2 * width)
+    cap = wl.n_requests + a * ticks + qcap
+    st = DeviceState(n_inst, window, wl.capacity_tokens, cap, wl.t_mem, wl.beta)
+    st.load_requests(wl.prompt, wl.generated, wl.predicted, wl.instance)
+    st.make_ring(width)
+    st.make_queue(qcap)
+    full = oracle.State(n_inst, width, wl.capacity_tokens, wl.prompt, wl.generated, wl.predicted, wl.instance,
+                        cap, wl.t_mem, wl.beta)
+    full.anticipate()
+    queue = None
+    rng = np.random.RandomState(seed)
+    routed_from_queue = joined = turned_away = 0
+    for t in range(ticks):
+        ap = rng.randint(1, 300, a).astype(np.int32)
+        ad = rng.randint(1, 2 * width + 1, a).astype(np.int32)
+        st.ring_step()
+        full.step()
+        st.ring_window()
+        nf = int(full.n[0])
+        win = oracle.State(n_inst, window, wl.capacity_tokens, full.prompt[:nf], full.generated[:nf],
+                           full.predicted[:nf], full.instance[:nf], cap, wl.t_mem, wl.beta)
+        win.curves[:] = full.curves[:, :window]
+        win.queued_p[:] = full.queued_p
+        win.current_d[:] = full.current_d
+        win.make_queue(qcap)
+        if queue is not None:
+            win.queue_prompt[:], win.queue_predicted[:], win.queue_state[:] = queue
+        waiting = int(win.queue_state[1])
+        n0 = st.sync_count()
+        qc, c, sc = st.route_admit(dev(ap), dev(ad), overload_level=level, overload_share=0.10)
+        n1 = st.sync_count()
+        if n1 > n0:   # the routed requests, each with its instance: the rows the call appended
+            st.ring_fold(st.prompt[n0:n1], st.predicted[n0:n1], st.instance[n0:n1])
+        want_qc, want_c, want_s = win.route_admit(ap, ad, level, 0.10)
+        queue = (win.queue_prompt.copy(), win.queue_predicted.copy(), win.queue_state.copy())
+        assert (qc.cpu().numpy()[:waiting] == want_qc).all(), f"tick {t}: waiting requests"
+        assert (c.cpu().numpy() == want_c).all(), f"tick {t}: arrivals"
+        assert_scores_close(sc.cpu().numpy(), want_s, want_c)
+        assert st.queue_state.cpu().tolist() == win.queue_state.tolist()
+        routed_from_queue += int((want_qc >= 0).sum())
+        joined += int((want_c == -2).sum())
+        turned_away += int((want_c == -3).sum())
+        nf = int(win.n[0])
+        full = oracle.State(n_inst, width, wl.capacity_tokens, win.prompt[:nf], win.generated[:nf],
+                            win.predicted[:nf], win.instance[:nf], cap, wl.t_mem, wl.beta)
+        full.anticipate()
+        full.queued_p[:] = win.queued_p
+        same(st, full, f"after tick {t}")
+    assert routed_from_queue > 0 and joined > 0 and turned_away > 0, "the case was meant to exercise the queue"
+    st.close()
+
+
 def test_ring_streaming_config_first_ticks():
     """The streaming configuration on maps of its full width (1,024) with the paper's window of 100."""
     wl = W.make_config(4, n_ticks=3)
