@@ -51,7 +51,7 @@ ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 12760381 / 2048}
 ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 639488 / 256}
 ANTICIPATE_DRAM_TRAFFIC = {3: 33807616 + 20817152}
 STEP_DRAM_TRAFFIC = {3: 33669120 + 67196160 + 9473792}
-SCALER_DRAM_TRAFFIC = {3: None}
+SCALER_DRAM_TRAFFIC = {3: 67128576 + 326912}   # profiles/ncu_full_scaler_rows_config3.txt
 REFINE_DRAM_TRAFFIC = {3: 44150272 + 29952}
 TICK_DRAM_TRAFFIC = {3: 44136960 + 50176 + 67199488 + 10226944}
 
