@@ -37,6 +37,7 @@ void release(pre_ctx* c) {
     cudaFree(c->d_fused_sync);
     cudaFree(c->d_rs_summary);
     cudaFree(c->d_rs_jtop);
+    cudaFree(c->d_rs_over);
     cudaFree(c->d_rs_guard);
     cudaFree(c->d_rs_handled);
     delete c;
@@ -121,6 +122,7 @@ int pre_create(const pre_config* cfg, pre_ctx** out) {
     if (e == cudaSuccess && c->route_summary_smem) {
         e = alloc_zero(&c->d_rs_summary, (size_t)2 * I);
         if (e == cudaSuccess) e = alloc_zero(&c->d_rs_jtop, (size_t)I);
+        if (e == cudaSuccess) e = alloc_zero(&c->d_rs_over, (size_t)I);
     }
     if (e != cudaSuccess) {
         const bool oom = (e == cudaErrorMemoryAllocation);

@@ -67,8 +67,10 @@ struct pre_ctx {
     // routing on per-row summaries: 0 bytes of shared memory when this shape does not use it
     int route_path;                 // PRE_ROUTE_AUTO / _SCAN / _SUMMARY
     size_t route_summary_smem;
+    size_t route_summary_smem_admit;    // the same for the kernel with the admission queue
     unsigned long long* d_rs_summary;   // [I] {token count, largest cell, largest cell + step, cell 0} per row (16 bytes)
     uint32_t* d_rs_jtop;            // [I] the first step of a row's largest cell + step
+    int32_t* d_rs_over;             // [I] steps of a row above the overload level (admission queue)
     unsigned long long* d_rs_guard; // [8] what the summarising kernel found (largest cell, totals of the batch, ...)
     int* d_rs_handled;              // 1 when the summary kernel routed the last batch, 0 when it left it to the scanning kernel
 };
@@ -115,6 +117,14 @@ cudaError_t pre_launch_ring_step(pre_ctx* ctx, int32_t* prompt, int32_t* generat
 cudaError_t pre_route_configure(pre_ctx* ctx);  // picks G and the shared-memory size
 cudaError_t pre_route_summary_configure(pre_ctx* ctx);   // sets ctx->route_summary_smem (0: this shape keeps the scanning kernel)
 bool pre_route_summary_fits(const pre_ctx* ctx);
+bool pre_route_summary_admit_fits(const pre_ctx* ctx);
+cudaError_t pre_launch_route_summary_admit(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                           int64_t n_arrivals, long long hot, double many, int32_t* queue_prompt,
+                                           int32_t* queue_predicted, int64_t* queue_state, int64_t queue_capacity,
+                                           int32_t* queue_choice, int64_t* curves, int64_t* queued_p,
+                                           int64_t* current_d, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                                           int32_t* instance, int64_t* n_requests, int32_t* choice, double* score,
+                                           cudaStream_t s);
 cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
                                      int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
                                      int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,

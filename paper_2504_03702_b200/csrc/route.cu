@@ -1075,20 +1075,31 @@ cudaError_t pre_launch_route_admit(pre_ctx* ctx, const int32_t* arr_prompt, cons
     // new ones: they read a copy taken here, in stream order.
     cudaError_t e = cudaMemcpyAsync(ctx->d_queue_entry, queue_state, 2 * sizeof(int64_t), cudaMemcpyDeviceToDevice, s);
     if (e != cudaSuccess) return e;
+    // For a whole number c, c > x holds exactly when c > floor(x): the per-cell test is done on integers.
+    double hot = floor(overload_level * (double)ctx->cfg.capacity_tokens);
+    if (hot > 9.2e18) hot = 9.2e18;
+    if (hot < -9.2e18) hot = -9.2e18;
+    const double many = overload_share * (double)ctx->cfg.horizon;
+    // as for pre_route_batch: the summary kernel first where the shape fits it, the scanning kernel behind it
+    const bool summaries = ctx->route_path != PRE_ROUTE_SCAN && pre_route_summary_admit_fits(ctx);
+    if (summaries) {
+        e = pre_launch_route_summary_admit(ctx, arr_prompt, arr_predicted, n_arrivals, (long long)hot, many, queue_prompt,
+                                           queue_predicted, queue_state, queue_capacity, queue_choice, curves, queued_p,
+                                           current_d, prompt, generated, predicted, instance, n_requests, choice, score,
+                                           s);
+        if (e != cudaSuccess) return e;
+    }
     e = cudaMemsetAsync(ctx->d_abort, 0, 3 * sizeof(int), s);
     if (e != cudaSuccess) return e;
     RouteArgs a;
     fill_route_args(a, ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
                     predicted, instance, n_requests, choice, score);
+    if (summaries) a.done_elsewhere = ctx->d_rs_handled;
     a.resident_bytes = ctx->route_resident_bytes_admit;
     a.queue_prompt = queue_prompt; a.queue_predicted = queue_predicted; a.queue_state = queue_state;
     a.queue_entry = ctx->d_queue_entry; a.queue_capacity = queue_capacity; a.queue_choice = queue_choice;
-    // For a whole number c, c > x holds exactly when c > floor(x): the per-cell test is done on integers.
-    double hot = floor(overload_level * (double)ctx->cfg.capacity_tokens);
-    if (hot > 9.2e18) hot = 9.2e18;
-    if (hot < -9.2e18) hot = -9.2e18;
     a.hot = (long long)hot;
-    a.many = overload_share * (double)a.H;
+    a.many = many;
     void* params[] = {(void*)&a};
     return cudaLaunchCooperativeKernel((const void*)pre_route_persistent<true>, dim3(ctx->route_blocks),
                                        dim3(ROUTE_THREADS), params, ctx->route_smem_admit, s);

@@ -145,6 +145,13 @@ struct SumArgs {
     RowSummary* summary;
     uint32_t* jtop;
     unsigned long long* guard;
+    // admission queue (pre_route_admit): steps above the overload level per row, the waiting requests' totals
+    int32_t* over;                 // NULL: not wanted
+    long long hot;
+    const int32_t* queue_prompt;
+    const int32_t* queue_predicted;
+    const int64_t* queue_entry;    // {head, length} as they were when the call was made
+    long long queue_capacity;
 };
 
 // One warp per row.
@@ -156,7 +163,9 @@ __global__ void __launch_bounds__(SUM_THREADS) pre_summarise_rows(const SumArgs 
     if (row < a.I) {
         const int64_t* src = a.curves + (size_t)row * H;
         unsigned int rmax = 0, top = 0, jtop = 0;
+        int above = 0;
         auto take = [&](long long v, int j) {
+            above += v > a.hot;
             bad |= (v < 0) || (v > 0xffffffffLL);
             const unsigned int c = (unsigned int)v;
             rmax = max(rmax, c);
@@ -176,6 +185,8 @@ __global__ void __launch_bounds__(SUM_THREADS) pre_summarise_rows(const SumArgs 
         rmax = __reduce_max_sync(0xffffffffu, rmax);
         const unsigned int t = __reduce_max_sync(0xffffffffu, top);
         const unsigned int jt = __reduce_min_sync(0xffffffffu, top == t ? jtop : 0xffffffffu);
+        above = __reduce_add_sync(0xffffffffu, above);
+        if (lane == 0 && a.over) a.over[row] = above;
         if (lane == 0) {
             const long long q = a.queued_p[row], d = a.current_d[row];
             const long long tok = q + d;
@@ -192,12 +203,23 @@ __global__ void __launch_bounds__(SUM_THREADS) pre_summarise_rows(const SumArgs 
     // the arrivals' own totals: what the batch can add to a cell (ramps) and to a row's token count
     unsigned long long ramp = 0, tokens = 0;
     unsigned int max_pd = 0;
-    for (long long k = (long long)blockIdx.x * SUM_THREADS + tid; k < a.n_arrivals; k += (long long)gridDim.x * SUM_THREADS) {
-        const int P = a.arr_prompt[k], D = a.arr_predicted[k];
-        if (P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX) continue;
+    auto count = [&](int P, int D) {
+        if (P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX) return;
         ramp += (unsigned long long)P + (unsigned long long)(D < H ? D : H);
         tokens += (unsigned long long)P + (unsigned long long)D;
         max_pd = max(max_pd, (unsigned int)P + (unsigned int)D);
+    };
+    for (long long k = (long long)blockIdx.x * SUM_THREADS + tid; k < a.n_arrivals; k += (long long)gridDim.x * SUM_THREADS)
+        count(a.arr_prompt[k], a.arr_predicted[k]);
+    if (a.queue_capacity > 0) {   // the waiting requests are routed before the arrivals
+        long long q_head = a.queue_entry[0], q_len = a.queue_entry[1];
+        if (q_head < 0 || q_head >= a.queue_capacity) q_head = 0;
+        if (q_len < 0) q_len = 0;
+        if (q_len > a.queue_capacity) q_len = a.queue_capacity;
+        for (long long k = (long long)blockIdx.x * SUM_THREADS + tid; k < q_len; k += (long long)gridDim.x * SUM_THREADS) {
+            const long long at = (q_head + k) % a.queue_capacity;
+            count(a.queue_prompt[at], a.queue_predicted[at]);
+        }
     }
     #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -235,13 +257,26 @@ struct RouteSumArgs {
     int* status;
     int* handled;   // 1: this kernel routed the batch; 0: the scanning kernel has to
     int score_warps;
+    // admission queue (ADMIT kernels only): a ring of waiting requests, entry q at (head + q) mod capacity
+    int32_t* queue_prompt;
+    int32_t* queue_predicted;
+    int64_t* queue_state;          // {head, length}, rewritten at the end
+    const int64_t* queue_entry;    // the same two words as they were when the call was made
+    long long queue_capacity;
+    int32_t* queue_choice;         // results for the entries that were waiting at entry
+    long long hot;                 // floor(overload_level * M): a cell counts when it is above
+    double many;                   // overload_share * H: overloaded when more cells than this count
+    const int32_t* over0;          // [I] steps above the level per row, from the summarising kernel
 };
 
 
 // CPT: cells of the folded row per fold thread (H <= CPT * RS_FOLD_THREADS).
 // VEC: H is even, so 16-byte accesses to the rows are legal.
-// The block has RS_FOLD_WARPS fold warps and a.score_warps score warps.
-template <int CPT, bool VEC>
+// The block has RS_FOLD_WARPS fold warps, the control warp and a.score_warps score warps.
+// ADMIT adds the admission queue of Sec. 4.3.3: the requests that were waiting come first; a request that
+// finds every instance overloaded (the scaler's criterion of Sec. 4.3.2: more than `many` steps of the
+// row above `hot`) is not routed and the batch stops there: what is left waits or is turned away.
+template <int CPT, bool VEC, bool ADMIT>
 __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const RouteSumArgs a) {
     extern __shared__ __align__(16) unsigned char rs_smem[];
     const int I = a.I, H = a.H;
@@ -250,6 +285,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
     uint2* aux = tt + Ip;                                   // [Ip] {rmax, c0}
     uint32_t* jst = reinterpret_cast<uint32_t*>(aux + Ip);  // [Ip] jtop
     int* list = reinterpret_cast<int*>(jst + Ip);           // [Ip] binary64 path: rows that have to be scanned
+    int* over = list + Ip;                                  // [Ip] ADMIT: steps of the row above the overload level
     __shared__ Item sh_item[2];             // the arrival to decide, by round parity
     __shared__ int sh_decided[2];           // whether the round decided its arrival
     __shared__ Pending pend[RS_PENDING];
@@ -262,6 +298,12 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
     __shared__ int sh_mode;                 // 0: decline the batch; 1: binary64 scores; 2: whole-number scores
     __shared__ long long sh_n0;
     __shared__ int sh_arr_p[64], sh_arr_d[64];   // the arrivals around the walker's position
+    __shared__ int sh_n_over;               // ADMIT: rows known to be overloaded
+    __shared__ int sh_blocked;              // ADMIT: a request found every instance overloaded ...
+    __shared__ long long sh_blocked_k;      // ... this one
+    __shared__ int sh_warp_ok[RS_MAX_THREADS / 32];
+    __shared__ long long sh_joined;
+    __shared__ int sh_any_bad;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nsw = a.score_warps, nst = 32 * nsw, nthreads = RS_FOLD_THREADS + 32 + nst;
@@ -283,6 +325,11 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
         sh_nlist[0] = sh_nlist[1] = 0;
         sh_jmax = (unsigned int)a.guard[GUARD_MAX_JTOP];
         for (int x = 0; x < RS_PENDING; ++x) pend[x].row = -1;
+        sh_n_over = 0;
+        sh_blocked = 0;
+        sh_blocked_k = 0;
+        sh_joined = 0;
+        sh_any_bad = 0;
     }
     __syncthreads();
     if (sh_mode == 0) {
@@ -297,7 +344,29 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
         tt[i] = make_uint2(q.x, q.z);
         aux[i] = make_uint2(q.y, q.w);
         jst[i] = i < I ? a.jtop0[i] : 0u;
+        if (ADMIT) {
+            over[i] = i < I ? a.over0[i] : 0;
+            if (i < I && (double)over[i] > a.many) atomicAdd(&sh_n_over, 1);
+        }
     }
+    // ADMIT: the requests that were waiting when the call was made come first, then the arrivals
+    long long q_head = 0, q_len = 0;
+    if (ADMIT && a.queue_capacity > 0) {   // kept inside the ring whatever the two words hold
+        q_head = a.queue_entry[0];
+        q_len = a.queue_entry[1];
+        if (q_head < 0 || q_head >= a.queue_capacity) q_head = 0;
+        if (q_len < 0) q_len = 0;
+        if (q_len > a.queue_capacity) q_len = a.queue_capacity;
+    }
+    const long long n_items = q_len + a.n_arrivals;
+    // where the result of item k goes
+    auto put_result = [&](long long k, int c, double sc) {
+        if (ADMIT && k < q_len) a.queue_choice[k] = c;
+        else {
+            a.choice[k - q_len] = c;
+            if (a.score) a.score[k - q_len] = sc;
+        }
+    };
     const long long n0 = sh_n0;
     long long room = a.max_requests - n0;
     if (room < 0) room = 0;
@@ -316,26 +385,33 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
         }
         cp_async_commit();
     };
-    long long cursor = 0, entered = 0;   // (control warp, all lanes alike)
-    int walk_flags = 0;
+    long long cursor = 0, entered = 0;   // (control warp, all lanes alike) items looked at, requests found
+    long long first_bad = 0x7fffffffffffffffLL, first_full = 0x7fffffffffffffffLL;   // the first items dropped as malformed / for a full table
     auto walk_next = [&]() {
         Item it;
         it.P = it.D = it.Dc = 0;
         it.k = -1;
-        while (cursor < a.n_arrivals) {
-            if ((cursor & 31) == 0) {   // a new chunk: its copy was started a chunk ago; start the next one
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
-                __syncwarp();
-                copy_chunk(cursor + 32);
+        while (cursor < n_items) {
+            int P, D;
+            if (ADMIT && cursor < q_len) {
+                const long long at = (q_head + cursor) % a.queue_capacity;
+                P = a.queue_prompt[at];
+                D = a.queue_predicted[at];
+            } else {
+                const long long ac = cursor - q_len;
+                if ((ac & 31) == 0) {   // a new chunk: its copy was started a chunk ago; start the next one
+                    asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    __syncwarp();
+                    copy_chunk(ac + 32);
+                }
+                P = sh_arr_p[ac & 63];
+                D = sh_arr_d[ac & 63];
             }
-            const int P = sh_arr_p[cursor & 63], D = sh_arr_d[cursor & 63];
             const bool bad = P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX;
             if (bad || entered >= room) {
-                walk_flags |= bad ? PRE_ST_BADREQ : PRE_ST_CAPACITY;
-                if (lane == 0) {
-                    a.choice[cursor] = -1;
-                    if (a.score) a.score[cursor] = 0.0;
-                }
+                if (bad && cursor < first_bad) first_bad = cursor;
+                if (!bad && cursor < first_full) first_full = cursor;
+                if (lane == 0) put_result(cursor, -1, 0.0);
                 ++cursor;
                 continue;
             }
@@ -353,7 +429,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
         if (out_w < 0) return;
         if (lane == 0) { a.prompt[out_slot] = out_P; a.generated[out_slot] = 0; }
         if (lane == 1) { a.predicted[out_slot] = out_D; a.instance[out_slot] = out_w; }
-        if (lane == 2) { a.choice[out_k] = out_w; if (a.score) a.score[out_k] = out_score; }
+        if (lane == 2) put_result(out_k, out_w, out_score);
         if (lane == 3) atomicAdd(reinterpret_cast<unsigned long long*>(a.queued_p + out_w), (unsigned long long)out_P);
         if (lane == 4) atomicAdd(reinterpret_cast<unsigned long long*>(a.current_d + out_w), (unsigned long long)out_D);
         out_w = -1;
@@ -409,20 +485,22 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
 
     long long ndec = 0, nfold = 0;   // decisions made, folds done: every thread keeps them
     bool stalled = false;
+    bool blocked = false;            // ADMIT: a request found every instance overloaded: no more decisions, the folds go on
     // Every arrival is decided after at most RS_PENDING stalled rounds and folded RS_LAG rounds later:
     // the loop below ends by itself.  The limit only keeps a mistake in that reasoning from spinning.
-    const long long round_limit = (a.n_arrivals + 2) * (RS_PENDING + 2) + 64;
+    const long long round_limit = (n_items + 2) * (RS_PENDING + 2) + 64;
     bool overrun = false;
     for (long long round = 0;; ++round) {
         if (round > round_limit) { overrun = true; break; }
         const int par = (int)(round & 1);
         const Item it = sh_item[par];
-        const bool have = it.k >= 0;
+        const bool have = it.k >= 0 && !blocked;
         if (!have && nfold == ndec) break;
         const bool do_fold = nfold < ndec && (ndec - nfold >= RS_LAG || !have || stalled);
         unsigned int pend_lb_i = 0xffffffffu;   // (control warp) lower bound of pending entry nfold + lane for this arrival
         double pend_lb_d = CUDART_INF;
         int pend_row = -1;
+        bool pend_uncertain = false;   // ADMIT: that row was not overloaded when it was decided; its fold may change that
         if (warp == RS_CONTROL_WARP) {
             // =============================== control warp, while the pass runs ===============================
             // what does not depend on the pass: the last decision's outputs, the pending rows' lower
@@ -435,6 +513,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                     const unsigned int peak_lb = (unsigned int)it.Dc > p.jw ? (unsigned int)it.P + p.top_lb
                                                                              : max(p.rmax, (unsigned int)it.P + p.c0);
                     pend_row = p.row;
+                    pend_uncertain = ADMIT && p.unused[0] == 0u;
                     if (whole) pend_lb_i = p.tokens + beta_i * whole_over(peak_lb);   // (without the arrival's own P + D, like the pass)
                     else pend_lb_d = summary_score(p.tokens, peak_lb, it.P, it.D, theta, beta);
                 }
@@ -582,10 +661,12 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                     if (cell(u) < Dc) grow[cell(u)] = (long long)c[u];
             }
             unsigned int rmax = 0, top = 0, jtop = 0xffffffffu;
+            int above = 0;
             #pragma unroll
             for (int u = 0; u < CPT; ++u) {   // a thread's steps ascend with u
                 const int j = cell(u);
                 if (j < H) {
+                    if (ADMIT) above += (long long)c[u] > a.hot;
                     rmax = max(rmax, c[u]);
                     const unsigned int t = c[u] + (unsigned int)j;
                     if (jtop == 0xffffffffu || t > top) { top = t; jtop = (unsigned int)j; }
@@ -596,7 +677,11 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
             const unsigned long long tk = warp_max_u64(jtop != 0xffffffffu ? ((unsigned long long)top << 32) | (0xffffffffu - jtop) : 0ull);
             const unsigned int wt = (unsigned int)(tk >> 32);
             const unsigned int wj = tk ? 0xffffffffu - (unsigned int)tk : 0xffffffffu;
-            if (lane == 0) sh_fold[warp] = make_uint4(rmax, wt, wj, 0u);
+            if (ADMIT) {
+                #pragma unroll
+                for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(0xffffffffu, above, off);
+            }
+            if (lane == 0) sh_fold[warp] = make_uint4(rmax, wt, wj, (unsigned int)above);
         }
         __syncthreads();   // the pass and the fold's per-warp maxima are complete
         if (warp == RS_CONTROL_WARP) {
@@ -632,6 +717,18 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                     if (pend_row == b1r || could_win) stall = true;
                 }
                 stall = __any_sync(0xffffffffu, stall);
+                if (ADMIT) {
+                    // every instance overloaded?  Rows are counted once their state is known; a pending row that was
+                    // not overloaded when it was decided may have become so.
+                    const int uncertain = __popc(__ballot_sync(0xffffffffu, pend_uncertain));
+                    const int n_over = sh_n_over;
+                    if (n_over >= I) {   // the request is not routed: the batch stops here
+                        stall = true;
+                        if (lane == 0) { sh_blocked = 1; sh_blocked_k = it.k; }
+                    } else if (n_over + uncertain >= I) {
+                        stall = true;
+                    }
+                }
                 if (!stall) {
                     // the row is pending from now on: exact token count, bounds for the rest
                     const int w = b1r;
@@ -641,7 +738,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                         uint4* dst = reinterpret_cast<uint4*>(&pend[ndec % RS_PENDING]);
                         dst[0] = make_uint4((unsigned int)w, (unsigned int)P, (unsigned int)D, (unsigned int)Dc);
                         dst[1] = make_uint4(q.x + PD, q.y + ((int)jw < Dc ? (unsigned int)P + jw : 0u), jw, x.x);
-                        dst[2] = make_uint4(x.y + (unsigned int)P, 0u, 0u, 0u);
+                        dst[2] = make_uint4(x.y + (unsigned int)P, (ADMIT && (double)over[w] > a.many) ? 1u : 0u, 0u, 0u);
                         tt[w] = make_uint2(RS_OUT, 0u);
                         *reinterpret_cast<uint4*>(&sh_item[par ^ 1]) = make_uint4((unsigned int)nxt.P, (unsigned int)nxt.D, (unsigned int)nxt.Dc, (unsigned int)nxt.k);
                     }
@@ -664,9 +761,11 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
             // ---- the folded row's new summary; the row takes part in the next pass again
             const Pending p = pend[nfold % RS_PENDING];
             unsigned int rmax = 0, top = 0, jtop = 0xffffffffu;
+            int above = 0;
             #pragma unroll
             for (int x = 0; x < RS_FOLD_WARPS; ++x) {   // the first step at which the largest cell + step is taken
                 const uint4 q = sh_fold[x];
+                above += (int)q.w;
                 rmax = max(rmax, q.x);
                 if (q.z != 0xffffffffu && (jtop == 0xffffffffu || q.y > top || (q.y == top && q.z < jtop))) { top = q.y; jtop = q.z; }
             }
@@ -674,6 +773,11 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
             aux[p.row] = make_uint2(rmax, c[0]);
             jst[p.row] = jtop;
             if (jtop > sh_jmax) sh_jmax = jtop;
+            if (ADMIT) {
+                const bool was = (double)over[p.row] > a.many;
+                over[p.row] = above;
+                if (!was && (double)above > a.many) sh_n_over += 1;
+            }
             tt[p.row] = make_uint2(p.tokens, top);
         }
         __syncthreads();
@@ -684,14 +788,70 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
             stalled = false;
         }
         if (do_fold) ++nfold;
+        if (ADMIT && sh_blocked) blocked = true;
     }
     if (warp == RS_CONTROL_WARP) flush_outputs();
     if (overrun && tid == 0) atomicOr(a.status, PRE_ST_TIMEOUT);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (tid == RS_FOLD_THREADS) {   // the control warp kept the walker's counts
-        *a.n_requests = n0 + entered;
-        if (walk_flags) atomicOr(a.status, walk_flags);
+    // what the walker noted beyond a blocked request is decided again below and does not count here
+    const long long decided = (ADMIT && blocked) ? sh_blocked_k : n_items;
+    if (tid == RS_FOLD_THREADS) {   // the control warp kept the walker's notes
+        *a.n_requests = n0 + ndec;
+        int flags = 0;
+        if (first_bad < decided) flags |= PRE_ST_BADREQ;
+        if (first_full < decided) flags |= PRE_ST_CAPACITY;
+        if (flags) atomicOr(a.status, flags);
         *a.handled = 1;
+    }
+    if (ADMIT) {
+        // Everything from the blocked request on: a request that was waiting keeps its place; an arrival joins
+        // the tail of the queue while there is room and is turned away otherwise (a malformed arrival is
+        // dropped).  Nothing else reads or writes these arrays any more.
+        __syncthreads();
+        const long long stop = decided;
+        const long long left = stop < q_len ? q_len - stop : 0;          // waiting entries that stay
+        for (long long k = stop + tid; k < q_len; k += nthreads) a.queue_choice[k] = -2;
+        const long long a0 = (stop > q_len ? stop : q_len) - q_len;      // first arrival that was not decided
+        const int nw = nthreads >> 5;
+        for (long long base = a0; base < a.n_arrivals; base += nthreads) {
+            const long long i = base + tid;
+            int P = -1, D = 0;
+            if (i < a.n_arrivals) { P = a.arr_prompt[i]; D = a.arr_predicted[i]; }
+            const bool ok = i < a.n_arrivals && !(P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX);
+            const unsigned int vote = __ballot_sync(0xffffffffu, ok);
+            if (lane == 0) sh_warp_ok[warp] = __popc(vote);
+            __syncthreads();
+            long long rank = sh_joined + __popc(vote & ((1u << lane) - 1u));
+            int total = 0;
+            for (int x = 0; x < nw; ++x) { if (x < warp) rank += sh_warp_ok[x]; total += sh_warp_ok[x]; }
+            if (i < a.n_arrivals) {
+                int c = -1;
+                if (ok) {
+                    if (left + rank < a.queue_capacity) {
+                        const long long pos = (q_head + q_len + rank) % a.queue_capacity;   // behind the last one waiting
+                        a.queue_prompt[pos] = P;
+                        a.queue_predicted[pos] = D;
+                        c = -2;
+                    } else {
+                        c = -3;
+                    }
+                } else {
+                    sh_any_bad = 1;
+                }
+                a.choice[i] = c;
+                if (a.score) a.score[i] = 0.0;
+            }
+            __syncthreads();
+            if (tid == 0) sh_joined += total;
+            __syncthreads();
+        }
+        if (tid == 0) {
+            long long joined = sh_joined;
+            if (left + joined > a.queue_capacity) joined = a.queue_capacity - left;
+            a.queue_state[0] = a.queue_capacity > 0 ? (q_head + (q_len - left)) % a.queue_capacity : 0;
+            a.queue_state[1] = left + joined;
+            if (blocked && sh_any_bad) atomicOr(a.status, PRE_ST_BADREQ);
+        }
     }
 }
 
@@ -699,9 +859,9 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
 
 // ---- host side
 
-static size_t summaries_smem_bytes(int I) {
+static size_t summaries_smem_bytes(int I, bool admit) {
     const size_t Ip = (size_t)((I + 31) & ~31);
-    return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + sizeof(int));
+    return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + sizeof(int) + (admit ? sizeof(int) : 0));
 }
 
 // Score warps: about sixteen rows per score thread (measured: 4,096 instances are fastest with 8 score warps,
@@ -712,58 +872,64 @@ static int summaries_score_warps(int I) {
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
 
-template <int CPT>
+template <int CPT, bool ADMIT>
 static const void* summaries_kernel(bool vec) {
-    return vec ? (const void*)pre_route_summaries<CPT, true> : (const void*)pre_route_summaries<CPT, false>;
+    return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT> : (const void*)pre_route_summaries<CPT, false, ADMIT>;
 }
+template <bool ADMIT>
 static const void* summaries_kernel_for(int H) {
     const bool vec = (H & 1) == 0;
-    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4>(vec);
-    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8>(vec);
-    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16>(vec);
-    return summaries_kernel<32>(vec);
+    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4, ADMIT>(vec);
+    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8, ADMIT>(vec);
+    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16, ADMIT>(vec);
+    return summaries_kernel<32, ADMIT>(vec);
 }
 
-cudaError_t pre_route_summary_configure(pre_ctx* ctx) {
+template <bool ADMIT>
+static cudaError_t summaries_configure_one(pre_ctx* ctx, size_t limit, size_t* smem_out) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
-    ctx->route_summary_smem = 0;
-    if (H > 32 * RS_FOLD_THREADS) return cudaSuccess;
-    cudaDeviceProp prop;
-    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
-    if (e != cudaSuccess) return e;
-    const void* fn = summaries_kernel_for(H);
+    *smem_out = 0;
+    const void* fn = summaries_kernel_for<ADMIT>(H);
     cudaFuncAttributes attr;
-    e = cudaFuncGetAttributes(&attr, fn);
+    cudaError_t e = cudaFuncGetAttributes(&attr, fn);
     if (e != cudaSuccess) return e;
-    const size_t limit = (size_t)prop.sharedMemPerBlockOptin;
-    const size_t smem = summaries_smem_bytes(I);
+    const size_t smem = summaries_smem_bytes(I, ADMIT);
     if (smem + attr.sharedSizeBytes + 256 > limit) return cudaSuccess;   // too many instances
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    ctx->route_summary_smem = smem;
+    *smem_out = smem;
     return cudaSuccess;
 }
 
-bool pre_route_summary_fits(const pre_ctx* ctx) { return ctx->route_summary_smem != 0 && ctx->d_rs_summary != nullptr; }
-
-cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
-                                     int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
-                                     int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
-                                     int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
-    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
-    cudaError_t e = cudaMemsetAsync(ctx->d_rs_guard, 0, 8 * sizeof(unsigned long long), s);
+cudaError_t pre_route_summary_configure(pre_ctx* ctx) {
+    ctx->route_summary_smem = 0;
+    ctx->route_summary_smem_admit = 0;
+    if (ctx->cfg.horizon > 32 * RS_FOLD_THREADS) return cudaSuccess;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, ctx->device);
     if (e != cudaSuccess) return e;
-    SumArgs p;
+    e = summaries_configure_one<false>(ctx, (size_t)prop.sharedMemPerBlockOptin, &ctx->route_summary_smem);
+    if (e != cudaSuccess) return e;
+    return summaries_configure_one<true>(ctx, (size_t)prop.sharedMemPerBlockOptin, &ctx->route_summary_smem_admit);
+}
+
+bool pre_route_summary_fits(const pre_ctx* ctx) { return ctx->route_summary_smem != 0 && ctx->d_rs_summary != nullptr; }
+bool pre_route_summary_admit_fits(const pre_ctx* ctx) {
+    return ctx->route_summary_smem_admit != 0 && ctx->d_rs_summary != nullptr && ctx->d_rs_over != nullptr;
+}
+
+static void fill_summary_args(pre_ctx* ctx, SumArgs& p, RouteSumArgs& a, const int32_t* arr_prompt,
+                              const int32_t* arr_predicted, int64_t n_arrivals, int64_t* curves, int64_t* queued_p,
+                              int64_t* current_d, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                              int32_t* instance, int64_t* n_requests, int32_t* choice, double* score) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     p.curves = curves; p.queued_p = queued_p; p.current_d = current_d;
     p.arr_prompt = arr_prompt; p.arr_predicted = arr_predicted; p.n_arrivals = n_arrivals;
     p.I = I; p.H = H;
     p.summary = reinterpret_cast<RowSummary*>(ctx->d_rs_summary);
     p.jtop = ctx->d_rs_jtop; p.guard = ctx->d_rs_guard;
-    const int rows_per_block = SUM_THREADS / 32;
-    pre_summarise_rows<<<(I + rows_per_block - 1) / rows_per_block, SUM_THREADS, 0, s>>>(p);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    RouteSumArgs a;
+    p.over = nullptr; p.hot = 0; p.queue_prompt = nullptr; p.queue_predicted = nullptr; p.queue_entry = nullptr;
+    p.queue_capacity = 0;
     a.arr_prompt = arr_prompt; a.arr_predicted = arr_predicted; a.n_arrivals = n_arrivals;
     a.curves = curves; a.queued_p = queued_p; a.current_d = current_d;
     a.prompt = prompt; a.generated = generated; a.predicted = predicted; a.instance = instance;
@@ -774,7 +940,52 @@ cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, co
     a.summary0 = p.summary; a.jtop0 = p.jtop; a.guard = p.guard;
     a.status = ctx->d_status; a.handled = ctx->d_rs_handled;
     a.score_warps = summaries_score_warps(I);
+    a.queue_prompt = nullptr; a.queue_predicted = nullptr; a.queue_state = nullptr; a.queue_entry = nullptr;
+    a.queue_capacity = 0; a.queue_choice = nullptr; a.hot = 0; a.many = 0.0; a.over0 = nullptr;
+}
+
+template <bool ADMIT>
+static cudaError_t launch_summary_kernels(pre_ctx* ctx, const SumArgs& p, const RouteSumArgs& a, cudaStream_t s) {
+    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    cudaError_t e = cudaMemsetAsync(ctx->d_rs_guard, 0, 8 * sizeof(unsigned long long), s);
+    if (e != cudaSuccess) return e;
+    const int rows_per_block = SUM_THREADS / 32;
+    pre_summarise_rows<<<(I + rows_per_block - 1) / rows_per_block, SUM_THREADS, 0, s>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     void* params[] = {(void*)&a};
-    return cudaLaunchKernel(summaries_kernel_for(H), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
-                            ctx->route_summary_smem, s);
+    return cudaLaunchKernel(summaries_kernel_for<ADMIT>(H), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
+                            ADMIT ? ctx->route_summary_smem_admit : ctx->route_summary_smem, s);
+}
+
+cudaError_t pre_launch_route_summary(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                     int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
+                                     int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
+                                     int64_t* n_requests, int32_t* choice, double* score, cudaStream_t s) {
+    SumArgs p;
+    RouteSumArgs a;
+    fill_summary_args(ctx, p, a, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
+                      predicted, instance, n_requests, choice, score);
+    return launch_summary_kernels<false>(ctx, p, a, s);
+}
+
+// The queue's head and length must have been copied to ctx->d_queue_entry on the stream before this call.
+cudaError_t pre_launch_route_summary_admit(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
+                                           int64_t n_arrivals, long long hot, double many, int32_t* queue_prompt,
+                                           int32_t* queue_predicted, int64_t* queue_state, int64_t queue_capacity,
+                                           int32_t* queue_choice, int64_t* curves, int64_t* queued_p,
+                                           int64_t* current_d, int32_t* prompt, int32_t* generated, int32_t* predicted,
+                                           int32_t* instance, int64_t* n_requests, int32_t* choice, double* score,
+                                           cudaStream_t s) {
+    SumArgs p;
+    RouteSumArgs a;
+    fill_summary_args(ctx, p, a, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt, generated,
+                      predicted, instance, n_requests, choice, score);
+    p.over = ctx->d_rs_over; p.hot = hot;
+    p.queue_prompt = queue_prompt; p.queue_predicted = queue_predicted; p.queue_entry = ctx->d_queue_entry;
+    p.queue_capacity = queue_capacity;
+    a.queue_prompt = queue_prompt; a.queue_predicted = queue_predicted; a.queue_state = queue_state;
+    a.queue_entry = ctx->d_queue_entry; a.queue_capacity = queue_capacity; a.queue_choice = queue_choice;
+    a.hot = hot; a.many = many; a.over0 = ctx->d_rs_over;
+    return launch_summary_kernels<true>(ctx, p, a, s);
 }

@@ -572,7 +572,7 @@ def admit_both(st, ref, ap, ad, level, share, what=""):
 
 @pytest.mark.parametrize("idx,level,first_blocked", [(0, 0.6, 25), (1, 0.6, 335), (2, 0.3, 5979), (1, 0.95, None),
                                                      (0, 0.3, 0)])
-def test_admit_configs(idx, level, first_blocked):
+def test_admit_configs(idx, level, first_blocked, router):
     wl = W.make_config(idx)
     st, ref = both_with_queue(wl, 100)
     ap, ad = wl.ticks[0]
@@ -585,7 +585,7 @@ def test_admit_configs(idx, level, first_blocked):
     st.close()
 
 
-def test_admit_never_blocking_equals_route_batch():
+def test_admit_never_blocking_equals_route_batch(router):
     wl = W.make_config(1)
     st, ref = both_with_queue(wl, 10)
     plain = DeviceState.from_workload(wl)
@@ -602,7 +602,7 @@ def test_admit_never_blocking_equals_route_batch():
                                                           (13, 5, 16, 80, 60, 100, 0.5), (14, 1, 4, 6, 12, 3, 0.9),
                                                           (15, 4, 12, 50, 64, 7, 0.7), (16, 300, 64, 4000, 900, 64, 0.8),
                                                           (17, 149, 128, 3000, 700, 1000, 0.75)])
-def test_admit_shapes_over_several_calls(seed, n_inst, h, n, a, qcap, level):
+def test_admit_shapes_over_several_calls(seed, n_inst, h, n, a, qcap, level, router):
     """Calls alternate with decode steps: requests wait, are routed later, the ring's head moves on."""
     wl = W.make_random(seed, n_inst, h, n, a, max_prompt=30, max_output=20)
     st, ref = both_with_queue(wl, qcap)
@@ -622,7 +622,7 @@ def test_admit_shapes_over_several_calls(seed, n_inst, h, n, a, qcap, level):
     st.close()
 
 
-def test_admit_long_tail_after_the_block_and_malformed_arrivals():
+def test_admit_long_tail_after_the_block_and_malformed_arrivals(router):
     """Thousands of arrivals behind the blocked one: they join the queue in order until it is full."""
     wl = W.make_config(2)
     st, ref = both_with_queue(wl, 1500)
@@ -645,7 +645,7 @@ def test_admit_long_tail_after_the_block_and_malformed_arrivals():
     st.close()
 
 
-def test_admit_table_full_and_empty_call():
+def test_admit_table_full_and_empty_call(router):
     wl = W.make_random(31, 4, 16, 20, 12)
     wl.max_requests = 25
     st, ref = both_with_queue(wl, 8)

@@ -64,6 +64,7 @@ def test_admission_router_wait_that_runs_out():
     ap, ad = wl.ticks[0]
     ap, ad = ap[:128], ad[:128]
     st.make_queue(16)
+    st.select_router(B.ROUTE_SCAN)      # the kernel whose blocks wait for one another
     B.pre_test_set_spin_limit(st.ctx, 0)
     _, choice, score = st.route_admit(dev(ap), dev(ad), overload_level=0.95, overload_share=0.10)
     assert st.status() == B.PRE_ETIMEOUT
