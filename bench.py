@@ -429,7 +429,8 @@ def extras_leg(res, wl, index, device):
     t_admit = e0.elapsed_time(e1)
     out["route_admit"] = {"routed": int((adm_choice >= 0).sum()), "waiting": int((adm_choice == -2).sum()),
                           "turned_away": int((adm_choice == -3).sum()), "ms": t_admit,
-                          "decided_per_s": a / (t_admit * 1e-3), "kernel": "pre_route_persistent<admit>",
+                          "decided_per_s": a / (t_admit * 1e-3),
+                          "kernel": "pre_route_summaries<admit>" if res["route_kernel"] == "summary" else "pre_route_persistent<admit>",
                           "overload_level": 0.95, "overload_share": 0.10, "queue_capacity": 4096,
                           "note": "separate call, not part of the step; same batch, same maps"}
     B.check(st.status(), "admission call")
@@ -440,8 +441,7 @@ def extras_leg(res, wl, index, device):
             "pre_route_batch")
     st.step()
 
-    # the scanning kernel on the first arrivals of the same batch (it routes what the summary kernel declines,
-    # and every call of the admission router)
+    # the scanning kernel on the first arrivals of the same batch (it routes what the summary kernel declines)
     if res["route_kernel"] == "summary":
         n_scan = min(a, 8192)
         st.select_router(B.ROUTE_SCAN)

@@ -308,7 +308,7 @@ int pre_status(pre_ctx* ctx, void* stream);
 /* The cudaError_t value of the last failed runtime call on this context (0 if none). */
 int pre_last_cuda_error(const pre_ctx* ctx);
 
-/* Which kernel routes the batches of pre_route_batch on this context: PRE_ROUTE_AUTO (default:
+/* Which kernel routes the batches of pre_route_batch and pre_route_admit on this context: PRE_ROUTE_AUTO (default:
  * the summary kernel when the shape fits it, the scanning kernel otherwise or when the summary
  * kernel declines a batch), PRE_ROUTE_SCAN (always the scanning kernel), PRE_ROUTE_SUMMARY (as
  * AUTO, but PRE_ESIZE here when the shape does not fit the summary kernel).  Results do not
