@@ -276,8 +276,9 @@ struct RouteSumArgs {
 // ADMIT adds the admission queue of Sec. 4.3.3: the requests that were waiting come first; a request that
 // finds every instance overloaded (the scaler's criterion of Sec. 4.3.2: more than `many` steps of the
 // row above `hot`) is not routed and the batch stops there: what is left waits or is turned away.
-template <int CPT, bool VEC, bool ADMIT>
-__global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const RouteSumArgs a) {
+// MAXT: the largest block this instantiation is launched with (a smaller one leaves the compiler more registers).
+template <int CPT, bool VEC, bool ADMIT, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArgs a) {
     extern __shared__ __align__(16) unsigned char rs_smem[];
     const int I = a.I, H = a.H;
     const int Ip = (I + 31) & ~31;
@@ -301,7 +302,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
     __shared__ int sh_n_over;               // ADMIT: rows known to be overloaded
     __shared__ int sh_blocked;              // ADMIT: a request found every instance overloaded ...
     __shared__ long long sh_blocked_k;      // ... this one
-    __shared__ int sh_warp_ok[RS_MAX_THREADS / 32];
+    __shared__ int sh_warp_ok[RS_MAX_THREADS / 32];   // (the tail of ADMIT)
     __shared__ long long sh_joined;
     __shared__ int sh_any_bad;
 
@@ -872,24 +873,31 @@ static int summaries_score_warps(int I) {
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
 
+constexpr int RS_SMALL_THREADS = 640;   // blocks of up to 10 score warps get the instantiation with more registers
+
 template <int CPT, bool ADMIT>
-static const void* summaries_kernel(bool vec) {
-    return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT> : (const void*)pre_route_summaries<CPT, false, ADMIT>;
+static const void* summaries_kernel(bool vec, bool small) {
+    if (small)
+        return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT, RS_SMALL_THREADS>
+                   : (const void*)pre_route_summaries<CPT, false, ADMIT, RS_SMALL_THREADS>;
+    return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT, RS_MAX_THREADS>
+               : (const void*)pre_route_summaries<CPT, false, ADMIT, RS_MAX_THREADS>;
 }
 template <bool ADMIT>
-static const void* summaries_kernel_for(int H) {
+static const void* summaries_kernel_for(int H, int I) {
     const bool vec = (H & 1) == 0;
-    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4, ADMIT>(vec);
-    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8, ADMIT>(vec);
-    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16, ADMIT>(vec);
-    return summaries_kernel<32, ADMIT>(vec);
+    const bool small = RS_FOLD_THREADS + 32 + 32 * summaries_score_warps(I) <= RS_SMALL_THREADS;
+    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4, ADMIT>(vec, small);
+    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8, ADMIT>(vec, small);
+    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16, ADMIT>(vec, small);
+    return summaries_kernel<32, ADMIT>(vec, small);
 }
 
 template <bool ADMIT>
 static cudaError_t summaries_configure_one(pre_ctx* ctx, size_t limit, size_t* smem_out) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     *smem_out = 0;
-    const void* fn = summaries_kernel_for<ADMIT>(H);
+    const void* fn = summaries_kernel_for<ADMIT>(H, I);
     cudaFuncAttributes attr;
     cudaError_t e = cudaFuncGetAttributes(&attr, fn);
     if (e != cudaSuccess) return e;
@@ -954,7 +962,7 @@ static cudaError_t launch_summary_kernels(pre_ctx* ctx, const SumArgs& p, const 
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     void* params[] = {(void*)&a};
-    return cudaLaunchKernel(summaries_kernel_for<ADMIT>(H), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
+    return cudaLaunchKernel(summaries_kernel_for<ADMIT>(H, I), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
                             ADMIT ? ctx->route_summary_smem_admit : ctx->route_summary_smem, s);
 }
 
