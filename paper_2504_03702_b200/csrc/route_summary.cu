@@ -37,7 +37,6 @@
 #include <math_constants.h>
 
 #include <cmath>
-#include <cstdlib>
 
 namespace {
 
@@ -869,7 +868,6 @@ static size_t summaries_smem_bytes(int I, bool admit) {
 // 1,024 with 2 to 4; more warps lengthen the block barriers more than they shorten the pass).
 static int summaries_score_warps(int I) {
     int w = (I + 16 * 32 - 1) / (16 * 32);
-    if (const char* e = getenv("PRE_RS_SCORE_WARPS")) w = atoi(e);
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
 
