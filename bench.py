@@ -36,24 +36,24 @@ METRIC_STREAM = "routes/sec over the whole stream (decode step + routing of the 
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (configuration 3; other
 # configurations report null).  profiles/ncu_full_route_scan_kernel_config3_256_arrivals.txt: the scanning routing kernel
-# reads the maps once per launch, whatever the batch length (67.32 MB), and wrote 639,488 B for 256 arrivals
+# reads the maps once per launch, whatever the batch length (67.32 MB), and wrote 688,640 B for 256 arrivals
 # (folded cells, appended requests): the written part is scaled to the batch.  The single-launch build reads the
 # table and moves the tiles' lists; most of the 64 MiB of maps is still in L2 when the launch ends, which is why
 # its figure is below the algorithmic bytes.  pre_step: its two kernels added.
 # profiles/ncu_full_tick_scaler_refine_config3.txt: refinement and the fused tick (two kernels added).
-ROUTE_DRAM_READ = {3: 67317760}
+ROUTE_DRAM_READ = {3: 67315968}
 # profiles/ncu_dram_route_summary_kernels_config3_full_batch.txt: both kernels of the summary router on the full
 # batch (the traffic does not grow in proportion to the batch, so the figure is used for the full batch only)
-ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67720000 + 124160 + 55920000 + 5480000}
+ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67730000 + 411900 + 55920000 + 5980000}
 # warp instructions per arrival of pre_route_summaries (smsp__inst_executed.sum of the 2,048-arrival capture in
-# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 12,760,381 / 2,048)
-ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 12760381 / 2048}
-ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 639488 / 256}
-ANTICIPATE_DRAM_TRAFFIC = {3: 33807616 + 20817152}
-STEP_DRAM_TRAFFIC = {3: 33669120 + 67196160 + 9473792}
+# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 11,746,427 / 2,048)
+ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 11746427 / 2048}
+ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 688640 / 256}
+ANTICIPATE_DRAM_TRAFFIC = {3: 33809408 + 19726848}
+STEP_DRAM_TRAFFIC = {3: 33669376 + 67196160 + 9161472}
 SCALER_DRAM_TRAFFIC = {3: 67128576 + 326912}   # profiles/ncu_full_scaler_rows_config3.txt
-REFINE_DRAM_TRAFFIC = {3: 44150272 + 29952}
-TICK_DRAM_TRAFFIC = {3: 44136960 + 50176 + 67199488 + 10226944}
+REFINE_DRAM_TRAFFIC = {3: 44150272 + 30208}
+TICK_DRAM_TRAFFIC = {3: 44138240 + 40704 + 67201536 + 9018624}
 
 
 def measured_peak_gbs():
