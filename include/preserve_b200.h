@@ -309,8 +309,8 @@ int pre_status(pre_ctx* ctx, void* stream);
 int pre_last_cuda_error(const pre_ctx* ctx);
 
 /* Which kernel routes the batches of pre_route_batch and pre_route_admit on this context: PRE_ROUTE_AUTO (default:
- * the summary kernel when the shape fits it, the scanning kernel otherwise or when the summary
- * kernel declines a batch), PRE_ROUTE_SCAN (always the scanning kernel), PRE_ROUTE_SUMMARY (as
+ * the summary kernel when the shape fits it and beta and t_mem * M are whole numbers - its fast case -, the
+ * scanning kernel otherwise or when the summary kernel declines a batch), PRE_ROUTE_SCAN (always the scanning kernel), PRE_ROUTE_SUMMARY (as
  * AUTO, but PRE_ESIZE here when the shape does not fit the summary kernel).  Results do not
  * depend on it. */
 #define PRE_ROUTE_AUTO    0

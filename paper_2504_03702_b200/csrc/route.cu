@@ -1038,6 +1038,17 @@ static void fill_route_args(RouteArgs& a, pre_ctx* ctx, const int32_t* arr_promp
     a.queue_capacity = 0; a.queue_choice = nullptr; a.hot = 0; a.many = 0.0;
 }
 
+// PRE_ROUTE_AUTO takes the summary kernel when its scores are whole numbers (beta and t_mem * M whole: one
+// integer pass per arrival); with binary64 scores it needs two passes and a few binary64 evaluations per arrival
+// and is slower than the scanning kernel (measured: 3.96 against 3.11 us per arrival on 4,096 x 2,048), so it runs
+// them only when it is selected outright.
+static bool pre_route_summary_wanted(const pre_ctx* ctx) {
+    if (ctx->route_path == PRE_ROUTE_SCAN) return false;
+    if (ctx->route_path == PRE_ROUTE_SUMMARY) return true;
+    const double beta = ctx->cfg.beta, theta = ctx->theta;
+    return beta == floor(beta) && theta == floor(theta) && beta <= 1048576.0 && theta < 1073741824.0;
+}
+
 cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int32_t* arr_predicted,
                              int64_t n_arrivals, int64_t* curves, int64_t* queued_p, int64_t* current_d,
                              int32_t* prompt, int32_t* generated, int32_t* predicted, int32_t* instance,
@@ -1046,7 +1057,7 @@ cudaError_t pre_launch_route(pre_ctx* ctx, const int32_t* arr_prompt, const int3
     // The summary kernel takes the batch when the shape fits it; it declines (on the device) when 32-bit
     // arithmetic could overflow during the batch, and the scanning kernel launched behind it then does
     // the work.  When the summary kernel has routed the batch the scanning kernel returns at once.
-    const bool summaries = ctx->route_path != PRE_ROUTE_SCAN && pre_route_summary_fits(ctx);
+    const bool summaries = pre_route_summary_wanted(ctx) && pre_route_summary_fits(ctx);
     cudaError_t e = cudaSuccess;
     if (summaries) {
         e = pre_launch_route_summary(ctx, arr_prompt, arr_predicted, n_arrivals, curves, queued_p, current_d, prompt,
@@ -1081,7 +1092,7 @@ cudaError_t pre_launch_route_admit(pre_ctx* ctx, const int32_t* arr_prompt, cons
     if (hot < -9.2e18) hot = -9.2e18;
     const double many = overload_share * (double)ctx->cfg.horizon;
     // as for pre_route_batch: the summary kernel first where the shape fits it, the scanning kernel behind it
-    const bool summaries = ctx->route_path != PRE_ROUTE_SCAN && pre_route_summary_admit_fits(ctx);
+    const bool summaries = pre_route_summary_wanted(ctx) && pre_route_summary_admit_fits(ctx);
     if (summaries) {
         e = pre_launch_route_summary_admit(ctx, arr_prompt, arr_predicted, n_arrivals, (long long)hot, many, queue_prompt,
                                            queue_predicted, queue_state, queue_capacity, queue_choice, curves, queued_p,

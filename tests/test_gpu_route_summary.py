@@ -202,3 +202,42 @@ def test_streaming_ticks_on_both_kernels():
         assert_scores_close(score.cpu().numpy(), want_s, want_c)
     assert_state_equal(st, ref)
     st.close()
+
+
+@pytest.mark.parametrize("beta,level", [(1.0, 0.7), (0.75, 0.7), (0.4, 0.5)])
+def test_admission_queue_on_the_summary_kernel(beta, level):
+    """Several calls with a queue that fills and drains, whole-number and binary64 scores, the kernel selected outright."""
+    wl = W.make_random(96, 5, 24, 120, 0, max_prompt=200, max_output=60, beta=beta)
+    wl.max_requests = 120 + 400
+    st = DeviceState.from_workload(wl)
+    st.select_router(B.ROUTE_SUMMARY)
+    ref = oracle.State.from_workload(wl)
+    st.anticipate()
+    ref.anticipate()
+    st.make_queue(12)
+    ref.make_queue(12)
+    rng = np.random.default_rng(14)
+    seen = set()
+    for call in range(10):
+        a = int(rng.integers(0, 40))
+        ap = rng.integers(0, 200, a).astype(np.int32)
+        ad = rng.integers(1, 60, a).astype(np.int32)
+        if a > 3 and call % 3 == 1:
+            ad[1] = 0                                   # malformed
+        waiting = int(ref.queue_state[1])
+        qc, c, s = st.route_admit(dev(ap), dev(ad), overload_level=level, overload_share=0.10)
+        wqc, wc, ws = ref.route_admit(ap, ad, overload_level=level, overload_share=0.10)
+        assert (c.cpu().numpy() == wc).all(), f"call {call}: arrivals"
+        assert (qc[:waiting].cpu().numpy() == wqc).all(), f"call {call}: waiting requests"
+        assert_scores_close(s.cpu().numpy(), ws, wc)
+        assert st.queue_state.cpu().tolist() == ref.queue_state.tolist()
+        assert_state_equal(st, ref, f"after call {call}")
+        seen.update(np.unique(wc).tolist())
+        seen.update((-10 - v for v in np.unique(wqc).tolist() if v >= 0))
+        st.status()
+        for _ in range(int(rng.integers(0, 4))):
+            st.step()
+            ref.step()
+    assert -2 in seen and -3 in seen and any(v >= 0 for v in seen) and any(v <= -10 for v in seen), \
+        "the case was meant to route, queue, turn away and route out of the queue"
+    st.close()
