@@ -54,12 +54,12 @@ constexpr int RS_PENDING = RS_LAG + 1;     // rows that can be pending at once (
 // estimate + 2 * beta * theta: eight roundings of 2^-24 each on terms that add up to at most that
 // (2^-21), taken four times as large.
 constexpr float RS_EPS = 1.9073486328125e-06f;   // 2^-19
+constexpr int RS_ROWS_PER_LANE = 16;       // rows of one score lane at most (the host picks the score warps accordingly)
 constexpr int SUM_THREADS = 256;
 // whole-number scores: token count of a row that is left out of the pass (pending, or padding)
 constexpr unsigned int RS_OUT = 0xc0000000u;
 
 // named barriers (0 is __syncthreads)
-constexpr int BAR_SCORE = 1;    // among the score warps
 
 // guard words written by the summarising kernel
 constexpr int GUARD_MAX_CELL = 0, GUARD_MAX_BASE = 1, GUARD_BAD = 2, GUARD_SUM_RAMP = 3, GUARD_SUM_TOKENS = 4,
@@ -114,10 +114,6 @@ __device__ __forceinline__ unsigned int warp_max_u32(unsigned int v) {
     return v;
 }
 
-__device__ __forceinline__ void bar_sync(int id, int count) {
-    __syncwarp();
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
 
 // Score of one instance, binary64, every operation rounded on its own (the sums of whole
 // numbers below 2^53 are exact, so adding the two token counts first changes nothing).
@@ -284,15 +280,12 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     uint2* tt = reinterpret_cast<uint2*>(rs_smem);          // [Ip] {token count (RS_OUT: left out of the pass), top}
     uint2* aux = tt + Ip;                                   // [Ip] {rmax, c0}
     uint32_t* jst = reinterpret_cast<uint32_t*>(aux + Ip);  // [Ip] jtop
-    int* list = reinterpret_cast<int*>(jst + Ip);           // [Ip] binary64 path: rows that have to be scanned
-    int* over = list + Ip;                                  // [Ip] ADMIT: steps of the row above the overload level
+    int* over = reinterpret_cast<int*>(jst + Ip);           // [Ip] ADMIT: steps of the row above the overload level
     __shared__ Item sh_item[2];             // the arrival to decide, by round parity
     __shared__ int sh_decided[2];           // whether the round decided its arrival
     __shared__ Pending pend[RS_PENDING];
     __shared__ unsigned long long sh_wkey[2][RS_MAX_SCORE_WARPS];   // the warps' best rows: score bits (binary64) or score << 32 | row
     __shared__ int sh_wrow[2][RS_MAX_SCORE_WARPS];
-    __shared__ unsigned int sh_emin[2];     // bits of the block's smallest binary32 upper estimate, by round parity
-    __shared__ int sh_nlist[2];
     __shared__ uint4 sh_fold[RS_FOLD_WARPS];   // per fold warp {rmax, top, jtop, -}
     __shared__ unsigned int sh_jmax;        // no row's jtop is larger
     __shared__ int sh_mode;                 // 0: decline the batch; 1: binary64 scores; 2: whole-number scores
@@ -321,8 +314,6 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
         if (whole) whole = token_bound + a.guard[GUARD_MAX_PD] + (unsigned long long)beta * peak_bound < (1ull << 30);
         sh_mode = ok ? (whole ? 2 : 1) : 0;
         sh_n0 = *a.n_requests;
-        sh_emin[0] = sh_emin[1] = 0x7f7fffffu;
-        sh_nlist[0] = sh_nlist[1] = 0;
         sh_jmax = (unsigned int)a.guard[GUARD_MAX_JTOP];
         for (int x = 0; x < RS_PENDING; ++x) pend[x].row = -1;
         sh_n_over = 0;
@@ -444,8 +435,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     }
     __syncthreads();
 
-    const int st = tid - RS_FOLD_THREADS - 32;      // score warps
-    const int sw_id = warp - RS_FOLD_WARPS - 1;
+    const int sw_id = warp - RS_FOLD_WARPS - 1;   // score warps
     // fold warps: thread t holds cells 2t, 2t+1, then the same 2 * RS_FOLD_THREADS further on (16-byte accesses, a warp
     // reads 512 contiguous bytes); without 16-byte accesses cells t, t + RS_FOLD_THREADS, ...
     auto cell = [&](int u) { return VEC ? 2 * tid + (u >> 1) * (2 * RS_FOLD_THREADS) + (u & 1) : tid + u * RS_FOLD_THREADS; };
@@ -574,59 +564,98 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     const unsigned long long wk = warp_min_u64(((unsigned long long)best << 32) | (unsigned int)brow);
                     if (lane == 0) sh_wkey[par][sw_id] = (unsigned int)(wk >> 32) < RS_OUT ? wk : 0xffffffffffffffffull;
                 } else {
-                    // Pass 1, binary32: a lower and an upper estimate of every row's score (the same number when
-                    // the summary gives the peak exactly).  The block's smallest upper estimate bounds which rows
-                    // can hold the smallest score; pass 2 takes the binary64 score of those rows only.
+                    // Binary64 scores, per warp.  First every row's score in binary32: a lower and an upper
+                    // estimate (the same number when the summary gives the peak exactly), kept in registers.
+                    // The warp's smallest upper estimate bounds which of its rows can hold its smallest score;
+                    // only those get the binary64 score (each operation rounded on its own), and a row that is
+                    // only bounded and passes the test is scanned.  The warps' exact best rows are compared by
+                    // the deciding warp, so the block's best row is found without a barrier among the warps.
                     auto estimate = [&](unsigned int tokens, unsigned int peak) {
                         return fmaf(betaf, fmaxf((float)peak - thetaf, 0.0f), (float)(tokens + PD));
                     };
+                    float est[RS_ROWS_PER_LANE];
                     float umin = 3.402823466e38f;
-                    auto pass1 = [&](int i) {
-                        const uint2 q = tt[i];
-                        if (q.x == RS_OUT) return CUDART_INF_F;
-                        const unsigned int up = (unsigned int)P + q.y;
-                        const uint2 x = aux[i];
-                        const unsigned int lo = (unsigned int)Dc > jst[i] ? up : max(x.x, (unsigned int)P + x.y);
-                        umin = fminf(umin, estimate(q.x, up));
-                        return estimate(q.x, lo);
-                    };
-                    for (int i = st; i < I; i += nst) pass1(i);
+                    const bool all_exact = (unsigned int)Dc > sh_jmax;   // every row's summary gives its peak: two words per row
+                    if (all_exact) {
+                        #pragma unroll
+                        for (int u = 0; u < RS_ROWS_PER_LANE; ++u) {
+                            const int i = sw_id * 32 + lane + u * nst;
+                            est[u] = CUDART_INF_F;
+                            if (i < Ip) {
+                                const uint2 q = tt[i];
+                                if (q.x != RS_OUT) est[u] = estimate(q.x, (unsigned int)P + q.y);
+                            }
+                            umin = fminf(umin, est[u]);
+                        }
+                    } else {
+                        #pragma unroll
+                        for (int u = 0; u < RS_ROWS_PER_LANE; ++u) {
+                            const int i = sw_id * 32 + lane + u * nst;
+                            est[u] = CUDART_INF_F;
+                            if (i < Ip) {
+                                const uint2 q = tt[i];
+                                if (q.x != RS_OUT) {
+                                    const unsigned int up = (unsigned int)P + q.y;
+                                    const uint2 x = aux[i];
+                                    const unsigned int lo = (unsigned int)Dc > jst[i] ? up : max(x.x, (unsigned int)P + x.y);
+                                    umin = fminf(umin, estimate(q.x, up));
+                                    est[u] = estimate(q.x, lo);
+                                }
+                            }
+                        }
+                    }
                     // estimates are >= 0 and never NaN here (fminf drops a NaN): their bit patterns order like the values
-                    const unsigned int wmin = __reduce_min_sync(0xffffffffu, __float_as_uint(umin));
-                    if (lane == 0) atomicMin(&sh_emin[par], wmin);
-                    bar_sync(BAR_SCORE, nst);
-                    const float E = __uint_as_float(sh_emin[par]);
-                    // lower_m * (1 - eps) <= E * (1 + eps) + 2 * eps * c0 for the row m of the smallest score
+                    const float E = __uint_as_float(0xffffffffu - warp_max_u32(0xffffffffu - __float_as_uint(umin)));
+                    // lower_m * (1 - eps) <= E * (1 + eps) + 2 * eps * c0 for the row m of the warp's smallest score
                     const float T = fmaf(E, 1.0f + RS_EPS, 2.0f * RS_EPS * c0f) * (1.0f + 3.0f * RS_EPS);
                     double dbs = CUDART_INF;
                     int dbi = 0x7fffffff;
-                    for (int i = st; i < I; i += nst) {
-                        if (pass1(i) > T) continue;
-                        const uint2 q = tt[i];
-                        if (q.x == RS_OUT) continue;
-                        if ((unsigned int)Dc > jst[i]) {
-                            const double sc = summary_score(q.x, (unsigned int)P + q.y, P, D, theta, beta);
-                            if (better_row(sc, i, dbs, dbi)) { dbs = sc; dbi = i; }
-                        } else {
-                            list[atomicAdd(&sh_nlist[par], 1)] = i;   // only bounded: the row itself decides
+                    bool bounded = false;   // a row of this lane passes the test but its summary only bounds its peak
+                    #pragma unroll
+                    for (int u = 0; u < RS_ROWS_PER_LANE; ++u) {
+                        if (!(est[u] > T)) {   // (never for a row that is left out: its estimate is infinite ... unless T is)
+                            const int i = sw_id * 32 + lane + u * nst;
+                            const uint2 q = i < Ip ? tt[i] : make_uint2(RS_OUT, 0u);
+                            if (q.x != RS_OUT) {
+                                if (all_exact || (unsigned int)Dc > jst[i]) {
+                                    const double sc = summary_score(q.x, (unsigned int)P + q.y, P, D, theta, beta);
+                                    if (better_row(sc, i, dbs, dbi)) { dbs = sc; dbi = i; }
+                                } else {
+                                    bounded = true;
+                                }
+                            }
                         }
                     }
-                    bar_sync(BAR_SCORE, nst);
-                    const int n_list = sh_nlist[par];
-                    for (int x = sw_id; x < n_list; x += nsw) {
-                        const int i = list[x];
-                        const unsigned int pk = scan_row(i, P, Dc);
-                        const double sc = summary_score(tt[i].x, pk, P, D, theta, beta);
-                        if (lane == 0 && better_row(sc, i, dbs, dbi)) { dbs = sc; dbi = i; }
+                    if (__any_sync(0xffffffffu, bounded)) {   // rare: the rows again, the bounded ones that pass are scanned
+                        for (int base = sw_id * 32; base < Ip; base += nst) {
+                            const int i = base + lane;
+                            const uint2 q = tt[i];
+                            bool undecided = false;
+                            if (q.x != RS_OUT && !((unsigned int)Dc > jst[i])) {
+                                const uint2 x = aux[i];
+                                undecided = !(estimate(q.x, max(x.x, (unsigned int)P + x.y)) > T);
+                            }
+                            unsigned int todo = __ballot_sync(0xffffffffu, undecided);
+                            while (todo) {
+                                const int src = __ffs(todo) - 1;
+                                todo &= todo - 1;
+                                const int row = base + src;
+                                const double sc = summary_score(tt[row].x, scan_row(row, P, Dc), P, D, theta, beta);
+                                if (lane == src && better_row(sc, row, dbs, dbi)) { dbs = sc; dbi = row; }
+                            }
+                        }
                     }
-                    // scores are >= 0: their bit patterns order like the values
+                    // the warp's smallest (score, row): scores are >= 0, their bit patterns order like the values
                     unsigned long long key = (unsigned long long)__double_as_longlong(dbs);
-                    unsigned int hi = (unsigned int)(key >> 32), lo = (unsigned int)key;
-                    unsigned int mh = __reduce_min_sync(0xffffffffu, hi);
-                    unsigned int ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
-                    int wrow = (int)__reduce_min_sync(0xffffffffu, (hi == mh && lo == ml) ? (unsigned int)dbi : 0x7fffffffu);
+                    int wrow = dbi;
+                    #pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) {
+                        const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, key, off);
+                        const int r2 = __shfl_xor_sync(0xffffffffu, wrow, off);
+                        if (k2 < key || (k2 == key && r2 < wrow)) { key = k2; wrow = r2; }
+                    }
                     if (lane == 0) {
-                        sh_wkey[par][sw_id] = ((unsigned long long)mh << 32) | ml;
+                        sh_wkey[par][sw_id] = key;
                         sh_wrow[par][sw_id] = wrow;
                     }
                 }
@@ -751,8 +780,6 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                 }
                 if (lane == 0) {
                     sh_decided[par] = stall ? 0 : 1;
-                    sh_emin[par] = 0x7f7fffffu;
-                    sh_nlist[par] = 0;
                 }
             } else if (lane == 0) {
                 sh_item[par ^ 1] = it;   // the batch has ended; the remaining folds go on
@@ -861,7 +888,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
 
 static size_t summaries_smem_bytes(int I, bool admit) {
     const size_t Ip = (size_t)((I + 31) & ~31);
-    return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + sizeof(int) + (admit ? sizeof(int) : 0));
+    return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + (admit ? sizeof(int) : 0));
 }
 
 // Score warps: about sixteen rows per score thread (measured: 4,096 instances are fastest with 8 score warps,
