@@ -90,24 +90,6 @@ __device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-// Warp-wide minimum / maximum of a 64-bit key with shuffles.  (Measured in this kernel: a redux.sync costs a warp
-// 250 to 300 cycles, five shuffle steps about half of that.)
-__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v) {
-    #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, off);
-        v = o < v ? o : v;
-    }
-    return v;
-}
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-    #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, off);
-        v = o > v ? o : v;
-    }
-    return v;
-}
 __device__ __forceinline__ unsigned int warp_max_u32(unsigned int v) {
     #pragma unroll
     for (int off = 16; off > 0; off >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, off));
@@ -416,13 +398,12 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     int out_w = -1, out_k = 0, out_P = 0, out_D = 0;
     long long out_slot = 0;
     double out_score = 0.0;
+    // (the instance's two token counts are brought up to date after the last round, from the new table rows)
     auto flush_outputs = [&]() {
         if (out_w < 0) return;
         if (lane == 0) { a.prompt[out_slot] = out_P; a.generated[out_slot] = 0; }
         if (lane == 1) { a.predicted[out_slot] = out_D; a.instance[out_slot] = out_w; }
         if (lane == 2) put_result(out_k, out_w, out_score);
-        if (lane == 3) atomicAdd(reinterpret_cast<unsigned long long*>(a.queued_p + out_w), (unsigned long long)out_P);
-        if (lane == 4) atomicAdd(reinterpret_cast<unsigned long long*>(a.current_d + out_w), (unsigned long long)out_D);
         out_w = -1;
     };
     Item nxt;               // (control warp) the arrival after the one being decided, walked to ahead of time
@@ -560,9 +541,11 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                             }
                         }
                     }
-                    // smallest (score, row) of the warp: one 64-bit key
-                    const unsigned long long wk = warp_min_u64(((unsigned long long)best << 32) | (unsigned int)brow);
-                    if (lane == 0) sh_wkey[par][sw_id] = (unsigned int)(wk >> 32) < RS_OUT ? wk : 0xffffffffffffffffull;
+                    // smallest (score, row) of the warp: the smallest score, then the first row that has it (two
+                    // warp reductions: shorter than a butterfly of shuffles over 64-bit keys, measured)
+                    const unsigned int wbest = __reduce_min_sync(0xffffffffu, best);
+                    const unsigned int wrow = __reduce_min_sync(0xffffffffu, best == wbest ? (unsigned int)brow : 0xffffffffu);
+                    if (lane == 0) sh_wkey[par][sw_id] = wbest < RS_OUT ? ((unsigned long long)wbest << 32) | wrow : 0xffffffffffffffffull;
                 } else {
                     // Binary64 scores, per warp.  First every row's score in binary32: a lower and an upper
                     // estimate (the same number when the summary gives the peak exactly), kept in registers.
@@ -701,15 +684,12 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     if (jtop == 0xffffffffu || t > top) { top = t; jtop = (unsigned int)j; }
                 }
             }
-            rmax = warp_max_u32(rmax);
-            // largest cell + step and the first step that has it: (top, ~step) as one 64-bit key
-            const unsigned long long tk = warp_max_u64(jtop != 0xffffffffu ? ((unsigned long long)top << 32) | (0xffffffffu - jtop) : 0ull);
-            const unsigned int wt = (unsigned int)(tk >> 32);
-            const unsigned int wj = tk ? 0xffffffffu - (unsigned int)tk : 0xffffffffu;
-            if (ADMIT) {
-                #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(0xffffffffu, above, off);
-            }
+            // the warp's largest cell, largest cell + step and the first step that has it (warp reductions: the fold
+            // warps are the longest chain of a round, and a butterfly of shuffles is three times as many instructions)
+            rmax = __reduce_max_sync(0xffffffffu, rmax);
+            const unsigned int wt = __reduce_max_sync(0xffffffffu, top);   // (a lane without cells has top 0 and no step)
+            const unsigned int wj = __reduce_min_sync(0xffffffffu, top == wt ? jtop : 0xffffffffu);
+            if (ADMIT) above = __reduce_add_sync(0xffffffffu, above);
             if (lane == 0) sh_fold[warp] = make_uint4(rmax, wt, wj, (unsigned int)above);
         }
         __syncthreads();   // the pass and the fold's per-warp maxima are complete
@@ -819,6 +799,15 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     }
     if (warp == RS_CONTROL_WARP) flush_outputs();
     if (overrun && tid == 0) atomicOr(a.status, PRE_ST_TIMEOUT);
+    // Every routed request adds its prompt to its instance's queued tokens and its predicted length to the tokens
+    // being decoded (Sec. 4.3.3): one reduction each per new table row, by the whole block, instead of two
+    // reductions in every round's chain.
+    __syncthreads();
+    for (long long i = tid; i < ndec; i += nthreads) {
+        const int w = a.instance[n0 + i];
+        atomicAdd(reinterpret_cast<unsigned long long*>(a.queued_p + w), (unsigned long long)a.prompt[n0 + i]);
+        atomicAdd(reinterpret_cast<unsigned long long*>(a.current_d + w), (unsigned long long)a.predicted[n0 + i]);
+    }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     // what the walker noted beyond a blocked request is decided again below and does not count here
     const long long decided = (ADMIT && blocked) ? sh_blocked_k : n_items;
@@ -894,7 +883,7 @@ static size_t summaries_smem_bytes(int I, bool admit) {
 // Score warps: about sixteen rows per score thread (measured: 4,096 instances are fastest with 8 score warps,
 // 1,024 with 2 to 4; more warps lengthen the block barriers more than they shorten the pass).
 static int summaries_score_warps(int I) {
-    int w = (I + 16 * 32 - 1) / (16 * 32);
+    int w = (I + RS_ROWS_PER_LANE * 32 - 1) / (RS_ROWS_PER_LANE * 32);
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
 
