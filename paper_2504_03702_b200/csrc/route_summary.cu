@@ -288,7 +288,9 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
         // every cell, every cell + step with a prompt added, and every token count stay below 2^32 all batch long
         const unsigned long long peak_bound = mc + a.guard[GUARD_SUM_RAMP] + (unsigned long long)H + (unsigned long long)PRE_FIELD_MAX;
         const unsigned long long token_bound = mb + a.guard[GUARD_SUM_TOKENS];
-        const bool ok = a.guard[GUARD_BAD] == 0 && peak_bound <= 0xffffffffull && token_bound < (unsigned long long)RS_OUT;
+        // (and the batch is short enough for the round counters below to be 32-bit numbers)
+        const bool ok = a.guard[GUARD_BAD] == 0 && peak_bound <= 0xffffffffull && token_bound < (unsigned long long)RS_OUT &&
+                        a.n_arrivals + (ADMIT ? a.queue_capacity : 0) < (1ll << 26);
         // Whole-number scores: with beta and theta whole numbers every term of the score is a whole number
         // below 2^53, each binary64 operation is exact, and the score is the same number in integer
         // arithmetic; it is taken in 32 bits when even the largest possible score stays below 2^30.
@@ -454,16 +456,16 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     };
     auto whole_over = [&](unsigned int peak) { return (int)peak > theta_i ? peak - (unsigned int)theta_i : 0u; };
 
-    long long ndec = 0, nfold = 0;   // decisions made, folds done: every thread keeps them
+    int ndec = 0, nfold = 0;   // decisions made, folds done: every thread keeps them
     bool stalled = false;
     bool blocked = false;            // ADMIT: a request found every instance overloaded: no more decisions, the folds go on
     // Every arrival is decided after at most RS_PENDING stalled rounds and folded RS_LAG rounds later:
     // the loop below ends by itself.  The limit only keeps a mistake in that reasoning from spinning.
-    const long long round_limit = (n_items + 2) * (RS_PENDING + 2) + 64;
+    const int round_limit = (int)((n_items + 2) * (RS_PENDING + 2) + 64);
     bool overrun = false;
-    for (long long round = 0;; ++round) {
+    for (int round = 0;; ++round) {
         if (round > round_limit) { overrun = true; break; }
-        const int par = (int)(round & 1);
+        const int par = round & 1;
         const Item it = sh_item[par];
         const bool have = it.k >= 0 && !blocked;
         if (!have && nfold == ndec) break;
@@ -478,7 +480,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
             // bounds, the arrival after this one
             flush_outputs();
             if (have) {
-                const long long d = nfold + lane;
+                const int d = nfold + lane;
                 if (lane < RS_PENDING && d < ndec) {
                     const Pending p = pend[d % RS_PENDING];
                     const unsigned int peak_lb = (unsigned int)it.Dc > p.jw ? (unsigned int)it.P + p.top_lb
@@ -681,7 +683,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     if (ADMIT) above += (long long)c[u] > a.hot;
                     rmax = max(rmax, c[u]);
                     const unsigned int t = c[u] + (unsigned int)j;
-                    if (jtop == 0xffffffffu || t > top) { top = t; jtop = (unsigned int)j; }
+                    if (t > top) { top = t; jtop = (unsigned int)j; }   // (a lane whose cells + steps are all 0 names no step)
                 }
             }
             // the warp's largest cell, largest cell + step and the first step that has it (warp reductions: the fold
@@ -803,7 +805,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     // being decoded (Sec. 4.3.3): one reduction each per new table row, by the whole block, instead of two
     // reductions in every round's chain.
     __syncthreads();
-    for (long long i = tid; i < ndec; i += nthreads) {
+    for (int i = tid; i < ndec; i += nthreads) {
         const int w = a.instance[n0 + i];
         atomicAdd(reinterpret_cast<unsigned long long*>(a.queued_p + w), (unsigned long long)a.prompt[n0 + i]);
         atomicAdd(reinterpret_cast<unsigned long long*>(a.current_d + w), (unsigned long long)a.predicted[n0 + i]);
