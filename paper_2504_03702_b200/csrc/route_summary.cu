@@ -703,10 +703,17 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                 double b1s = CUDART_INF;   // binary64 path: the pass's best score
                 unsigned int b1i = 0xffffffffu;   // whole-number path: the same without the arrival's own P + D
                 int b1r = -1;
-                {   // the best of the warps' rows: (key, row) pairs, smallest first (shuffles: a warp reduction
-                    // instruction costs a lone warp a few hundred cycles here)
+                if (whole) {
+                    // the best of the warps' rows: the smallest score, then the smallest row that has it (two warp
+                    // reductions: shorter than a butterfly of shuffles over 64-bit keys)
+                    const unsigned long long key = lane < nsw ? sh_wkey[par][lane] : 0xffffffffffffffffull;
+                    const unsigned int ks = (unsigned int)(key >> 32);
+                    const unsigned int m = __reduce_min_sync(0xffffffffu, ks);
+                    const unsigned int r = __reduce_min_sync(0xffffffffu, ks == m ? (unsigned int)key : 0xffffffffu);
+                    if (m != 0xffffffffu) { b1i = m; b1r = (int)r; }
+                } else {   // binary64 scores: (score bits, row) pairs, smallest first, by shuffles
                     unsigned long long key = lane < nsw ? sh_wkey[par][lane] : 0xffffffffffffffffull;
-                    int row = (!whole && lane < nsw) ? sh_wrow[par][lane] : 0x7fffffff;
+                    int row = lane < nsw ? sh_wrow[par][lane] : 0x7fffffff;
                     for (int off = 1; off < nsw; off <<= 1) {
                         const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, key, off);
                         const int r2 = __shfl_xor_sync(0xffffffffu, row, off);
@@ -714,9 +721,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     }
                     key = __shfl_sync(0xffffffffu, key, 0);   // lanes beyond the warps' count hold no result of their own
                     row = __shfl_sync(0xffffffffu, row, 0);
-                    if (whole) {
-                        if (key != 0xffffffffffffffffull) { b1i = (unsigned int)(key >> 32); b1r = (int)(unsigned int)key; }
-                    } else if (row != 0x7fffffff) {
+                    if (row != 0x7fffffff) {
                         b1s = __longlong_as_double((long long)key);
                         b1r = row;
                     }
