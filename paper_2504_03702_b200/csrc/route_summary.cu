@@ -266,7 +266,8 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     __shared__ Item sh_item[2];             // the arrival to decide, by round parity
     __shared__ int sh_decided[2];           // whether the round decided its arrival
     __shared__ Pending pend[RS_PENDING];
-    __shared__ unsigned long long sh_wkey[2][RS_MAX_SCORE_WARPS];   // the warps' best rows: score bits (binary64) or score << 32 | row
+    __shared__ unsigned long long sh_wkey[2][RS_MAX_SCORE_WARPS];   // binary64 scores: the warps' best rows, score bits
+    __shared__ unsigned long long sh_best[2];   // whole-number scores: the smallest score << 32 | row of all warps (atomic minimum)
     __shared__ int sh_wrow[2][RS_MAX_SCORE_WARPS];
     __shared__ uint4 sh_fold[RS_FOLD_WARPS];   // per fold warp {rmax, top, jtop, -}
     __shared__ unsigned int sh_jmax;        // no row's jtop is larger
@@ -300,6 +301,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
         sh_n0 = *a.n_requests;
         sh_jmax = (unsigned int)a.guard[GUARD_MAX_JTOP];
         for (int x = 0; x < RS_PENDING; ++x) pend[x].row = -1;
+        sh_best[0] = sh_best[1] = 0xffffffffffffffffull;
         sh_n_over = 0;
         sh_blocked = 0;
         sh_blocked_k = 0;
@@ -479,6 +481,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
             // what does not depend on the pass: the last decision's outputs, the pending rows' lower
             // bounds, the arrival after this one
             flush_outputs();
+            if (lane == 0) sh_best[par ^ 1] = 0xffffffffffffffffull;   // the next round's minimum starts afresh
             if (have) {
                 const int d = nfold + lane;
                 if (lane < RS_PENDING && d < ndec) {
@@ -543,11 +546,10 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                             }
                         }
                     }
-                    // smallest (score, row) of the warp: the smallest score, then the first row that has it (two
-                    // warp reductions: shorter than a butterfly of shuffles over 64-bit keys, measured)
+                    // The smallest (score, row) of all score warps: the warp's smallest score by a warp reduction, then
+                    // the lanes that hold it (one, but for ties) take the block's minimum of score << 32 | row.
                     const unsigned int wbest = __reduce_min_sync(0xffffffffu, best);
-                    const unsigned int wrow = __reduce_min_sync(0xffffffffu, best == wbest ? (unsigned int)brow : 0xffffffffu);
-                    if (lane == 0) sh_wkey[par][sw_id] = wbest < RS_OUT ? ((unsigned long long)wbest << 32) | wrow : 0xffffffffffffffffull;
+                    if (best == wbest && wbest < RS_OUT) atomicMin(&sh_best[par], ((unsigned long long)best << 32) | (unsigned int)brow);
                 } else {
                     // Binary64 scores, per warp.  First every row's score in binary32: a lower and an upper
                     // estimate (the same number when the summary gives the peak exactly), kept in registers.
@@ -704,13 +706,9 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                 unsigned int b1i = 0xffffffffu;   // whole-number path: the same without the arrival's own P + D
                 int b1r = -1;
                 if (whole) {
-                    // the best of the warps' rows: the smallest score, then the smallest row that has it (two warp
-                    // reductions: shorter than a butterfly of shuffles over 64-bit keys)
-                    const unsigned long long key = lane < nsw ? sh_wkey[par][lane] : 0xffffffffffffffffull;
-                    const unsigned int ks = (unsigned int)(key >> 32);
-                    const unsigned int m = __reduce_min_sync(0xffffffffu, ks);
-                    const unsigned int r = __reduce_min_sync(0xffffffffu, ks == m ? (unsigned int)key : 0xffffffffu);
-                    if (m != 0xffffffffu) { b1i = m; b1r = (int)r; }
+                    // the score warps took the minimum over all of them already
+                    const unsigned long long key = sh_best[par];
+                    if (key != 0xffffffffffffffffull) { b1i = (unsigned int)(key >> 32); b1r = (int)(unsigned int)key; }
                 } else {   // binary64 scores: (score bits, row) pairs, smallest first, by shuffles
                     unsigned long long key = lane < nsw ? sh_wkey[par][lane] : 0xffffffffffffffffull;
                     int row = lane < nsw ? sh_wrow[par][lane] : 0x7fffffff;
