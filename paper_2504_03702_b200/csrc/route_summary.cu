@@ -916,6 +916,7 @@ template <bool ADMIT>
 static cudaError_t summaries_configure_one(pre_ctx* ctx, size_t limit, size_t* smem_out) {
     const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
     *smem_out = 0;
+    if (I > RS_MAX_SCORE_WARPS * 32 * RS_ROWS_PER_LANE) return cudaSuccess;   // more rows than the score lanes take
     const void* fn = summaries_kernel_for<ADMIT>(H, I);
     cudaFuncAttributes attr;
     cudaError_t e = cudaFuncGetAttributes(&attr, fn);
