@@ -185,6 +185,21 @@ def test_many_instances_close_to_the_shared_memory_limit():
     route_and_compare(wl, ap, ad)
 
 
+@pytest.mark.parametrize("n_inst", [40, 700, 2100])
+@pytest.mark.parametrize("path", [B.ROUTE_SUMMARY, B.ROUTE_SCAN])
+def test_equal_scores_go_to_the_lowest_index(n_inst, path):
+    """Empty instances and identical arrivals: every score is shared by many rows, in the same lane, in
+    other lanes of the warp and in other warps, and the lowest index among them has to win each time
+    (Sec. 4.3.3 names no tie rule; the oracle's argmin takes the first)."""
+    wl = W.make_random(3, n_inst, 64, 0, 0, capacity=100000)
+    n = 3 * n_inst + 17
+    ap = np.full(n, 10, dtype=np.int32)
+    ad = np.full(n, 5, dtype=np.int32)
+    wl.max_requests = n
+    ref = route_and_compare(wl, ap, ad, path=path)
+    assert ref.instance[:n].tolist() == [k % n_inst for k in range(n)]
+
+
 def test_streaming_ticks_on_both_kernels():
     """Route, step, route ... over the first ticks of the streaming configuration, both kernels in turn."""
     wl = W.make_config(4, n_ticks=4)
