@@ -506,11 +506,16 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     const int K = P - theta_i;
                     if ((unsigned int)Dc > sh_jmax) {
                         // every row's summary gives its peak: two words per row
-                        #pragma unroll 4
-                        for (int i = sw_id * 32 + lane; i < Ip; i += nst) {
-                            const uint2 q = tt[i];
-                            const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
-                            if (t < best) { best = t; brow = i; }
+                        // (a trip count known to the compiler, unrolled by eight: measured against a run-time trip
+                        // count, 4 and 16; the host gives a lane RS_ROWS_PER_LANE rows at most)
+                        #pragma unroll 8
+                        for (int u = 0; u < RS_ROWS_PER_LANE; ++u) {
+                            const int i = sw_id * 32 + lane + u * nst;
+                            if (i < Ip) {
+                                const uint2 q = tt[i];
+                                const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
+                                if (t < best) { best = t; brow = i; }
+                            }
                         }
                     } else {
                         // Some rows are only bounded.  First the smallest upper bound among the warp's rows
