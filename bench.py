@@ -41,19 +41,19 @@ METRIC_STREAM = "routes/sec over the whole stream (decode step + routing of the 
 # table and moves the tiles' lists; most of the 64 MiB of maps is still in L2 when the launch ends, which is why
 # its figure is below the algorithmic bytes.  pre_step: its two kernels added.
 # profiles/ncu_full_tick_scaler_refine_config3.txt: refinement and the fused tick (two kernels added).
-ROUTE_DRAM_READ = {3: 67319296}
+ROUTE_DRAM_READ = {3: 67318016}
 # profiles/ncu_dram_route_summary_kernels_config3_full_batch.txt: both kernels of the summary router on the full
 # batch (the traffic does not grow in proportion to the batch, so the figure is used for the full batch only)
-ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67724032 + 106240 + 55568128 + 5410048}
+ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67724544 + 92160 + 55802880 + 5716480}
 # warp instructions per arrival of pre_route_summaries (smsp__inst_executed.sum of the 2,048-arrival capture in
-# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 10,257,626 / 2,048)
-ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 10257626 / 2048}
-ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 493312 / 256}
-ANTICIPATE_DRAM_TRAFFIC = {3: 33807872 + 19569920}
-STEP_DRAM_TRAFFIC = {3: 33668864 + 67196160 + 9327104}
+# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 9,795,476 / 2,048)
+ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 9795476 / 2048}
+ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 645632 / 256}
+ANTICIPATE_DRAM_TRAFFIC = {3: 33810688 + 20138496}
+STEP_DRAM_TRAFFIC = {3: 33669120 + 67195904 + 11600896}
 SCALER_DRAM_TRAFFIC = {3: 67127552 + 291584}   # profiles/ncu_full_scaler_rows_config3.txt
-REFINE_DRAM_TRAFFIC = {3: 44152320 + 32768}
-TICK_DRAM_TRAFFIC = {3: 44136704 + 63488 + 67200000 + 9139712}
+REFINE_DRAM_TRAFFIC = {3: 44151808 + 26368}
+TICK_DRAM_TRAFFIC = {3: 44136704 + 44032 + 67199744 + 9539584}
 
 
 def measured_peak_gbs():
