@@ -20,13 +20,18 @@
 //   pre_route_summaries  routes the batch with ONE block: summaries in shared memory, no exchange
 //                        between blocks, hence no device-side wait on another block anywhere.
 //
-// pre_route_summaries works in rounds, one block barrier per round, two groups of warps:
-//   score warps: decide one arrival per round.  Every row's score comes from its summary; the
-//                last warp to finish takes the block's best row, writes the decision and hands
-//                the row to the fold warps.
-//   fold warps:  add an arrival to its row in the map (Sec. 4.3.1 update) and take the row's new
-//                summary in the same pass - RS_LAG rounds after the decision, so that the row's
-//                cells can be fetched a round ahead and no decision waits for a fold.
+// pre_route_summaries works in rounds, one arrival and two block barriers per round, three groups of warps:
+//   score warps:  every row's score for the arrival from its summary; the warp's smallest score by a
+//                 warp reduction, the block's smallest (score, row) by a shared-memory atomic minimum
+//                 (whole-number scores) or one (score, row) per warp (binary64 scores);
+//   control warp: before the first barrier it writes the last decision's outputs, takes the pending
+//                 rows' lower bounds and walks to the next well-formed arrival; between the barriers
+//                 it decides: the pass's best row unless a pending row could do better;
+//   fold warps:   add an arrival to its row in the map (Sec. 4.3.1 update) and take the row's new
+//                 summary in the same pass - RS_LAG rounds after the decision, so that the row's
+//                 cells can be fetched a round ahead and no decision waits for a fold.
+// The instances' token counts (Sec. 4.3.3: queued prompt tokens, tokens being decoded) are brought up
+// to date once, after the last round, from the new table rows.
 // Between its decision and its fold a row is "pending": it is left out of the scoring pass and
 // represented by a lower bound of its score (its token count is exact at once; the cell that
 // held `top` only grows).  A pending row whose lower bound could win makes the round a stall:
