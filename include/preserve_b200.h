@@ -137,8 +137,9 @@ int pre_anticipate_static(int32_t n_instances, int32_t horizon, const int32_t* d
  * kernel keeps four numbers per row (largest cell, largest cell + step and where it sits, cell 0)
  * that give the peak of almost every row for any arrival without reading the row, scans the few
  * rows they leave undecided, routes with a single block and waits for nobody; it takes the batch
- * when the context's instances fit its shared memory and every value stays below 2^32 during the
- * batch, which it checks on the device.  Otherwise the scanning kernel routes: it reads every cell
+ * when the context's instances fit its shared memory, every value stays below 2^32 during the
+ * batch and the batch (with the waiting requests of pre_route_admit) has fewer than 2^26 entries,
+ * which it checks on the device.  Otherwise the scanning kernel routes: it reads every cell
  * for every arrival, its blocks exchange their best instances through device memory and wait
  * for one another a bounded number of polls.  If such a wait runs out (PRE_ETIMEOUT from
  * pre_status; it should never happen on a GPU that runs the kernel alone), the blocks agree on
