@@ -48,7 +48,7 @@ namespace {
 constexpr int RS_FOLD_WARPS = 8;
 constexpr int RS_FOLD_THREADS = 32 * RS_FOLD_WARPS;
 constexpr int RS_CONTROL_WARP = RS_FOLD_WARPS;     // the warp after the fold warps decides; the score warps follow it
-constexpr int RS_MAX_SCORE_WARPS = 23;
+constexpr int RS_MAX_SCORE_WARPS = 10;      // 640 threads with the fold and control warps: 96 registers per thread, no spills
 constexpr int RS_MAX_THREADS = RS_FOLD_THREADS + 32 + 32 * RS_MAX_SCORE_WARPS;
 #ifndef PRE_RS_LAG
 #define PRE_RS_LAG 3
@@ -258,9 +258,18 @@ struct RouteSumArgs {
 // ADMIT adds the admission queue of Sec. 4.3.3: the requests that were waiting come first; a request that
 // finds every instance overloaded (the scaler's criterion of Sec. 4.3.2: more than `many` steps of the
 // row above `hot`) is not routed and the batch stops there: what is left waits or is turned away.
-// MAXT: the largest block this instantiation is launched with (a smaller one leaves the compiler more registers).
-template <int CPT, bool VEC, bool ADMIT, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArgs a) {
+// KIND: which scores the instantiation takes, chosen by the host from beta and theta (measured: with both kinds in
+// one kernel and the choice made at run time the whole-number rounds take 6 % longer, 8 % with the queue):
+//   RS_WHOLE      whole-number scores (beta and theta whole numbers); the kernel declines the batch when the
+//                 device-side bounds do not keep every score below 2^30;
+//   RS_WHOLE_BIG  the same for more than RS_ROWS_PER_LANE rows per score lane (contexts of more than 5,120
+//                 instances): the pass goes on beyond its unrolled part;
+//   RS_BINARY64   binary64 scores, RS_ROWS_PER_LANE rows per score lane at most.
+constexpr int RS_WHOLE = 0, RS_WHOLE_BIG = 1, RS_BINARY64 = 2;
+template <int CPT, bool VEC, bool ADMIT, int KIND>
+__global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const RouteSumArgs a) {
+    constexpr bool BIG = KIND == RS_WHOLE_BIG;
+    constexpr bool whole = KIND != RS_BINARY64;
     extern __shared__ __align__(16) unsigned char rs_smem[];
     const int I = a.I, H = a.H;
     const int Ip = (I + 31) & ~31;
@@ -276,7 +285,7 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
     __shared__ int sh_wrow[2][RS_MAX_SCORE_WARPS];
     __shared__ uint4 sh_fold[RS_FOLD_WARPS];   // per fold warp {rmax, top, jtop, -}
     __shared__ unsigned int sh_jmax;        // no row's jtop is larger
-    __shared__ int sh_mode;                 // 0: decline the batch; 1: binary64 scores; 2: whole-number scores
+    __shared__ int sh_mode;                 // 0: decline the batch
     __shared__ long long sh_n0;
     __shared__ int sh_arr_p[64], sh_arr_d[64];   // the arrivals around the walker's position
     __shared__ int sh_n_over;               // ADMIT: rows known to be overloaded
@@ -300,9 +309,9 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
         // Whole-number scores: with beta and theta whole numbers every term of the score is a whole number
         // below 2^53, each binary64 operation is exact, and the score is the same number in integer
         // arithmetic; it is taken in 32 bits when even the largest possible score stays below 2^30.
-        bool whole = ok && beta == floor(beta) && theta == floor(theta) && beta <= 1048576.0 && theta < 1073741824.0;
-        if (whole) whole = token_bound + a.guard[GUARD_MAX_PD] + (unsigned long long)beta * peak_bound < (1ull << 30);
-        sh_mode = ok ? (whole ? 2 : 1) : 0;
+        bool exact = ok && beta == floor(beta) && theta == floor(theta) && beta <= 1048576.0 && theta < 1073741824.0;
+        if (exact) exact = token_bound + a.guard[GUARD_MAX_PD] + (unsigned long long)beta * peak_bound < (1ull << 30);
+        sh_mode = ok && (exact || !whole) ? 1 : 0;
         sh_n0 = *a.n_requests;
         sh_jmax = (unsigned int)a.guard[GUARD_MAX_JTOP];
         for (int x = 0; x < RS_PENDING; ++x) pend[x].row = -1;
@@ -318,7 +327,6 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
         if (tid == 0) *a.handled = 0;
         return;
     }
-    const bool whole = sh_mode == 2;
     const unsigned int beta_i = whole ? (unsigned int)beta : 0u;
     const int theta_i = whole ? (int)theta : 0;
     for (int i = tid; i < Ip; i += nthreads) {
@@ -512,11 +520,18 @@ __global__ void __launch_bounds__(MAXT, 1) pre_route_summaries(const RouteSumArg
                     if ((unsigned int)Dc > sh_jmax) {
                         // every row's summary gives its peak: two words per row
                         // (a trip count known to the compiler, unrolled by eight: measured against a run-time trip
-                        // count, 4 and 16; the host gives a lane RS_ROWS_PER_LANE rows at most)
+                        // count and against 4 and 16)
                         #pragma unroll 8
                         for (int u = 0; u < RS_ROWS_PER_LANE; ++u) {
                             const int i = sw_id * 32 + lane + u * nst;
                             if (i < Ip) {
+                                const uint2 q = tt[i];
+                                const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
+                                if (t < best) { best = t; brow = i; }
+                            }
+                        }
+                        if (BIG) {   // the lane's rows beyond those
+                            for (int i = sw_id * 32 + lane + RS_ROWS_PER_LANE * nst; i < Ip; i += nst) {
                                 const uint2 q = tt[i];
                                 const unsigned int t = q.x + beta_i * (unsigned int)max((int)q.y + K, 0);
                                 if (t < best) { best = t; brow = i; }
@@ -895,39 +910,48 @@ static size_t summaries_smem_bytes(int I, bool admit) {
     return Ip * (2 * sizeof(uint2) + sizeof(uint32_t) + (admit ? sizeof(int) : 0));
 }
 
-// Score warps: about sixteen rows per score thread (measured: 4,096 instances are fastest with 8 score warps,
-// 1,024 with 2 to 4; more warps lengthen the block barriers more than they shorten the pass).
+// Score warps: sixteen rows per score thread up to RS_MAX_SCORE_WARPS warps, more rows per thread beyond (measured:
+// 4,096 instances are fastest with 8 score warps, 1,024 with 2 to 4; more warps lengthen the block barriers more
+// than they shorten the pass, and a block of more than 640 threads leaves 64 registers per thread: 70 % slower).
 static int summaries_score_warps(int I) {
     int w = (I + RS_ROWS_PER_LANE * 32 - 1) / (RS_ROWS_PER_LANE * 32);
     return w < 1 ? 1 : (w > RS_MAX_SCORE_WARPS ? RS_MAX_SCORE_WARPS : w);
 }
 
-constexpr int RS_SMALL_THREADS = 640;   // blocks of up to 10 score warps get the instantiation with more registers
-
-template <int CPT, bool ADMIT>
-static const void* summaries_kernel(bool vec, bool small) {
-    if (small)
-        return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT, RS_SMALL_THREADS>
-                   : (const void*)pre_route_summaries<CPT, false, ADMIT, RS_SMALL_THREADS>;
-    return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT, RS_MAX_THREADS>
-               : (const void*)pre_route_summaries<CPT, false, ADMIT, RS_MAX_THREADS>;
+// beta and theta = t_mem * M whole numbers of moderate size: the scores can be taken in whole-number arithmetic
+static bool summaries_whole_numbers(const pre_ctx* ctx) {
+    const double beta = ctx->cfg.beta, theta = ctx->theta;
+    return beta == floor(beta) && theta == floor(theta) && beta <= 1048576.0 && theta < 1073741824.0;
 }
-template <bool ADMIT>
-static const void* summaries_kernel_for(int H, int I) {
+
+template <int CPT, bool ADMIT, int KIND>
+static const void* summaries_kernel(bool vec) {
+    return vec ? (const void*)pre_route_summaries<CPT, true, ADMIT, KIND> : (const void*)pre_route_summaries<CPT, false, ADMIT, KIND>;
+}
+template <bool ADMIT, int KIND>
+static const void* summaries_kernel_of_kind(int H) {
     const bool vec = (H & 1) == 0;
-    const bool small = RS_FOLD_THREADS + 32 + 32 * summaries_score_warps(I) <= RS_SMALL_THREADS;
-    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4, ADMIT>(vec, small);
-    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8, ADMIT>(vec, small);
-    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16, ADMIT>(vec, small);
-    return summaries_kernel<32, ADMIT>(vec, small);
+    if (H <= 4 * RS_FOLD_THREADS) return summaries_kernel<4, ADMIT, KIND>(vec);
+    if (H <= 8 * RS_FOLD_THREADS) return summaries_kernel<8, ADMIT, KIND>(vec);
+    if (H <= 16 * RS_FOLD_THREADS) return summaries_kernel<16, ADMIT, KIND>(vec);
+    return summaries_kernel<32, ADMIT, KIND>(vec);
+}
+// nullptr: no instantiation takes this context (binary64 scores with more than RS_ROWS_PER_LANE rows per score lane)
+template <bool ADMIT>
+static const void* summaries_kernel_for(const pre_ctx* ctx) {
+    const int H = ctx->cfg.horizon, I = ctx->cfg.n_instances;
+    const bool big = I > RS_ROWS_PER_LANE * 32 * RS_MAX_SCORE_WARPS;
+    if (summaries_whole_numbers(ctx))
+        return big ? summaries_kernel_of_kind<ADMIT, RS_WHOLE_BIG>(H) : summaries_kernel_of_kind<ADMIT, RS_WHOLE>(H);
+    return big ? nullptr : summaries_kernel_of_kind<ADMIT, RS_BINARY64>(H);
 }
 
 template <bool ADMIT>
 static cudaError_t summaries_configure_one(pre_ctx* ctx, size_t limit, size_t* smem_out) {
-    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    const int I = ctx->cfg.n_instances;
     *smem_out = 0;
-    if (I > RS_MAX_SCORE_WARPS * 32 * RS_ROWS_PER_LANE) return cudaSuccess;   // more rows than the score lanes take
-    const void* fn = summaries_kernel_for<ADMIT>(H, I);
+    const void* fn = summaries_kernel_for<ADMIT>(ctx);
+    if (fn == nullptr) return cudaSuccess;
     cudaFuncAttributes attr;
     cudaError_t e = cudaFuncGetAttributes(&attr, fn);
     if (e != cudaSuccess) return e;
@@ -984,7 +1008,7 @@ static void fill_summary_args(pre_ctx* ctx, SumArgs& p, RouteSumArgs& a, const i
 
 template <bool ADMIT>
 static cudaError_t launch_summary_kernels(pre_ctx* ctx, const SumArgs& p, const RouteSumArgs& a, cudaStream_t s) {
-    const int I = ctx->cfg.n_instances, H = ctx->cfg.horizon;
+    const int I = ctx->cfg.n_instances;
     cudaError_t e = cudaMemsetAsync(ctx->d_rs_guard, 0, 8 * sizeof(unsigned long long), s);
     if (e != cudaSuccess) return e;
     const int rows_per_block = SUM_THREADS / 32;
@@ -992,7 +1016,7 @@ static cudaError_t launch_summary_kernels(pre_ctx* ctx, const SumArgs& p, const 
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     void* params[] = {(void*)&a};
-    return cudaLaunchKernel(summaries_kernel_for<ADMIT>(H, I), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
+    return cudaLaunchKernel(summaries_kernel_for<ADMIT>(ctx), dim3(1), dim3(RS_FOLD_THREADS + 32 + 32 * a.score_warps), params,
                             ADMIT ? ctx->route_summary_smem_admit : ctx->route_summary_smem, s);
 }
 
