@@ -1039,9 +1039,9 @@ static void fill_route_args(RouteArgs& a, pre_ctx* ctx, const int32_t* arr_promp
 }
 
 // PRE_ROUTE_AUTO takes the summary kernel when its scores are whole numbers (beta and t_mem * M whole: one
-// integer pass per arrival); with binary64 scores its chains of binary64 operations make it no faster than the
-// scanning kernel (measured: 3.28 against 3.11 us per arrival on 4,096 x 2,048), so it runs them only when it is
-// selected outright.
+// integer pass per arrival); with binary64 scores its chains of binary64 operations leave it level with the
+// scanning kernel (measured: 2.83 against 3.12 us per arrival on 4,096 x 2,048 instances x steps, 2.57 against
+// 2.43 on 1,024 x 1,024), so it runs them only when it is selected outright.
 static bool pre_route_summary_wanted(const pre_ctx* ctx) {
     if (ctx->route_path == PRE_ROUTE_SCAN) return false;
     if (ctx->route_path == PRE_ROUTE_SUMMARY) return true;
