@@ -157,6 +157,18 @@ def test_values_that_could_leave_32_bits_go_to_the_scanning_kernel():
     route_and_compare(wl, (ap // 1000).astype(np.int32), ad)
 
 
+def test_whole_number_scores_that_could_reach_2_to_the_30_go_to_the_scanning_kernel():
+    """beta and theta are whole numbers, so the context gets the whole-number kind of the summary kernel; with
+    beta = 4096 and peaks around 2^19 the score bound passes 2^30 and the kernel declines on the device."""
+    wl = W.make_random(97, 25, 40, 600, 0, max_prompt=2 ** 16, max_output=60, capacity=10 ** 5, beta=4096.0)
+    rng = np.random.default_rng(15)
+    ap = rng.integers(2 ** 12, 2 ** 14, 120).astype(np.int32)
+    ad = rng.integers(1, 80, 120).astype(np.int32)
+    wl.max_requests = 600 + 120
+    ref = route_and_compare(wl, ap, ad)
+    assert ref.curves.max() * 4096.0 > 2.0 ** 30, "the case was meant to pass the whole-number bound"
+
+
 def test_selecting_the_kernel():
     wl = W.make_random(93, 20000, 4, 100, 0)
     st = DeviceState.from_workload(wl)
@@ -174,6 +186,22 @@ def test_selecting_the_kernel():
     wl.max_requests = 2300
     for path in (B.ROUTE_AUTO, B.ROUTE_SCAN, B.ROUTE_SUMMARY):
         route_and_compare(wl, ap, ad, path=path)
+
+
+def test_many_instances_with_binary64_scores_take_the_scanning_kernel():
+    """More than 5,120 instances give a score lane more rows than the binary64 kind of the summary kernel
+    keeps in registers: selecting that kernel outright is refused, the default routes with the other."""
+    wl = W.make_random(96, 6000, 8, 20000, 0, max_prompt=100, max_output=20, beta=0.75)
+    st = DeviceState.from_workload(wl)
+    assert B.pre_route_select(st.ctx, B.ROUTE_SUMMARY) == B.PRE_ESIZE
+    st.close()
+    rng = np.random.default_rng(14)
+    ap = rng.integers(0, 100, 200).astype(np.int32)
+    ad = rng.integers(1, 20, 200).astype(np.int32)
+    wl.max_requests = 20200
+    route_and_compare(wl, ap, ad, path=B.ROUTE_AUTO)
+    wl.beta = 2.0      # whole-number scores: the summary kernel takes this many instances
+    route_and_compare(wl, ap, ad, path=B.ROUTE_SUMMARY)
 
 
 def test_many_instances_close_to_the_shared_memory_limit():
