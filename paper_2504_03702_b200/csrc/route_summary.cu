@@ -434,6 +434,9 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
     __syncthreads();
 
     const int sw_id = warp - RS_FOLD_WARPS - 1;   // score warps
+    // ADMIT: the overload level against 32-bit cells (a negative level: every cell is above it)
+    const int hot_all = (ADMIT && a.hot < 0) ? 1 : 0;
+    const unsigned int hot_u = a.hot < 0 ? 0u : (a.hot > 0xffffffffLL ? 0xffffffffu : (unsigned int)a.hot);
     // fold warps: thread t holds cells 2t, 2t+1, then the same 2 * RS_FOLD_THREADS further on (16-byte accesses, a warp
     // reads 512 contiguous bytes); without 16-byte accesses cells t, t + RS_FOLD_THREADS, ...
     auto cell = [&](int u) { return VEC ? 2 * tid + (u >> 1) * (2 * RS_FOLD_THREADS) + (u & 1) : tid + u * RS_FOLD_THREADS; };
@@ -707,7 +710,7 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
             for (int u = 0; u < CPT; ++u) {   // a thread's steps ascend with u
                 const int j = cell(u);
                 if (j < H) {
-                    if (ADMIT) above += (long long)c[u] > a.hot;
+                    if (ADMIT) above += hot_all | (c[u] > hot_u);
                     rmax = max(rmax, c[u]);
                     const unsigned int t = c[u] + (unsigned int)j;
                     if (t > top) { top = t; jtop = (unsigned int)j; }   // (a lane whose cells + steps are all 0 names no step)
