@@ -375,20 +375,23 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
         }
         cp_async_commit();
     };
-    long long cursor = 0, entered = 0;   // (control warp, all lanes alike) items looked at, requests found
-    long long first_bad = 0x7fffffffffffffffLL, first_full = 0x7fffffffffffffffLL;   // the first items dropped as malformed / for a full table
+    // (32-bit numbers: the batch has fewer than 2^26 items, or the kernel has declined it above)
+    const int items = (int)n_items, waiting = (int)q_len;
+    const int room_i = room > 0x7fffffffLL ? 0x7fffffff : (int)room;
+    int cursor = 0, entered = 0;   // (control warp, all lanes alike) items looked at, requests found
+    int first_bad = 0x7fffffff, first_full = 0x7fffffff;   // the first items dropped as malformed / for a full table
     auto walk_next = [&]() {
         Item it;
         it.P = it.D = it.Dc = 0;
         it.k = -1;
-        while (cursor < n_items) {
+        while (cursor < items) {
             int P, D;
-            if (ADMIT && cursor < q_len) {
+            if (ADMIT && cursor < waiting) {
                 const long long at = (q_head + cursor) % a.queue_capacity;
                 P = a.queue_prompt[at];
                 D = a.queue_predicted[at];
             } else {
-                const long long ac = cursor - q_len;
+                const int ac = cursor - waiting;
                 if ((ac & 31) == 0) {   // a new chunk: its copy was started a chunk ago; start the next one
                     asm volatile("cp.async.wait_group 0;" ::: "memory");
                     __syncwarp();
@@ -398,14 +401,14 @@ __global__ void __launch_bounds__(RS_MAX_THREADS, 1) pre_route_summaries(const R
                 D = sh_arr_d[ac & 63];
             }
             const bool bad = P < 0 || D < 1 || P > PRE_FIELD_MAX || D > PRE_FIELD_MAX;
-            if (bad || entered >= room) {
+            if (bad || entered >= room_i) {
                 if (bad && cursor < first_bad) first_bad = cursor;
                 if (!bad && cursor < first_full) first_full = cursor;
                 if (lane == 0) put_result(cursor, -1, 0.0);
                 ++cursor;
                 continue;
             }
-            it.P = P; it.D = D; it.Dc = D < H ? D : H; it.k = (int)cursor;
+            it.P = P; it.D = D; it.Dc = D < H ? D : H; it.k = cursor;
             ++cursor; ++entered;
             break;
         }
