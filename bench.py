@@ -41,19 +41,19 @@ METRIC_STREAM = "routes/sec over the whole stream (decode step + routing of the 
 # table and moves the tiles' lists; most of the 64 MiB of maps is still in L2 when the launch ends, which is why
 # its figure is below the algorithmic bytes.  pre_step: its two kernels added.
 # profiles/ncu_full_tick_scaler_refine_config3.txt: refinement and the fused tick (two kernels added).
-ROUTE_DRAM_READ = {3: 67317504}
+ROUTE_DRAM_READ = {3: 67322880}
 # profiles/ncu_dram_route_summary_kernels_config3_full_batch.txt: both kernels of the summary router on the full
 # batch (the traffic does not grow in proportion to the batch, so the figure is used for the full batch only)
-ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67726592 + 323072 + 56641024 + 6615808}
+ROUTE_SUMMARY_DRAM_TRAFFIC = {(3, 65536): 67724288 + 116224 + 55949824 + 5290240}
 # warp instructions per arrival of pre_route_summaries (smsp__inst_executed.sum of the 2,048-arrival capture in
-# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 9,455,912 / 2,048)
-ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 9455912 / 2048}
-ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 640000 / 256}
-ANTICIPATE_DRAM_TRAFFIC = {3: 33807872 + 20092928}
-STEP_DRAM_TRAFFIC = {3: 33669120 + 67196160 + 9998592}
+# profiles/ncu_full_step_kernels_config3_2048_arrivals.txt: 9,365,991 / 2,048)
+ROUTE_SUMMARY_WARP_INSTRUCTIONS_PER_ARRIVAL = {3: 9365991 / 2048}
+ROUTE_DRAM_WRITE_PER_ARRIVAL = {3: 679168 / 256}
+ANTICIPATE_DRAM_TRAFFIC = {3: 33808640 + 21654272}
+STEP_DRAM_TRAFFIC = {3: 33668864 + 67196416 + 8912640}
 SCALER_DRAM_TRAFFIC = {3: 67127552 + 291584}   # profiles/ncu_full_scaler_rows_config3.txt
-REFINE_DRAM_TRAFFIC = {3: 44151040 + 26624}
-TICK_DRAM_TRAFFIC = {3: 44138752 + 43264 + 67199488 + 9040640}
+REFINE_DRAM_TRAFFIC = {3: 44151040 + 25344}
+TICK_DRAM_TRAFFIC = {3: 44137216 + 46080 + 67199744 + 9207552}
 
 
 def measured_peak_gbs():
